@@ -1,0 +1,347 @@
+"""Pins for the CPU checker: closed forms, library special cases, invariants, brute force.
+
+Each test is chosen so that a plausible slip in the checker (dropped term, wrong sign or
+index, transposed operand, off-by-one position) fails at least one of them.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+from oracle import mdi_oracle as O
+from paper_2505_18164_b200 import inputs as I
+from helpers import make_oracle, tiny_shape
+
+rng = np.random.default_rng(1234)
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ---------------- elementary operations -----------------------------------------------------
+
+def test_linear_brute_force_and_torch():
+    W = rng.standard_normal((5, 7)).astype(np.float32)
+    b = rng.standard_normal(5).astype(np.float32)
+    X = rng.standard_normal((3, 7)).astype(np.float32)
+    Y = O.linear(W, b, X)
+    ref = np.zeros((3, 5))
+    for t in range(3):
+        for o in range(5):
+            ref[t, o] = sum(float(W[o, i]) * float(X[t, i]) for i in range(7)) + float(b[o])
+    assert np.abs(Y - ref).max() < 1e-6
+    Yt = F.linear(torch.from_numpy(X).double(), torch.from_numpy(W).double(), torch.from_numpy(b).double())
+    assert np.abs(Y - Yt.numpy()).max() < 1e-6
+    assert np.abs(O.linear(W, None, X) - (ref - b)).max() < 1e-6
+
+
+def test_linear_bf16_weights_are_widened_exactly():
+    Wf = rng.standard_normal((4, 8)).astype(np.float32)
+    bits = (Wf.view(np.uint32) >> 16).astype(np.uint16)          # truncate: any bf16 pattern will do
+    X = rng.standard_normal((2, 8)).astype(np.float32)
+    Wexact = (bits.astype(np.uint32) << 16).view(np.float32)
+    assert np.array_equal(O.linear(bits, None, X), O.linear(Wexact, None, X))
+
+
+def test_layernorm_closed_forms_and_torch():
+    d, eps = 48, 1e-5
+    x = (rng.standard_normal(d) * 3 + 1).astype(np.float32)
+    ones, zeros = np.ones(d, np.float32), np.zeros(d, np.float32)
+    y = O.layernorm(x, ones, zeros, eps).astype(np.float64)
+    var = x.astype(np.float64).var()
+    assert abs(y.mean()) < 1e-6
+    assert abs(y.var() - var / (var + eps)) < 1e-6
+    g = rng.standard_normal(d).astype(np.float32)
+    b = rng.standard_normal(d).astype(np.float32)
+    const = np.full(d, 2.5, np.float32)
+    assert np.allclose(O.layernorm(const, g, b, eps), b, atol=1e-7)  # constant input -> offset
+    yt = F.layer_norm(torch.from_numpy(x).double(), (d,), torch.from_numpy(g).double(),
+                      torch.from_numpy(b).double(), eps).numpy()
+    assert np.abs(O.layernorm(x, g, b, eps) - yt).max() < 1e-6
+
+
+def test_rmsnorm_closed_form_and_torch():
+    d, eps = 40, 1e-5
+    g = rng.standard_normal(d).astype(np.float32)
+    e = np.zeros(d, np.float32)
+    e[7] = 1.0
+    y = O.rmsnorm(e, g, eps)
+    expect = np.zeros(d)
+    expect[7] = math.sqrt(d) * g[7] / math.sqrt(1 + eps * d)
+    assert np.abs(y - expect).max() < 1e-6
+    x = rng.standard_normal(d).astype(np.float32)
+    yt = F.rms_norm(torch.from_numpy(x).double(), (d,), torch.from_numpy(g).double(), eps).numpy()
+    assert np.abs(O.rmsnorm(x, g, eps) - yt).max() < 1e-6
+
+
+def test_activations_values_and_torch():
+    assert O.gelu_tanh(0.0) == 0.0 and O.gelu_erf(0.0) == 0.0 and O.silu(0.0) == 0.0
+    assert abs(O.gelu_erf(1.0) - 0.8413447460685429) < 1e-12     # Phi(1)
+    assert abs(O.gelu_erf(-1.0) + 0.15865525393145707) < 1e-12   # -(1 - Phi(1))
+    assert abs(O.silu(1.0) - 1 / (1 + math.exp(-1))) < 1e-15
+    assert abs(O.gelu_tanh(20.0) - 20.0) < 1e-12 and abs(O.gelu_tanh(-20.0)) < 1e-12
+    assert abs(O.silu(40.0) - 40.0) < 1e-12 and abs(O.silu(-40.0)) < 1e-12
+    xs = torch.linspace(-6, 6, 101, dtype=torch.float64)
+    gt = F.gelu(xs, approximate="tanh").numpy()
+    ge = F.gelu(xs).numpy()
+    si = F.silu(xs).numpy()
+    for i, x in enumerate(xs.tolist()):
+        assert abs(O.gelu_tanh(x) - gt[i]) < 1e-12
+        assert abs(O.gelu_erf(x) - ge[i]) < 1e-12
+        assert abs(O.silu(x) - si[i]) < 1e-12
+
+
+def test_attention_special_cases_and_torch():
+    hd, n = 16, 9
+    q = rng.standard_normal(hd).astype(np.float32)
+    K = rng.standard_normal((n, hd)).astype(np.float32)
+    V = rng.standard_normal((n, hd)).astype(np.float32)
+    assert np.array_equal(O.attend(q, K[:1], V[:1]), V[0])                       # one key -> its value
+    assert np.abs(O.attend(np.zeros(hd, np.float32), K, V) - V.astype(np.float64).mean(0)).max() < 1e-6
+    big = O.attend((K[4] * 200).astype(np.float32), K, V)                          # sharp softmax picks the best key
+    s = (K.astype(np.float64) @ (K[4].astype(np.float64) * 200)) / math.sqrt(hd)
+    assert np.abs(big - V[int(s.argmax())]).max() < 1e-5
+    qt, Kt, Vt = (torch.from_numpy(a).double() for a in (q, K, V))
+    ref = F.scaled_dot_product_attention(qt[None, None, None], Kt[None, None], Vt[None, None])[0, 0, 0].numpy()
+    assert np.abs(O.attend(q, K, V) - ref).max() < 1e-6
+
+
+def test_rope_properties():
+    hd, theta = 32, 1e4
+    v = rng.standard_normal(hd).astype(np.float32)
+    k = rng.standard_normal(hd).astype(np.float32)
+    assert np.array_equal(O.rope(v, 0, theta), v)                                  # position 0: identity
+    for pos in (1, 5, 100, 2047):
+        r = O.rope(v, pos, theta).astype(np.float64)
+        assert abs(np.linalg.norm(r) - np.linalg.norm(v.astype(np.float64))) < 1e-5   # rotation keeps the norm
+    base = float(O.rope(v, 7, theta).astype(np.float64) @ O.rope(k, 3, theta).astype(np.float64))
+    for shift in (1, 10, 500):                                                     # depends on m - n only
+        d2 = float(O.rope(v, 7 + shift, theta).astype(np.float64) @ O.rope(k, 3 + shift, theta).astype(np.float64))
+        assert abs(d2 - base) < 2e-5
+    # element hd/2-1 turns slowest: angle pos * theta^(-(hd-2)/hd); element 0 turns by pos radians
+    e = np.zeros(hd, np.float32)
+    e[0] = 1.0
+    r = O.rope(e, 2, theta)
+    assert abs(r[0] - math.cos(2.0)) < 1e-6 and abs(r[hd // 2] - math.sin(2.0)) < 1e-6
+    e = np.zeros(hd, np.float32)
+    e[hd // 2 - 1] = 1.0
+    ang = 3 * theta ** (-(hd - 2) / hd)
+    r = O.rope(e, 3, theta)
+    assert abs(r[hd // 2 - 1] - math.cos(ang)) < 1e-6 and abs(r[hd - 1] - math.sin(ang)) < 1e-6
+
+
+def test_argmax_brute_force_and_ties():
+    for _ in range(20):
+        x = rng.standard_normal(50).astype(np.float32)
+        assert O.argmax(x) == max(range(50), key=lambda i: x[i])
+    x = np.array([0.5, 2.0, -1.0, 2.0, 2.0], np.float32)
+    assert O.argmax(x) == 1                                                        # lowest index wins
+
+
+# ---------------- whole model ---------------------------------------------------------------
+
+def _torch_reference_logits(shape, w, tokens):
+    """The same decoder assembled from torch fp64 library ops (textbook form), all positions."""
+    W = {k: torch.from_numpy(I.as_f32(v)).double() for k, v in w.items()}
+    T = len(tokens)
+    tok = torch.tensor(tokens)
+    H, hd, Hk, d = shape.n_head, shape.head_dim, shape.n_kv_head, shape.d_model
+    x = W["wte"][tok]
+    if shape.arch == I.ARCH_GPT:
+        x = x + W["wpe"][:T]
+
+    def norm(x, pfx):
+        if shape.arch == I.ARCH_GPT:
+            return F.layer_norm(x, (d,), W[pfx + ".g"], W[pfx + ".b"], shape.norm_eps)
+        return F.rms_norm(x, (d,), W[pfx + ".g"], shape.norm_eps)
+
+    def rope(t):  # t [heads, T, hd]; rotate-half form of the split-halves pairing
+        half = hd // 2
+        inv = shape.rope_theta ** (-torch.arange(half, dtype=torch.float64) * 2 / hd)
+        ang = torch.arange(T, dtype=torch.float64)[:, None] * inv[None, :]
+        cos = torch.cat([ang.cos(), ang.cos()], -1).float().double()
+        sin = torch.cat([ang.sin(), ang.sin()], -1).float().double()
+        rot = torch.cat([-t[..., half:], t[..., :half]], -1)
+        return t * cos + rot * sin
+
+    for i in range(shape.n_layer):
+        p = f"h.{i}."
+        h = norm(x, p + "ln1")
+        qkv = F.linear(h, W[p + "attn.wqkv"], W.get(p + "attn.bqkv"))
+        q, k, v = qkv.split([H * hd, Hk * hd, Hk * hd], dim=-1)
+        q = q.view(T, H, hd).transpose(0, 1)
+        k = k.view(T, Hk, hd).transpose(0, 1)
+        v = v.view(T, Hk, hd).transpose(0, 1)
+        if shape.arch == I.ARCH_LLAMA:
+            q, k = rope(q), rope(k)
+        k = k.repeat_interleave(H // Hk, 0)
+        v = v.repeat_interleave(H // Hk, 0)
+        o = F.scaled_dot_product_attention(q[None], k[None], v[None], is_causal=True)[0]
+        o = o.transpose(0, 1).reshape(T, H * hd)
+        x = x + F.linear(o, W[p + "attn.wo"], W.get(p + "attn.bo"))
+        n = norm(x, p + "ln2")
+        if shape.act == I.ACT_SWIGLU:
+            m = F.linear(F.silu(F.linear(n, W[p + "mlp.wgate"])) * F.linear(n, W[p + "mlp.wup"]), W[p + "mlp.wdown"])
+        else:
+            a = F.linear(n, W[p + "mlp.w1"], W[p + "mlp.b1"])
+            a = F.gelu(a, approximate="tanh") if shape.act == I.ACT_GELU_TANH else F.gelu(a)
+            m = F.linear(a, W[p + "mlp.w2"], W[p + "mlp.b2"])
+        x = x + m
+    x = norm(x, "lnf")
+    head = W["wte"] if shape.tied_lm_head else W["lm_head"]
+    return F.linear(x, head).numpy()
+
+
+@pytest.mark.parametrize("arch,dtype,n_kv", [("gpt", I.DT_F32, None), ("gpt", I.DT_BF16, None),
+                                             ("llama", I.DT_BF16, None), ("llama", I.DT_F32, 2)])
+def test_full_forward_matches_torch_fp64(arch, dtype, n_kv):
+    shape = tiny_shape(arch, dtype, L=3, d=32, H=4, V=23, C=16, n_kv=n_kv)
+    orc, w = make_oracle(shape, seed=5, std=0.3)       # large weights: every term matters
+    tokens = [int(t) for t in I.make_prompts(shape.vocab, 1, 12, seed=9)[0]]
+    got = orc.full_logits(tokens)
+    ref = _torch_reference_logits(shape, w, tokens)
+    assert np.abs(got - ref).max() < 2e-5 * max(1.0, np.abs(ref).max())
+
+
+def test_zero_blocks_special_case():
+    """All block matrices zero: logits = Norm_f(wte[tok] + wpe[pos]) . W_head^T."""
+    shape = tiny_shape("gpt", I.DT_F32)
+    w = I.make_weights(shape, 3, 0.5)
+    for k in w:
+        if k.startswith("h.") and (".attn." in k or ".mlp." in k):
+            w[k][...] = 0
+    orc = O.Oracle(shape, w)
+    tokens = [3, 11, 5, 0]
+    got = orc.full_logits(tokens)
+    for pos, t in enumerate(tokens):
+        x = w["wte"][t].astype(np.float64) + w["wpe"][pos].astype(np.float64)
+        n = (x - x.mean()) / np.sqrt(x.var() + shape.norm_eps) * w["lnf.g"] + w["lnf.b"]
+        assert np.abs(got[pos] - w["wte"].astype(np.float64) @ n).max() < 1e-4
+
+
+# ---------------- invariants the method relies on ---------------------------------------------
+
+@pytest.mark.parametrize("arch,dtype", [("gpt", I.DT_F32), ("llama", I.DT_BF16)])
+def test_I1_cached_decode_equals_full_recompute(arch, dtype):
+    shape = tiny_shape(arch, dtype)
+    orc, _ = make_oracle(shape, std=0.2)
+    prompt = [int(t) for t in I.make_prompts(shape.vocab, 1, 5)[0]]
+    t_full, l_full = orc.generate_full_recompute(prompt, 10)
+    t_kv, l_kv = orc.generate_sequential(prompt, 10)
+    assert t_full == t_kv
+    assert np.abs(l_full - l_kv).max() <= 1e-5
+    # every prompt position too: prefill of the whole prompt vs positions fed one at a time
+    c1 = O.Cache(orc, 0, shape.n_layer)
+    X1 = orc.blocks(c1, orc.embed(prompt, 0))
+    c2 = O.Cache(orc, 0, shape.n_layer)
+    rows = [orc.blocks(c2, orc.embed([t], i))[0] for i, t in enumerate(prompt)]
+    assert np.abs(X1 - np.stack(rows)).max() <= 1e-5
+    full = orc.full_logits(prompt)
+    for i in range(len(prompt)):
+        assert np.abs(orc.head(X1[i]) - full[i]).max() <= 1e-5
+
+
+def test_I1_on_the_tiny_gpt_workload():
+    w = I.WORKLOADS["tiny_gpt_fp32"]
+    orc, _ = make_oracle(w.shape, w.weight_seed)
+    prompt = [int(t) for t in I.make_prompts(w.shape.vocab, 1, w.n_prompt, w.prompt_seed)[0]]
+    t_full, l_full = orc.generate_full_recompute(prompt, 6)
+    t_kv, l_kv = orc.generate_sequential(prompt, 6)
+    assert t_full == t_kv and np.abs(l_full - l_kv).max() <= 1e-5
+
+
+def test_I2_partition_boundaries_do_not_change_logits():
+    shape = tiny_shape("gpt", I.DT_BF16, L=4)
+    orc, _ = make_oracle(shape, std=0.2)
+    prompt = [1, 7, 3, 9, 2]
+    _, base = orc.generate_sequential(prompt, 6, [0, 4])
+    cuts = []
+    for k in range(0, 4):
+        for inner in itertools.combinations(range(1, 4), k):
+            cuts.append([0, *inner, 4])
+    assert len(cuts) == 8
+    for b in cuts:
+        _, lg = orc.generate_sequential(prompt, 6, b)
+        assert np.array_equal(lg, base), b
+
+
+@pytest.mark.parametrize("S,K", [(1, 1), (1, 3), (2, 3), (3, 3), (5, 3), (3, 2), (5, 2), (2, 1)])
+def test_I3_pipeline_equals_sequential(S, K):
+    shape = tiny_shape("llama", I.DT_BF16, L=3)
+    orc, _ = make_oracle(shape, std=0.2)
+    bounds = {1: [0, 3], 2: [0, 1, 3], 3: [0, 1, 2, 3]}[K]
+    prompts = [[int(t) for t in p[: 2 + s % 3]] for s, p in enumerate(I.make_prompts(shape.vocab, S, 4))]
+    n_new = 5
+    for head_on_starter in (True, False):
+        toks, lgs, _ = orc.generate_pipeline(prompts, n_new, bounds, head_on_starter)
+        for s in range(S):
+            t_seq, l_seq = orc.generate_sequential(prompts[s], n_new)
+            assert toks[s] == t_seq
+            assert np.array_equal(lgs[s], l_seq)
+
+
+def test_pipeline_schedule_matches_the_papers_worked_example():
+    gold = [tuple(int(v) for v in ln.split()) for ln in open(os.path.join(GOLD, "pipeline_schedule_3x3.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    shape = tiny_shape("gpt", I.DT_F32, L=3)
+    orc, _ = make_oracle(shape)
+    prompts = [[1, 2], [3, 4], [5, 6]]
+    _, _, trace = orc.generate_pipeline(prompts, 3, [0, 1, 2, 3], head_on_starter=True)
+    blocks = [(t, p, n) for (t, p, n, kind) in trace if kind != "head" and t <= 3]
+    assert blocks == gold
+    # tick 3: the starter first applies the output layers to sample 0 (its first new token)
+    assert (3, 0, 0, "head") in trace
+    first_head = min(t for (t, p, n, kind) in trace if kind == "head")
+    assert first_head == 3
+    # general rule behind the example: node p at tick tau serves sample (tau - p) mod S
+    for (t, p, n, kind) in trace:
+        assert n == (t - p) % 3
+
+
+def test_generate_counts_exactly_n_new_tokens_and_last_visit_is_not_fed_back():
+    shape = tiny_shape("gpt", I.DT_F32, L=2, C=16)
+    orc, _ = make_oracle(shape)
+    prompts = [[1, 2, 3], [4, 5, 6]]
+    toks, lgs, trace = orc.generate_pipeline(prompts, 4, [0, 1, 2])
+    assert all(len(t) == 4 for t in toks) and all(l.shape == (4, shape.vocab) for l in lgs)
+    # per sample: 1 prefill + 3 decode passes through each node, 4 head evaluations
+    for n in range(2):
+        assert sum(1 for e in trace if e[2] == n and e[1] == 0 and e[3] != "head") == 4
+        assert sum(1 for e in trace if e[2] == n and e[3] == "head") == 4
+    # context boundary: prompt + n_new == n_ctx is legal (the last token is never fed), one more is not
+    t_ok, _ = orc.generate_sequential([1] * 10, 6)
+    assert len(t_ok) == 6
+    with pytest.raises(ValueError):
+        orc.generate_sequential([1] * 10, 8)
+
+
+def test_tied_head_duplicate_row_tie_goes_to_lowest_id():
+    shape = tiny_shape("gpt", I.DT_F32)
+    w = I.make_weights(shape, 2, 0.3)
+    orc = O.Oracle(shape, w)
+    lg = orc.head(orc.embed([3], 0)[0])
+    top = int(np.argmax(lg))
+    other = (top + 5) % shape.vocab
+    w["wte"][other] = w["wte"][top]
+    orc2 = O.Oracle(shape, w)
+    x = np.ascontiguousarray(rng.standard_normal(shape.d_model), np.float32)
+    lg2 = orc2.head(x)
+    assert lg2[other] == lg2[top]
+    w["wte"][:] = 0
+    assert O.argmax(O.Oracle(shape, w).head(x)) == 0
+
+
+def test_forced_tokens_only_change_what_is_fed_back():
+    shape = tiny_shape("gpt", I.DT_F32)
+    orc, _ = make_oracle(shape, std=0.2)
+    free_t, free_l = orc.generate_sequential([1, 2, 3], 5)
+    t2, l2 = orc.generate_sequential([1, 2, 3], 5, forced=free_t)
+    assert t2 == free_t and np.array_equal(l2, free_l)
+    forced = [(t + 1) % shape.vocab for t in free_t]
+    t3, l3 = orc.generate_sequential([1, 2, 3], 5, forced=forced)
+    assert np.array_equal(l3[0], free_l[0]) and not np.array_equal(l3[1], free_l[1])
+    # equals recomputing from the forced history
+    full = orc.full_logits([1, 2, 3] + forced[:4])
+    assert np.abs(full[2:] - l3).max() <= 1e-5
