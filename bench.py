@@ -1,0 +1,303 @@
+#!/usr/bin/env python
+"""Benchmark of recurrent-pipeline decoding on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: every sample's
+first visit (prompt through all partitions) followed by the recurrent pipeline until each sample
+has n_new greedy tokens.  Workload: the GPT-2-small shape (12 layers, d 768, bf16 seeded weights,
+3 partitions of 4 layers, 3 samples in flight, 64-token prompts, 512 new tokens).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+Prints ONE JSON line.  `value` = generated tokens/s over all samples with the prompts already in
+device memory (device time from library-side CUDA events on its own streams); `e2e` = the same
+through the host-pointer entry points, prompts copied in and tokens copied out every step;
+`roofline` = decode phase against the measured HBM copy bandwidth; `cpu_baseline` = the CPU
+checker timed on a bounded sample of the same workload.  With N > 1 every rank runs an
+independent replica (the path does not shard) and the values add up.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2505_18164_b200 import inputs as I  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def decode_bytes(w: I.Workload, n_samples: int) -> dict:
+    """Algorithmic bytes of the decode phase of one step (what the schedule must move).
+
+    Per pass (every sample gains one token) each of the G groups streams every block matrix and
+    vector once and the output projection once; each sample reads its whole cache (keys and values
+    of every layer, rows 0..t) and writes one row per layer.  Embedding rows and activations are
+    negligible and left out."""
+    s = w.shape
+    bpe = 4 if s.weight_dtype == I.DT_F32 else 2
+    specs = I.tensor_specs(s)
+    block = sum(int(np.prod(shp)) for n, shp, _ in specs if n.startswith("h."))
+    head = s.vocab * s.d_model + s.d_model * (2 if s.arch == I.ARCH_GPT else 1)
+    G = min(n_samples, w.n_partitions)
+    per_pass_w = G * (block + head) * bpe
+    kvw = s.n_kv_head * s.head_dim
+    n_pass = w.n_new - 1
+    kv = 0
+    for i in range(n_pass):
+        t = w.n_prompt + i                       # rows cached before this pass
+        kv += n_samples * s.n_layer * (2 * (t + 1) * kvw + 2 * kvw) * bpe
+    return {"weights": per_pass_w * n_pass, "kv": kv, "total": per_pass_w * n_pass + kv, "passes": n_pass,
+            "per_pass_weights": per_pass_w}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self) -> dict:
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_baseline(w: I.Workload, weights, n_new_sample: int = 24):
+    """The CPU checker, as it stands, on a bounded sample of the workload: all samples, full prompts,
+    the first n_new_sample of the new tokens, scheduled by its own recurrent-pipeline simulation."""
+    from oracle import mdi_oracle as O
+    orc = O.Oracle(w.shape, weights)
+    prompts = I.make_prompts(w.shape.vocab, w.n_samples, w.n_prompt, w.prompt_seed)
+    t0 = time.perf_counter()
+    toks, _, _ = orc.generate_pipeline([[int(t) for t in p] for p in prompts], n_new_sample, list(w.part_bounds),
+                                       head_on_starter=False)
+    dt = time.perf_counter() - t0
+    n = sum(len(t) for t in toks)
+    return {"value": n / dt, "unit": "tokens/s", "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"{w.n_samples} samples, {w.n_prompt}-token prompts, first {n_new_sample} of {w.n_new} new tokens each, "
+                      f"{dt:.1f} s of CPU work"}, dt
+
+
+def run_reference(args, w: I.Workload):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    weights = I.make_weights(w.shape, w.weight_seed)
+    times, val = [], None
+    n_sample = 8
+    for i in range(args.warmup + args.steps):
+        cb, dt = cpu_baseline(w, weights, n_sample)
+        if i >= args.warmup:
+            times.append(dt)
+            val = cb
+    tok = w.n_samples * n_sample
+    v = tok * len(times) / sum(times)
+    val["value"] = v
+    print(json.dumps({
+        "impl": "reference", "metric": "generated tokens/s (all in-flight samples)", "value": v, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "note": "CPU checker on host cores; each step a bounded sample of the workload"},
+        "cpu_baseline": val,
+        "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="mdi", choices=["mdi", "reference"])
+    ap.add_argument("--workload", default="gpt2_small", choices=I.WORKLOAD_ORDER)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rounds-per-graph", type=int, default=0)
+    args = ap.parse_args()
+    w = I.WORKLOADS[args.workload]
+    from paper_2505_18164_b200 import build
+    build.build_inputs()
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2505_18164_b200 import mdi
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decoding path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    s = w.shape
+    S, P, N = w.n_samples, w.n_prompt, w.n_new
+    ctx = mdi.Context(s, list(w.part_bounds), S, kv_pool_tokens=S * (P + N), rounds_per_graph=args.rounds_per_graph)
+    weights = {}
+    for name, a in I.iter_weights(s, w.weight_seed):
+        ctx.load_weights(name, a)
+        if rank == 0 and not args.no_cpu_baseline and args.workload in ("tiny_gpt_fp32", "gpt2_small", "gpt2_medium"):
+            weights[name] = a
+    prompts_host = torch.from_numpy(I.make_prompts(s.vocab, S, P, w.prompt_seed)).pin_memory()
+    prompts_dev = prompts_host.cuda()
+    out_dev = torch.empty((S, N), dtype=torch.int32, device="cuda")
+    out_host = torch.empty((S, N), dtype=torch.int32).pin_memory()
+    out_np = out_host.numpy()
+    prompts_np = prompts_host.numpy()
+
+    def step_device():
+        for smp in range(S):
+            ctx.reset_sample(smp)
+        for smp in range(S):
+            ctx.prefill_dev(smp, prompts_dev[smp], P)
+        ctx.generate_dev(S, N, out_dev)
+
+    def step_host():
+        for smp in range(S):
+            ctx.reset_sample(smp)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for smp in range(S):
+            ctx.prefill(smp, prompts_np[smp])
+        ctx.generate(S, N, out_np)
+        return time.perf_counter() - t0
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step_device()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    st0 = ctx.stats()
+    run_ms, gen_ms, pf_ms = [], [], []
+    for _ in range(args.steps):
+        step_device()
+        st = ctx.stats()
+        run_ms.append(st.last_run_ms)
+        gen_ms.append(st.last_generate_ms)
+        pf_ms.append(st.last_prefill_ms)
+    barrier()
+    st1 = ctx.stats()
+    clocks = sampler.stop() if rank == 0 else None
+    tokens_dev = out_dev.cpu().numpy().copy()
+
+    # end to end through the host-pointer entry points
+    step_host()
+    barrier()
+    e2e_s = [step_host() for _ in range(args.steps)]
+    barrier()
+    assert np.array_equal(out_np, tokens_dev), "host and device entry points disagree"
+
+    tot_ms = torch.tensor([sum(run_ms), sum(e2e_s) * 1e3], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(tot_ms, op=dist.ReduceOp.MAX)
+    tot_run_ms, tot_e2e_ms = (float(v) for v in tot_ms.cpu())
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        db = decode_bytes(w, S)
+        gen_avg_ms = sum(gen_ms) / len(gen_ms)
+        achieved = db["total"] / (gen_avg_ms * 1e-3) / 1e9
+        value = world * S * N * args.steps / (tot_run_ms * 1e-3)
+        e2e_value = world * S * N * args.steps / (tot_e2e_ms * 1e-3)
+        launches = int(st1.kernel_launches - st0.kernel_launches)
+        line = {
+            "metric": "generated tokens/s (all in-flight samples)", "value": value, "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot_run_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if s.weight_dtype == I.DT_BF16 else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "n_layer": s.n_layer, "d_model": s.d_model, "vocab": s.vocab,
+                       "partitions": list(w.part_bounds), "samples_in_flight": S, "n_prompt": P, "n_new": N,
+                       "l2": "weights streamed per tick (model + cache) exceed the 126 MB L2; no flush between steps",
+                       "multi_gpu": "replicas only" if world > 1 else "single"},
+            "decode_tokens_per_s": world * S * (N - 1) / (gen_avg_ms * 1e-3),
+            "prefill_ms": sum(pf_ms) / len(pf_ms), "decode_ms": gen_avg_ms,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                         "traffic": None, "scope": "decode phase of one step (all kernels of mdi_generate)",
+                         "algorithmic_bytes": db["total"], "weight_bytes": db["weights"], "kv_bytes": db["kv"]},
+            "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(S * P * 4),
+                    "d2h_bytes_per_step": int(S * N * 4)},
+            "gpu_launches": launches,
+            "clocks": clocks,
+        }
+        if weights:
+            line["cpu_baseline"], _ = cpu_baseline(w, weights)
+        else:
+            line["cpu_baseline"] = None
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,165 @@
+/* mdi.h - C ABI of the recurrent-pipeline decoding library (MDI-LLM hot path on one GPU).
+ *
+ * The method (paper, Section III): a decoder-only transformer is cut into K contiguous
+ * chunks of blocks ("nodes"); several text samples are kept in flight; each node
+ * repeatedly takes the next sample's activation from its input queue, selects that
+ * sample's key/value cache (Section III-D), runs its blocks, and hands the result to the
+ * next node; the last result returns to the first node, which produces a token and feeds
+ * it back (Section III-C, Algorithms 1 and 2).  Here the K nodes are K CUDA streams of one
+ * GPU, the links between nodes are device-resident activation ring buffers handed over
+ * with events, and every sample owns a slot of a paged key/value pool.
+ *
+ * Conventions
+ *  - Every function returns MDI_OK (0) or a negative MDI_ERR_* code; nothing aborts.
+ *    mdi_last_error() gives the text of the last failure on that context.
+ *  - "host" pointers are ordinary CPU memory owned by the caller; the library copies
+ *    what it needs before returning.  "dev" pointers are CUDA device memory owned by the
+ *    caller.  All other device memory (weights, caches, rings, logits) belongs to the
+ *    context and is released by mdi_destroy().
+ *  - A context is bound to the CUDA device current at mdi_create() and is not
+ *    thread-safe.  The library never falls back to the CPU.
+ *  - slot == sample index in [0, n_samples).
+ */
+#ifndef MDI_H_
+#define MDI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    MDI_OK = 0,
+    MDI_ERR_ARG = -1,     /* null pointer, index out of range, bad enum value */
+    MDI_ERR_SHAPE = -2,   /* model shape or tensor size the kernels do not support */
+    MDI_ERR_OOM = -3,     /* device allocation failed or key/value page pool exhausted */
+    MDI_ERR_CONTEXT = -4, /* prompt + new tokens would exceed n_ctx */
+    MDI_ERR_STATE = -5,   /* call out of order: missing weights, sample not prefilled, ... */
+    MDI_ERR_TIMEOUT = -6, /* a bounded wait ran out */
+    MDI_ERR_CUDA = -7     /* a CUDA runtime call failed */
+};
+
+enum { MDI_ARCH_GPT = 0, MDI_ARCH_LLAMA = 1 };
+enum { MDI_DTYPE_F32 = 0, MDI_DTYPE_BF16 = 1 };
+enum { MDI_ACT_GELU_TANH = 0, MDI_ACT_GELU_ERF = 1, MDI_ACT_SWIGLU = 2 };
+
+typedef struct mdi_ctx mdi_ctx;
+
+/* Shape of the decoder (the block of Section III-B: attention + fully connected layer,
+ * each with a residual connection; equal input and output width d_model). */
+typedef struct {
+    int arch;         /* MDI_ARCH_GPT: LayerNorm, learned positions, biases, GELU MLP;
+                         MDI_ARCH_LLAMA: RMSNorm, rotary positions (split-halves pairing), SwiGLU, no biases */
+    int n_layer, d_model, n_head, head_dim, n_kv_head, d_ff, vocab, n_ctx;
+    int weight_dtype; /* MDI_DTYPE_*: element type of every tensor given to mdi_load_weights; the
+                         key/value cache uses the same type; activations and accumulation are fp32 */
+    int tied_lm_head; /* 1: the output projection reuses "wte" */
+    int has_bias;     /* 1: linear layers carry biases (GPT) */
+    int act;          /* MDI_ACT_* */
+    float norm_eps, rope_theta;
+} mdi_model_shape;
+
+/* Optional tuning; zero means "default". */
+typedef struct {
+    int page_tokens;   /* rows per key/value page (default 16; power of two) */
+    int kv_pool_tokens;/* tokens of cache each partition's pool can hold over all samples
+                          (default n_samples * n_ctx, rounded up to pages) */
+    int attn_splits;   /* sequence splits of decode attention (default: chosen from n_ctx) */
+    int rounds_per_graph; /* rounds of the recurrent schedule captured per CUDA graph (default 16; <0: no graphs) */
+} mdi_options;
+
+typedef struct {
+    int n_partitions, n_samples, n_groups;
+    int64_t weight_bytes[16];   /* per partition, device bytes of parameters (first 16 partitions) */
+    int64_t kv_pool_bytes[16];  /* per partition, device bytes of the key/value pool */
+    int64_t kv_pages_in_use[16];
+    int64_t tokens_generated;   /* head evaluations since creation */
+    int64_t stage_steps;        /* partition steps launched since creation */
+    int64_t kernel_launches;    /* kernels of this library launched (or replayed in graphs) since creation */
+    float last_prefill_ms;      /* device time from the first mdi_prefill after the previous mdi_generate to the
+                                   end of the last one (events on the partition streams) */
+    float last_generate_ms;     /* device time of the last mdi_generate, first to last partition step */
+    float last_run_ms;          /* device time from that first mdi_prefill to the end of the last mdi_generate */
+} mdi_stats;
+
+/* Set-up of the nodes (Section III-A: the starter assigns each node its chunk).
+ * part_bounds: K+1 ascending layer indices, part_bounds[0] = 0, part_bounds[K] = n_layer;
+ * partition p holds blocks [part_bounds[p], part_bounds[p+1]).  Partition 0 also holds the
+ * input layers (embeddings); partition K-1 also holds the output layers (final norm and
+ * vocabulary projection) - the paper keeps them on the starter, which changes only where
+ * the work runs.  n_samples = samples in flight (slots).  opts may be NULL.
+ * Errors: ARG (nulls, K < 1, bounds not ascending), SHAPE (unsupported sizes), OOM. */
+int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int n_samples,
+               const mdi_options *opts, mdi_ctx **out);
+void mdi_destroy(mdi_ctx *ctx);
+
+/* "Load model chunk" (Algorithms 1 and 2).  One call per tensor; host_data is row-major
+ * [out_features][in_features] for matrices, element type shape.weight_dtype, nbytes its
+ * exact size.  Names: "wte" [vocab][d], "wpe" [n_ctx][d] (GPT), "lnf.g", "lnf.b" (GPT),
+ * "lm_head" [vocab][d] (untied), and per block i: "h.<i>.ln1.g", "h.<i>.ln1.b" (GPT),
+ * "h.<i>.attn.wqkv" [(n_head+2 n_kv_head) head_dim][d] (q rows, then k, then v),
+ * "h.<i>.attn.bqkv", "h.<i>.attn.wo" [d][n_head head_dim], "h.<i>.attn.bo", "h.<i>.ln2.g",
+ * "h.<i>.ln2.b", GPT: "h.<i>.mlp.w1" [d_ff][d], ".b1", ".w2" [d][d_ff], ".b2";
+ * Llama: "h.<i>.mlp.wgate" [d_ff][d], ".wup" [d_ff][d], ".wdown" [d][d_ff].
+ * The data is copied to the device before the call returns.
+ * Errors: ARG (unknown name), SHAPE (nbytes mismatch), CUDA. */
+int mdi_load_weights(mdi_ctx *ctx, const char *tensor_name, const void *host_data, size_t nbytes);
+
+/* First visit of a sample (Algorithm 1 "first iteration", Algorithm 2 "n-th cache is None"):
+ * the whole prompt goes through every partition in turn, filling cache rows 0..n_prompt-1 of
+ * the sample's slot; only the last position reaches the output layers, whose result is the
+ * sample's first new token (kept pending until mdi_generate returns it).  Work is enqueued
+ * on the partition streams with event handoff, so consecutive calls for different samples
+ * overlap like the paper's start-up phase; it completes by the next mdi_sync/mdi_generate.
+ * prompt_host: n_prompt token ids in [0, vocab).  The _dev form reads them from device memory.
+ * Errors: ARG, STATE (slot already holds tokens: mdi_reset_sample first; weights missing),
+ * CONTEXT (n_prompt > n_ctx), OOM (page pool). */
+int mdi_prefill(mdi_ctx *ctx, int sample, const int32_t *prompt_host, int n_prompt);
+int mdi_prefill_dev(mdi_ctx *ctx, int sample, const int32_t *prompt_dev, int n_prompt);
+
+/* One visit of one sample to one node (body of the loop of Algorithm 2; for partition 0 the
+ * "forward through input layers" of Algorithm 1): select the slot's cache, run the partition's
+ * blocks on one new position, append its keys and values.
+ * act_in_dev:  partition 0: one int32 token id; otherwise fp32[d_model].
+ * act_out_dev: last partition: one int32 token id (greedy argmax, lowest id on ties; the logits
+ * are kept for mdi_get_logits); otherwise fp32[d_model].  Both in device memory.
+ * Advances the slot's position in that partition by one.  Enqueued on the partition's stream;
+ * mdi_sync() waits.  Errors: ARG, STATE, CONTEXT (slot full), OOM. */
+int mdi_step(mdi_ctx *ctx, int partition, int slot, const void *act_in_dev, void *act_out_dev);
+
+/* Recurrent pipeline (Section III-C; Algorithm 1's loop over n_samples x n_tokens): returns the
+ * next n_new_tokens greedy tokens of samples 0..n_samples-1, which must all have been
+ * prefilled.  Samples are dealt into G = min(n_samples, K) groups (sample s in group s mod G);
+ * at tick t partition p serves group (t - p) mod K (an idle tick if that is >= G, i.e. fewer
+ * samples than partitions); a group's samples share one pass over the partition's weights.  A token produced by the last partition is fed to partition 0 one tick
+ * later; the last token of the call is produced but not fed (it is fed first by a later call).
+ * out_tokens: [n_samples][n_new_tokens] int32, host (or device for the _dev form).
+ * Blocks until the tokens are there.  Errors: ARG, STATE, CONTEXT, OOM. */
+int mdi_generate(mdi_ctx *ctx, int n_samples, int n_new_tokens, int32_t *out_tokens_host);
+int mdi_generate_dev(mdi_ctx *ctx, int n_samples, int n_new_tokens, int32_t *out_tokens_dev);
+
+/* Logits (fp32[vocab]) of the sample's most recent output-layer evaluation, copied to host. */
+int mdi_get_logits(mdi_ctx *ctx, int sample, float *out_host);
+
+/* Checking aid: the i-th output-layer evaluation of the sample (counted from its prefill)
+ * still reports its own argmax, but tokens_host[i] is what gets fed back for i < n.
+ * Must be set after mdi_reset_sample/creation and before the sample's prefill. */
+int mdi_set_teacher_tokens(mdi_ctx *ctx, int sample, const int32_t *tokens_host, int n);
+
+/* Forget a sample: its pages go back to the pools, its position and counters to zero. */
+int mdi_reset_sample(mdi_ctx *ctx, int sample);
+
+int mdi_get_stats(mdi_ctx *ctx, mdi_stats *out);
+/* Device bytes held by one partition (parameters + key/value pool + buffers), cf. Tables I-II. */
+int64_t mdi_memory_bytes(mdi_ctx *ctx, int partition);
+/* Wait for everything enqueued on the context's streams. */
+int mdi_sync(mdi_ctx *ctx);
+/* Text of the last error of this context (or of the last failed mdi_create if ctx is NULL). */
+const char *mdi_last_error(mdi_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MDI_H_ */

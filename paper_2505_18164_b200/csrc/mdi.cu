@@ -1,0 +1,887 @@
+// Host side of the recurrent-pipeline decoding library: contexts, weights, the paged key/value
+// slot allocator, the partition streams with their activation rings and event handoff, and the
+// scheduler that rotates sample groups through the partitions (paper, Section III-C, Algorithms 1-2).
+#include "mdi.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "step_kernels.cuh"
+
+using namespace mdi;
+
+namespace {
+
+std::string g_create_error;
+
+struct LayerW {
+    void *wqkv = nullptr, *wo = nullptr, *w1 = nullptr, *w2 = nullptr, *wgate = nullptr, *wup = nullptr, *wdown = nullptr;
+    float *ln1g = nullptr, *ln1b = nullptr, *bqkv = nullptr, *bo = nullptr, *ln2g = nullptr, *ln2b = nullptr,
+          *b1 = nullptr, *b2 = nullptr;
+};
+
+struct TensorSlot {
+    void **mat = nullptr;  // destination pointer for matrices (weight dtype on device)
+    float **vec = nullptr; // destination pointer for small vectors (fp32 on device)
+    size_t elems = 0;
+    int partition = 0;
+    bool loaded = false;
+};
+
+struct Partition {
+    int lo = 0, hi = 0;
+    cudaStream_t stream = nullptr;
+    // key/value pool
+    void *kv_pool = nullptr;
+    size_t kv_bytes = 0;
+    int n_pages = 0;
+    std::vector<int> free_pages;
+    std::vector<int> pt_host; // [S][L_p][pages_per_seq], -1 = unmapped (uploaded as 0)
+    std::vector<int> pages_of_slot; // count per slot (pages per layer)
+    int *pt_dev = nullptr;
+    int *pos_dev = nullptr;
+    std::vector<int> pos_host;
+    // scratch (one step at a time runs on the partition's stream)
+    float *x_embed = nullptr, *qbuf = nullptr, *obuf = nullptr, *hbuf = nullptr, *part = nullptr, *x_last = nullptr;
+    unsigned *attn_ticket = nullptr;
+    // output edge: ring of group slots, and two buffers for first-visit (whole prompt) activations
+    float *ring = nullptr;
+    float *pf_buf[2] = {nullptr, nullptr};
+    std::vector<cudaEvent_t> ev_edge, ev_edge_cap;
+    cudaEvent_t ev_pf_out[2] = {nullptr, nullptr}, ev_pf_used[2] = {nullptr, nullptr};
+    bool pf_used_valid[2] = {false, false};
+    cudaEvent_t ev_join = nullptr, ev_join_cap = nullptr;
+    int64_t weight_bytes = 0, buffer_bytes = 0;
+};
+
+struct GraphEntry {
+    cudaGraphExec_t exec = nullptr;
+    int64_t launches = 0, steps = 0;
+};
+
+} // namespace
+
+struct mdi_ctx {
+    mdi_model_shape s{};
+    mdi_options o{};
+    int K = 0, S = 0, dev = 0;
+    int page_tokens = 16, page_shift = 4, pages_per_seq = 0, n_split = 1, gmax = 1, rounds_per_graph = 16;
+    size_t page_elems = 0, esize = 2;
+    std::vector<Partition> part;
+    std::vector<LayerW> layer;
+    void *wte = nullptr, *wpe = nullptr, *lm_head = nullptr;
+    float *lnfg = nullptr, *lnfb = nullptr;
+    std::map<std::string, TensorSlot> tensors;
+    int n_loaded = 0;
+    float *rope_cos = nullptr, *rope_sin = nullptr;
+    // output layers
+    float *logits = nullptr; // [S][V]
+    float *head_pv = nullptr;
+    int *head_pi = nullptr;
+    unsigned *head_ticket = nullptr;
+    int head_grid = 0;
+    // token state
+    int *cur_tok = nullptr, *tok_log = nullptr, *gen_count = nullptr, *teacher = nullptr, *n_teacher = nullptr;
+    int *prompt_buf = nullptr; // [S][n_ctx]
+    std::vector<int> gen_host, returned_host, prefilled;
+    int pf_count = 0;
+    cudaStream_t main = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_fork_cap = nullptr, ev_t0 = nullptr, ev_t1 = nullptr, ev_pf0 = nullptr, ev_pf1 = nullptr;
+    bool pf_open = false; // ev_pf0 recorded by the first prefill since the last generate
+    std::map<std::pair<int, int>, GraphEntry> graphs; // (n_samples, window ticks)
+    bool capturing = false;
+    int64_t cap_launches = 0, cap_steps = 0;
+    mdi_stats st{};
+    std::string err;
+};
+
+namespace {
+
+int fail(mdi_ctx *c, int code, const char *fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (c) c->err = buf; else g_create_error = buf;
+    return code;
+}
+
+#define CU(call)                                                                                             \
+    do {                                                                                                     \
+        cudaError_t e_ = (call);                                                                             \
+        if (e_ != cudaSuccess)                                                                               \
+            return fail(c, e_ == cudaErrorMemoryAllocation ? MDI_ERR_OOM : MDI_ERR_CUDA, "%s: %s", #call,     \
+                        cudaGetErrorString(e_));                                                             \
+    } while (0)
+
+template <typename T> int dalloc(mdi_ctx *c, T **p, size_t n, int64_t *account = nullptr) {
+    size_t bytes = std::max<size_t>(n, 1) * sizeof(T);
+    CU(cudaMalloc((void **)p, bytes));
+    CU(cudaMemset(*p, 0, bytes));
+    if (account) *account += (int64_t)bytes;
+    return MDI_OK;
+}
+
+inline void count_launch(mdi_ctx *c) {
+    if (c->capturing) ++c->cap_launches; else ++c->st.kernel_launches;
+}
+
+// ---- kernel dispatch ------------------------------------------------------------------------------
+constexpr size_t LIN_SMEM_MAX = 200 * 1024;
+
+template <int NB, typename WT, int MODE> void lin_launch(const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st) {
+    k_linear<NB, WT, MODE><<<grid, LIN_THREADS, smem, st>>>(a, bt);
+}
+template <int NB, typename WT, int MODE> cudaError_t lin_attr() {
+    return cudaFuncSetAttribute(k_linear<NB, WT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LIN_SMEM_MAX);
+}
+template <typename WT, int MODE> void lin_nb(int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st) {
+    switch (nb) {
+        case 1: lin_launch<1, WT, MODE>(a, bt, grid, smem, st); break;
+        case 2: lin_launch<2, WT, MODE>(a, bt, grid, smem, st); break;
+        case 4: lin_launch<4, WT, MODE>(a, bt, grid, smem, st); break;
+        default: lin_launch<8, WT, MODE>(a, bt, grid, smem, st); break;
+    }
+}
+template <typename WT> void lin_mode(int mode, int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st) {
+    switch (mode) {
+        case LIN_QKV: lin_nb<WT, LIN_QKV>(nb, a, bt, grid, smem, st); break;
+        case LIN_ACT: lin_nb<WT, LIN_ACT>(nb, a, bt, grid, smem, st); break;
+        case LIN_GATEUP: lin_nb<WT, LIN_GATEUP>(nb, a, bt, grid, smem, st); break;
+        case LIN_HEAD: lin_nb<WT, LIN_HEAD>(nb, a, bt, grid, smem, st); break;
+        default: lin_nb<WT, LIN_RESID>(nb, a, bt, grid, smem, st); break;
+    }
+}
+template <typename WT, int MODE> cudaError_t lin_attr_nb() {
+    cudaError_t e;
+    if ((e = lin_attr<1, WT, MODE>()) != cudaSuccess) return e;
+    if ((e = lin_attr<2, WT, MODE>()) != cudaSuccess) return e;
+    if ((e = lin_attr<4, WT, MODE>()) != cudaSuccess) return e;
+    return lin_attr<8, WT, MODE>();
+}
+template <typename WT> cudaError_t lin_attr_all() {
+    cudaError_t e;
+    if ((e = lin_attr_nb<WT, LIN_QKV>()) != cudaSuccess) return e;
+    if ((e = lin_attr_nb<WT, LIN_ACT>()) != cudaSuccess) return e;
+    if ((e = lin_attr_nb<WT, LIN_GATEUP>()) != cudaSuccess) return e;
+    if ((e = lin_attr_nb<WT, LIN_HEAD>()) != cudaSuccess) return e;
+    return lin_attr_nb<WT, LIN_RESID>();
+}
+
+inline int round_nb(int n) { return n <= 1 ? 1 : n <= 2 ? 2 : n <= 4 ? 4 : 8; }
+
+Batch slice(const Batch &bt, int first, int n) {
+    Batch r{};
+    r.n = n;
+    for (int i = 0; i < n; ++i) { r.slot[i] = bt.slot[first + i]; r.off[i] = bt.off[first + i]; r.adv[i] = bt.adv[first + i]; }
+    return r;
+}
+
+// One linear layer over a batch; splits the batch when its inputs would not fit in shared memory.
+int linear(mdi_ctx *c, int mode, LinArgs a, const Batch &bt, cudaStream_t st) {
+    const bool f32 = c->s.weight_dtype == MDI_DTYPE_F32;
+    int maxb = (int)(LIN_SMEM_MAX / ((size_t)a.in_dim * 4));
+    maxb = maxb >= 8 ? 8 : maxb >= 4 ? 4 : maxb >= 2 ? 2 : 1;
+    if ((size_t)a.in_dim * 4 > LIN_SMEM_MAX) return fail(c, MDI_ERR_SHAPE, "input width %d too large", a.in_dim);
+    const int units = mode == LIN_GATEUP ? a.n_rows : (a.n_rows + 1) / 2;
+    const int grid = (units + LIN_WARPS - 1) / LIN_WARPS;
+    if (mode == LIN_HEAD && bt.n > maxb) return fail(c, MDI_ERR_SHAPE, "output layer batch does not fit");
+    for (int first = 0; first < bt.n; first += maxb) {
+        const int n = std::min(maxb, bt.n - first);
+        const int nb = round_nb(n);
+        Batch sb = slice(bt, first, n);
+        LinArgs b = a;
+        b.x_in = a.x_in + (size_t)first * a.in_dim;
+        if (a.q_out) b.q_out = a.q_out + (size_t)first * a.q_rows;
+        if (a.h_out) b.h_out = a.h_out + (size_t)first * a.n_rows;
+        if (a.x_res) b.x_res = a.x_res + (size_t)first * a.n_rows;
+        if (a.x_out) b.x_out = a.x_out + (size_t)first * a.n_rows;
+        const size_t smem = (size_t)nb * a.in_dim * 4;
+        if (f32) lin_mode<float>(mode, nb, b, sb, grid, smem, st);
+        else lin_mode<__nv_bfloat16>(mode, nb, b, sb, grid, smem, st);
+        count_launch(c);
+    }
+    return MDI_OK;
+}
+
+template <typename KT> void attn_hd(int hd, const AttnArgs &a, const Batch &bt, dim3 grid, cudaStream_t st) {
+    switch (hd) {
+        case 16: k_attn_decode<KT, 16><<<grid, ATT_THREADS, 0, st>>>(a, bt); break;
+        case 32: k_attn_decode<KT, 32><<<grid, ATT_THREADS, 0, st>>>(a, bt); break;
+        case 64: k_attn_decode<KT, 64><<<grid, ATT_THREADS, 0, st>>>(a, bt); break;
+        default: k_attn_decode<KT, 128><<<grid, ATT_THREADS, 0, st>>>(a, bt); break;
+    }
+}
+
+KvView kv_view(const mdi_ctx *c, const Partition &P) {
+    KvView v{};
+    v.pool = P.kv_pool;
+    v.page_table = P.pt_dev;
+    v.n_layers_local = P.hi - P.lo;
+    v.pages_per_seq = c->pages_per_seq;
+    v.page_tokens = c->page_tokens;
+    v.page_shift = c->page_shift;
+    v.n_kv_head = c->s.n_kv_head;
+    v.head_dim = c->s.head_dim;
+    v.page_elems = c->page_elems;
+    return v;
+}
+
+struct HeadReq {
+    int item = -1;          // item of the batch whose activation goes through the output layers (-1: all items)
+    bool update_state = true; // advance gen_count / cur_tok / tok_log
+    int *tok_out = nullptr;
+};
+
+// All kernels of one visit of a batch of items to partition p.
+//   x_in:  [n][d] input activations (ignored for p == 0, which embeds tokens from tok_src)
+//   x_out: [n][d] where the partition's output activations are written
+int enqueue_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in, const int *tok_src, int tok_by_slot,
+                           float *x_out, const HeadReq *head, cudaStream_t st) {
+    Partition &P = c->part[p];
+    const mdi_model_shape &s = c->s;
+    const bool f32 = s.weight_dtype == MDI_DTYPE_F32;
+    const int d = s.d_model, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim;
+    const int norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS;
+    if (p == 0) {
+        dim3 g((d + 255) / 256, bt.n);
+        if (f32) k_embed<float><<<g, 256, 0, st>>>((const float *)c->wte, (const float *)c->wpe, d, s.vocab, tok_src, tok_by_slot, P.pos_dev, bt, P.x_embed);
+        else k_embed<__nv_bfloat16><<<g, 256, 0, st>>>((const __nv_bfloat16 *)c->wte, (const __nv_bfloat16 *)c->wpe, d, s.vocab, tok_src, tok_by_slot, P.pos_dev, bt, P.x_embed);
+        count_launch(c);
+        x_in = P.x_embed;
+    }
+    const KvView kv = kv_view(c, P);
+    for (int l = P.lo; l < P.hi; ++l) {
+        const LayerW &L = c->layer[l];
+        const float *xin_l = l == P.lo ? x_in : x_out;
+        int rc;
+        {   // norm 1 + QKV projection (+ rotary) + cache append
+            LinArgs a{};
+            a.W = L.wqkv; a.bias = L.bqkv; a.n_rows = qw + 2 * kw; a.in_dim = d;
+            a.x_in = xin_l; a.norm = norm; a.gamma = L.ln1g; a.beta = L.ln1b; a.eps = s.norm_eps;
+            a.q_out = P.qbuf; a.q_rows = qw; a.kv_rows = kw; a.rope = s.arch == MDI_ARCH_LLAMA;
+            a.rope_cos = c->rope_cos; a.rope_sin = c->rope_sin; a.kv = kv; a.layer_local = l - P.lo; a.pos = P.pos_dev;
+            if ((rc = linear(c, LIN_QKV, a, bt, st)) != MDI_OK) return rc;
+        }
+        {   // attention over the slot's cache
+            AttnArgs a{};
+            a.q = P.qbuf; a.o = P.obuf; a.part = P.part; a.ticket = P.attn_ticket; a.kv = kv;
+            a.layer_local = l - P.lo; a.n_head = s.n_head; a.n_split = c->n_split; a.pos = P.pos_dev;
+            a.scale = 1.0f / std::sqrt((float)s.head_dim);
+            dim3 g(s.n_head, c->n_split, bt.n);
+            if (f32) attn_hd<float>(s.head_dim, a, bt, g, st); else attn_hd<__nv_bfloat16>(s.head_dim, a, bt, g, st);
+            count_launch(c);
+        }
+        {   // output projection + residual
+            LinArgs a{};
+            a.W = L.wo; a.bias = L.bo; a.n_rows = d; a.in_dim = qw; a.x_in = P.obuf; a.norm = NORM_NONE;
+            a.x_res = xin_l; a.x_out = x_out;
+            if ((rc = linear(c, LIN_RESID, a, bt, st)) != MDI_OK) return rc;
+        }
+        if (s.act == MDI_ACT_SWIGLU) {
+            LinArgs a{};
+            a.W = L.wgate; a.W2 = L.wup; a.n_rows = s.d_ff; a.in_dim = d; a.x_in = x_out; a.norm = norm;
+            a.gamma = L.ln2g; a.beta = L.ln2b; a.eps = s.norm_eps; a.h_out = P.hbuf;
+            if ((rc = linear(c, LIN_GATEUP, a, bt, st)) != MDI_OK) return rc;
+        } else {
+            LinArgs a{};
+            a.W = L.w1; a.bias = L.b1; a.n_rows = s.d_ff; a.in_dim = d; a.x_in = x_out; a.norm = norm;
+            a.gamma = L.ln2g; a.beta = L.ln2b; a.eps = s.norm_eps; a.h_out = P.hbuf; a.act = s.act == MDI_ACT_GELU_ERF;
+            if ((rc = linear(c, LIN_ACT, a, bt, st)) != MDI_OK) return rc;
+        }
+        {   // second MLP matrix + residual; the last block also advances the slots' positions
+            LinArgs a{};
+            a.W = s.act == MDI_ACT_SWIGLU ? L.wdown : L.w2; a.bias = L.b2; a.n_rows = d; a.in_dim = s.d_ff;
+            a.x_in = P.hbuf; a.norm = NORM_NONE; a.x_res = x_out; a.x_out = x_out;
+            a.pos_adv = l == P.hi - 1 ? P.pos_dev : nullptr;
+            if ((rc = linear(c, LIN_RESID, a, bt, st)) != MDI_OK) return rc;
+        }
+    }
+    if (head && p == c->K - 1) {
+        Batch hb = head->item < 0 ? bt : slice(bt, head->item, 1);
+        LinArgs a{};
+        a.W = s.tied_lm_head ? c->wte : c->lm_head; a.n_rows = s.vocab; a.in_dim = d;
+        a.x_in = head->item < 0 ? x_out : x_out + (size_t)head->item * d;
+        a.norm = norm; a.gamma = c->lnfg; a.beta = c->lnfb; a.eps = s.norm_eps;
+        a.logits = c->logits; a.part_val = c->head_pv; a.part_idx = c->head_pi; a.ticket = c->head_ticket;
+        a.tok_out = head->tok_out; a.log_stride = s.n_ctx;
+        if (head->update_state) {
+            a.cur_tok = c->cur_tok; a.tok_log = c->tok_log; a.gen_count = c->gen_count;
+            a.teacher = c->teacher; a.n_teacher = c->n_teacher;
+        }
+        int rc = linear(c, LIN_HEAD, a, hb, st);
+        if (rc != MDI_OK) return rc;
+    }
+    if (c->capturing) ++c->cap_steps; else ++c->st.stage_steps;
+    return MDI_OK;
+}
+
+int check_weights(mdi_ctx *c) {
+    if (c->n_loaded == (int)c->tensors.size()) return MDI_OK;
+    for (auto &kv : c->tensors)
+        if (!kv.second.loaded) return fail(c, MDI_ERR_STATE, "tensor '%s' was never loaded", kv.first.c_str());
+    return MDI_OK;
+}
+
+// Map pages so that rows [0, rows) of `slot` exist in every local layer of partition p.
+int ensure_pages(mdi_ctx *c, int p, int slot, int rows) {
+    Partition &P = c->part[p];
+    const int Lp = P.hi - P.lo;
+    const int need = (rows + c->page_tokens - 1) >> c->page_shift;
+    int &have = P.pages_of_slot[slot];
+    if (need <= have) return MDI_OK;
+    if (need > c->pages_per_seq) return fail(c, MDI_ERR_CONTEXT, "slot %d: %d rows exceed n_ctx", slot, rows);
+    if ((size_t)(need - have) * Lp > P.free_pages.size())
+        return fail(c, MDI_ERR_OOM, "key/value page pool of partition %d exhausted (%zu free, %d needed)", p,
+                    P.free_pages.size(), (need - have) * Lp);
+    for (int l = 0; l < Lp; ++l)
+        for (int g = have; g < need; ++g) {
+            P.pt_host[((size_t)slot * Lp + l) * c->pages_per_seq + g] = P.free_pages.back();
+            P.free_pages.pop_back();
+        }
+    have = need;
+    const size_t off = (size_t)slot * Lp * c->pages_per_seq, n = (size_t)Lp * c->pages_per_seq;
+    CU(cudaMemcpyAsync(P.pt_dev + off, P.pt_host.data() + off, n * sizeof(int), cudaMemcpyHostToDevice, P.stream));
+    return MDI_OK;
+}
+
+} // namespace
+
+// ====================================================================================================
+extern "C" {
+
+const char *mdi_last_error(mdi_ctx *ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+void mdi_destroy(mdi_ctx *c) {
+    if (!c) return;
+    cudaSetDevice(c->dev);
+    cudaDeviceSynchronize();
+    for (auto &g : c->graphs) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
+    for (auto &t : c->tensors) {
+        if (t.second.mat && *t.second.mat) cudaFree(*t.second.mat);
+        if (t.second.vec && *t.second.vec) cudaFree(*t.second.vec);
+    }
+    for (auto &P : c->part) {
+        void *ptrs[] = {P.kv_pool, P.pt_dev, P.pos_dev, P.x_embed, P.qbuf, P.obuf, P.hbuf, P.part, P.x_last, P.attn_ticket,
+                        P.ring, P.pf_buf[0], P.pf_buf[1]};
+        for (void *q : ptrs) if (q) cudaFree(q);
+        for (auto e : P.ev_edge) cudaEventDestroy(e);
+        for (auto e : P.ev_edge_cap) cudaEventDestroy(e);
+        for (int i = 0; i < 2; ++i) { if (P.ev_pf_out[i]) cudaEventDestroy(P.ev_pf_out[i]); if (P.ev_pf_used[i]) cudaEventDestroy(P.ev_pf_used[i]); }
+        if (P.ev_join) cudaEventDestroy(P.ev_join);
+        if (P.ev_join_cap) cudaEventDestroy(P.ev_join_cap);
+        if (P.stream) cudaStreamDestroy(P.stream);
+    }
+    void *ptrs[] = {c->rope_cos, c->rope_sin, c->logits, c->head_pv, c->head_pi, c->head_ticket, c->cur_tok, c->tok_log,
+                    c->gen_count, c->teacher, c->n_teacher, c->prompt_buf};
+    for (void *q : ptrs) if (q) cudaFree(q);
+    cudaEvent_t evs[] = {c->ev_fork, c->ev_fork_cap, c->ev_t0, c->ev_t1, c->ev_pf0, c->ev_pf1};
+    for (auto e : evs) if (e) cudaEventDestroy(e);
+    if (c->main) cudaStreamDestroy(c->main);
+    delete c;
+}
+
+int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int n_samples, const mdi_options *opts,
+               mdi_ctx **out) {
+    mdi_ctx *c = nullptr;
+    if (!shape || !part_bounds || !out) return fail(c, MDI_ERR_ARG, "null argument");
+    *out = nullptr;
+    const mdi_model_shape &s = *shape;
+    if (K < 1 || n_samples < 1) return fail(c, MDI_ERR_ARG, "K and n_samples must be positive");
+    if (part_bounds[0] != 0 || part_bounds[K] != s.n_layer) return fail(c, MDI_ERR_ARG, "partition bounds must run from 0 to n_layer");
+    for (int p = 0; p < K; ++p)
+        if (part_bounds[p + 1] <= part_bounds[p]) return fail(c, MDI_ERR_ARG, "partition bounds must be strictly ascending");
+    if (s.arch != MDI_ARCH_GPT && s.arch != MDI_ARCH_LLAMA) return fail(c, MDI_ERR_ARG, "unknown arch");
+    if (s.weight_dtype != MDI_DTYPE_F32 && s.weight_dtype != MDI_DTYPE_BF16) return fail(c, MDI_ERR_ARG, "unknown weight dtype");
+    if (s.act < 0 || s.act > 2) return fail(c, MDI_ERR_ARG, "unknown activation");
+    if (s.n_layer < 1 || s.d_model < 1 || s.n_head < 1 || s.n_kv_head < 1 || s.d_ff < 1 || s.vocab < 1 || s.n_ctx < 1)
+        return fail(c, MDI_ERR_ARG, "non-positive dimension");
+    if ((s.arch == MDI_ARCH_LLAMA) != (s.act == MDI_ACT_SWIGLU)) return fail(c, MDI_ERR_SHAPE, "SwiGLU goes with the Llama block, GELU with the GPT block");
+    if (s.arch == MDI_ARCH_LLAMA && (s.has_bias || s.tied_lm_head)) return fail(c, MDI_ERR_SHAPE, "Llama block: no biases, untied output layer");
+    if (s.arch == MDI_ARCH_GPT && !s.has_bias) return fail(c, MDI_ERR_SHAPE, "GPT block: biases required");
+    const int vec = s.weight_dtype == MDI_DTYPE_F32 ? 4 : 8;
+    if (s.head_dim != 16 && s.head_dim != 32 && s.head_dim != 64 && s.head_dim != 128)
+        return fail(c, MDI_ERR_SHAPE, "head_dim must be 16, 32, 64 or 128");
+    if (s.n_head % s.n_kv_head) return fail(c, MDI_ERR_SHAPE, "n_head must be a multiple of n_kv_head");
+    if (s.d_model % vec || s.d_ff % vec || (s.n_head * s.head_dim) % vec)
+        return fail(c, MDI_ERR_SHAPE, "d_model, d_ff and n_head*head_dim must be multiples of %d", vec);
+    if ((size_t)std::max(s.d_model, s.d_ff) * 4 > LIN_SMEM_MAX) return fail(c, MDI_ERR_SHAPE, "layer width too large");
+
+    c = new mdi_ctx();
+    c->s = s;
+    if (opts) c->o = *opts;
+    c->K = K;
+    c->S = n_samples;
+    cudaError_t e = cudaGetDevice(&c->dev);
+    if (e != cudaSuccess) { int rc = fail(nullptr, MDI_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(e)); delete c; return rc; }
+    auto bail = [&](int rc) { g_create_error = c->err; mdi_destroy(c); return rc; };
+    int rc;
+#define TRY(x) do { if ((rc = (x)) != MDI_OK) return bail(rc); } while (0)
+#define CUB(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return bail(fail(c, e_ == cudaErrorMemoryAllocation ? MDI_ERR_OOM : MDI_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_))); } while (0)
+
+    c->page_tokens = c->o.page_tokens > 0 ? c->o.page_tokens : 16;
+    if (c->page_tokens & (c->page_tokens - 1)) return bail(fail(c, MDI_ERR_ARG, "page_tokens must be a power of two"));
+    c->page_shift = 0;
+    while ((1 << c->page_shift) < c->page_tokens) ++c->page_shift;
+    c->pages_per_seq = (s.n_ctx + c->page_tokens - 1) / c->page_tokens;
+    c->esize = s.weight_dtype == MDI_DTYPE_F32 ? 4 : 2;
+    c->page_elems = (size_t)2 * s.n_kv_head * c->page_tokens * s.head_dim;
+    c->n_split = c->o.attn_splits > 0 ? c->o.attn_splits : std::max(1, std::min(16, s.n_ctx / 128));
+    c->rounds_per_graph = c->o.rounds_per_graph != 0 ? c->o.rounds_per_graph : 16;
+    const int G = std::min(n_samples, K);
+    c->gmax = (n_samples + G - 1) / G;
+    const long pool_tokens = c->o.kv_pool_tokens > 0 ? c->o.kv_pool_tokens : (long)n_samples * s.n_ctx;
+
+    CUB((lin_attr_all<float>()));
+    CUB((lin_attr_all<__nv_bfloat16>()));
+    CUB(cudaStreamCreateWithFlags(&c->main, cudaStreamNonBlocking));
+    cudaEvent_t *evs[] = {&c->ev_fork, &c->ev_fork_cap};
+    for (auto ev : evs) CUB(cudaEventCreateWithFlags(ev, cudaEventDisableTiming));
+    cudaEvent_t *tevs[] = {&c->ev_t0, &c->ev_t1, &c->ev_pf0, &c->ev_pf1};
+    for (auto ev : tevs) CUB(cudaEventCreate(ev));
+
+    // tensors
+    c->layer.resize(s.n_layer);
+    const int d = s.d_model, F = s.d_ff, V = s.vocab, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim;
+    auto part_of = [&](int l) { int p = 0; while (l >= part_bounds[p + 1]) ++p; return p; };
+    auto mat = [&](const std::string &n, void **dst, size_t el, int p) { TensorSlot t; t.mat = dst; t.elems = el; t.partition = p; c->tensors[n] = t; };
+    auto vecr = [&](const std::string &n, float **dst, size_t el, int p) { TensorSlot t; t.vec = dst; t.elems = el; t.partition = p; c->tensors[n] = t; };
+    mat("wte", &c->wte, (size_t)V * d, 0);
+    if (s.arch == MDI_ARCH_GPT) mat("wpe", &c->wpe, (size_t)s.n_ctx * d, 0);
+    for (int i = 0; i < s.n_layer; ++i) {
+        LayerW &L = c->layer[i];
+        const std::string pfx = "h." + std::to_string(i) + ".";
+        const int p = part_of(i);
+        vecr(pfx + "ln1.g", &L.ln1g, d, p);
+        if (s.arch == MDI_ARCH_GPT) vecr(pfx + "ln1.b", &L.ln1b, d, p);
+        mat(pfx + "attn.wqkv", &L.wqkv, (size_t)(qw + 2 * kw) * d, p);
+        if (s.has_bias) vecr(pfx + "attn.bqkv", &L.bqkv, qw + 2 * kw, p);
+        mat(pfx + "attn.wo", &L.wo, (size_t)d * qw, p);
+        if (s.has_bias) vecr(pfx + "attn.bo", &L.bo, d, p);
+        vecr(pfx + "ln2.g", &L.ln2g, d, p);
+        if (s.arch == MDI_ARCH_GPT) vecr(pfx + "ln2.b", &L.ln2b, d, p);
+        if (s.act == MDI_ACT_SWIGLU) {
+            mat(pfx + "mlp.wgate", &L.wgate, (size_t)F * d, p);
+            mat(pfx + "mlp.wup", &L.wup, (size_t)F * d, p);
+            mat(pfx + "mlp.wdown", &L.wdown, (size_t)d * F, p);
+        } else {
+            mat(pfx + "mlp.w1", &L.w1, (size_t)F * d, p);
+            vecr(pfx + "mlp.b1", &L.b1, F, p);
+            mat(pfx + "mlp.w2", &L.w2, (size_t)d * F, p);
+            vecr(pfx + "mlp.b2", &L.b2, d, p);
+        }
+    }
+    vecr("lnf.g", &c->lnfg, d, K - 1);
+    if (s.arch == MDI_ARCH_GPT) vecr("lnf.b", &c->lnfb, d, K - 1);
+    if (!s.tied_lm_head) mat("lm_head", &c->lm_head, (size_t)V * d, K - 1);
+
+    // rotary tables, evaluated in fp64 on the host
+    if (s.arch == MDI_ARCH_LLAMA) {
+        const int half = s.head_dim / 2;
+        std::vector<float> hc((size_t)s.n_ctx * half), hs((size_t)s.n_ctx * half);
+        for (int pos = 0; pos < s.n_ctx; ++pos)
+            for (int i = 0; i < half; ++i) {
+                const double ang = (double)pos * std::pow((double)s.rope_theta, -2.0 * i / (double)s.head_dim);
+                hc[(size_t)pos * half + i] = (float)std::cos(ang);
+                hs[(size_t)pos * half + i] = (float)std::sin(ang);
+            }
+        TRY(dalloc(c, &c->rope_cos, hc.size()));
+        TRY(dalloc(c, &c->rope_sin, hs.size()));
+        CUB(cudaMemcpy(c->rope_cos, hc.data(), hc.size() * 4, cudaMemcpyHostToDevice));
+        CUB(cudaMemcpy(c->rope_sin, hs.data(), hs.size() * 4, cudaMemcpyHostToDevice));
+    }
+
+    // partitions
+    c->part.resize(K);
+    for (int p = 0; p < K; ++p) {
+        Partition &P = c->part[p];
+        P.lo = part_bounds[p];
+        P.hi = part_bounds[p + 1];
+        const int Lp = P.hi - P.lo;
+        CUB(cudaStreamCreateWithFlags(&P.stream, cudaStreamNonBlocking));
+        const long pages_per_layer = (pool_tokens + c->page_tokens - 1) / c->page_tokens;
+        P.n_pages = (int)(pages_per_layer * Lp);
+        P.kv_bytes = (size_t)P.n_pages * c->page_elems * c->esize;
+        CUB(cudaMalloc(&P.kv_pool, std::max<size_t>(P.kv_bytes, 16)));
+        CUB(cudaMemset(P.kv_pool, 0, std::max<size_t>(P.kv_bytes, 16)));
+        P.free_pages.resize(P.n_pages);
+        for (int i = 0; i < P.n_pages; ++i) P.free_pages[i] = P.n_pages - 1 - i;
+        P.pt_host.assign((size_t)n_samples * Lp * c->pages_per_seq, 0);
+        P.pages_of_slot.assign(n_samples, 0);
+        P.pos_host.assign(n_samples, 0);
+        TRY(dalloc(c, &P.pt_dev, P.pt_host.size(), &P.buffer_bytes));
+        TRY(dalloc(c, &P.pos_dev, (size_t)n_samples, &P.buffer_bytes));
+        if (p == 0) TRY(dalloc(c, &P.x_embed, (size_t)MAXB * d, &P.buffer_bytes));
+        TRY(dalloc(c, &P.qbuf, (size_t)MAXB * qw, &P.buffer_bytes));
+        TRY(dalloc(c, &P.obuf, (size_t)MAXB * qw, &P.buffer_bytes));
+        TRY(dalloc(c, &P.hbuf, (size_t)MAXB * F, &P.buffer_bytes));
+        TRY(dalloc(c, &P.part, (size_t)MAXB * s.n_head * c->n_split * (s.head_dim + 2), &P.buffer_bytes));
+        TRY(dalloc(c, &P.attn_ticket, (size_t)MAXB * s.n_head, &P.buffer_bytes));
+        TRY(dalloc(c, &P.x_last, (size_t)std::max(MAXB, c->gmax) * d, &P.buffer_bytes));
+        if (p < K - 1) {
+            TRY(dalloc(c, &P.ring, (size_t)G * c->gmax * d, &P.buffer_bytes));
+            for (int i = 0; i < 2; ++i) TRY(dalloc(c, &P.pf_buf[i], (size_t)s.n_ctx * d, &P.buffer_bytes));
+        }
+        P.ev_edge.resize(G);
+        P.ev_edge_cap.resize(G);
+        for (int j = 0; j < G; ++j) {
+            CUB(cudaEventCreateWithFlags(&P.ev_edge[j], cudaEventDisableTiming));
+            CUB(cudaEventCreateWithFlags(&P.ev_edge_cap[j], cudaEventDisableTiming));
+        }
+        for (int i = 0; i < 2; ++i) {
+            CUB(cudaEventCreateWithFlags(&P.ev_pf_out[i], cudaEventDisableTiming));
+            CUB(cudaEventCreateWithFlags(&P.ev_pf_used[i], cudaEventDisableTiming));
+        }
+        CUB(cudaEventCreateWithFlags(&P.ev_join, cudaEventDisableTiming));
+        CUB(cudaEventCreateWithFlags(&P.ev_join_cap, cudaEventDisableTiming));
+    }
+    for (auto &t : c->tensors) c->part[t.second.partition].weight_bytes += (int64_t)t.second.elems * (t.second.mat ? c->esize : 4);
+
+    // output layers and token state
+    const int head_units = (V + 1) / 2;
+    c->head_grid = (head_units + LIN_WARPS - 1) / LIN_WARPS;
+    int64_t *acc = &c->part[K - 1].buffer_bytes;
+    TRY(dalloc(c, &c->logits, (size_t)n_samples * V, acc));
+    TRY(dalloc(c, &c->head_pv, (size_t)MAXB * c->head_grid, acc));
+    TRY(dalloc(c, &c->head_pi, (size_t)MAXB * c->head_grid, acc));
+    TRY(dalloc(c, &c->head_ticket, 1, acc));
+    TRY(dalloc(c, &c->cur_tok, (size_t)n_samples));
+    TRY(dalloc(c, &c->gen_count, (size_t)n_samples));
+    TRY(dalloc(c, &c->n_teacher, (size_t)n_samples));
+    TRY(dalloc(c, &c->tok_log, (size_t)n_samples * s.n_ctx));
+    TRY(dalloc(c, &c->teacher, (size_t)n_samples * s.n_ctx));
+    TRY(dalloc(c, &c->prompt_buf, (size_t)n_samples * s.n_ctx));
+    c->gen_host.assign(n_samples, 0);
+    c->returned_host.assign(n_samples, 0);
+    c->prefilled.assign(n_samples, 0);
+    CUB(cudaDeviceSynchronize());
+#undef TRY
+#undef CUB
+    *out = c;
+    return MDI_OK;
+}
+
+int mdi_load_weights(mdi_ctx *c, const char *name, const void *host, size_t nbytes) {
+    if (!c || !name || !host) return fail(c, MDI_ERR_ARG, "null argument");
+    auto it = c->tensors.find(name);
+    if (it == c->tensors.end()) return fail(c, MDI_ERR_ARG, "unknown tensor '%s'", name);
+    TensorSlot &t = it->second;
+    if (nbytes != t.elems * c->esize) return fail(c, MDI_ERR_SHAPE, "tensor '%s': %zu bytes given, %zu expected", name, nbytes, t.elems * c->esize);
+    CU(cudaSetDevice(c->dev));
+    if (t.mat) {
+        if (!*t.mat) CU(cudaMalloc(t.mat, nbytes));
+        CU(cudaMemcpy(*t.mat, host, nbytes, cudaMemcpyHostToDevice));
+    } else {
+        std::vector<float> f(t.elems);
+        if (c->s.weight_dtype == MDI_DTYPE_F32) memcpy(f.data(), host, nbytes);
+        else {
+            const uint16_t *h = (const uint16_t *)host;
+            for (size_t i = 0; i < t.elems; ++i) { uint32_t u = (uint32_t)h[i] << 16; memcpy(&f[i], &u, 4); }
+        }
+        if (!*t.vec) CU(cudaMalloc((void **)t.vec, t.elems * 4));
+        CU(cudaMemcpy(*t.vec, f.data(), t.elems * 4, cudaMemcpyHostToDevice));
+    }
+    if (!t.loaded) { t.loaded = true; ++c->n_loaded; }
+    return MDI_OK;
+}
+
+int mdi_reset_sample(mdi_ctx *c, int sample) {
+    if (!c) return MDI_ERR_ARG;
+    if (sample < 0 || sample >= c->S) return fail(c, MDI_ERR_ARG, "sample %d out of range", sample);
+    CU(cudaSetDevice(c->dev));
+    CU(cudaDeviceSynchronize());
+    const int zero = 0;
+    for (auto &P : c->part) {
+        const int Lp = P.hi - P.lo;
+        for (int l = 0; l < Lp; ++l)
+            for (int g = 0; g < P.pages_of_slot[sample]; ++g) {
+                int &pg = P.pt_host[((size_t)sample * Lp + l) * c->pages_per_seq + g];
+                P.free_pages.push_back(pg);
+                pg = 0;
+            }
+        P.pages_of_slot[sample] = 0;
+        P.pos_host[sample] = 0;
+        CU(cudaMemcpy(P.pos_dev + sample, &zero, 4, cudaMemcpyHostToDevice));
+    }
+    CU(cudaMemcpy(c->gen_count + sample, &zero, 4, cudaMemcpyHostToDevice));
+    CU(cudaMemcpy(c->n_teacher + sample, &zero, 4, cudaMemcpyHostToDevice));
+    c->gen_host[sample] = c->returned_host[sample] = c->prefilled[sample] = 0;
+    return MDI_OK;
+}
+
+int mdi_set_teacher_tokens(mdi_ctx *c, int sample, const int32_t *tok, int n) {
+    if (!c) return MDI_ERR_ARG;
+    if (sample < 0 || sample >= c->S || n < 0 || (n > 0 && !tok)) return fail(c, MDI_ERR_ARG, "bad argument");
+    if (n > c->s.n_ctx) return fail(c, MDI_ERR_CONTEXT, "more teacher tokens than n_ctx");
+    if (c->prefilled[sample]) return fail(c, MDI_ERR_STATE, "set teacher tokens before the sample's prefill");
+    CU(cudaSetDevice(c->dev));
+    if (n) CU(cudaMemcpy(c->teacher + (size_t)sample * c->s.n_ctx, tok, (size_t)n * 4, cudaMemcpyHostToDevice));
+    CU(cudaMemcpy(c->n_teacher + sample, &n, 4, cudaMemcpyHostToDevice));
+    return MDI_OK;
+}
+
+static int prefill_impl(mdi_ctx *c, int sample, const int32_t *prompt, int n, bool on_device) {
+    if (!c || !prompt) return fail(c, MDI_ERR_ARG, "null argument");
+    if (sample < 0 || sample >= c->S || n < 1) return fail(c, MDI_ERR_ARG, "bad sample or prompt length");
+    if (n > c->s.n_ctx) return fail(c, MDI_ERR_CONTEXT, "prompt of %d tokens exceeds n_ctx %d", n, c->s.n_ctx);
+    if (c->prefilled[sample]) return fail(c, MDI_ERR_STATE, "sample %d already holds tokens", sample);
+    for (auto &P : c->part) if (P.pos_host[sample]) return fail(c, MDI_ERR_STATE, "sample %d already holds tokens", sample);
+    int rc = check_weights(c);
+    if (rc != MDI_OK) return rc;
+    CU(cudaSetDevice(c->dev));
+    if (!on_device)
+        for (int i = 0; i < n; ++i)
+            if (prompt[i] < 0 || prompt[i] >= c->s.vocab) return fail(c, MDI_ERR_ARG, "token id %d out of range", prompt[i]);
+    for (int p = 0; p < c->K; ++p) if ((rc = ensure_pages(c, p, sample, n)) != MDI_OK) return rc;
+    const int d = c->s.d_model, K = c->K;
+    int *pbuf = c->prompt_buf + (size_t)sample * c->s.n_ctx;
+    CU(cudaMemcpyAsync(pbuf, prompt, (size_t)n * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->part[0].stream));
+    const int par = c->pf_count & 1;
+    if (!c->pf_open) { CU(cudaEventRecord(c->ev_pf0, c->part[0].stream)); c->pf_open = true; }
+    for (int p = 0; p < K; ++p) {
+        Partition &P = c->part[p];
+        if (p > 0) CU(cudaStreamWaitEvent(P.stream, c->part[p - 1].ev_pf_out[par], 0));
+        if (p < K - 1 && c->part[p + 1].pf_used_valid[par]) CU(cudaStreamWaitEvent(P.stream, c->part[p + 1].ev_pf_used[par], 0));
+        for (int c0 = 0; c0 < n; c0 += MAXB) {
+            const int m = std::min(MAXB, n - c0);
+            Batch bt{};
+            bt.n = m;
+            for (int i = 0; i < m; ++i) { bt.slot[i] = sample; bt.off[i] = i; bt.adv[i] = i == 0 ? m : 0; }
+            const float *x_in = p > 0 ? c->part[p - 1].pf_buf[par] + (size_t)c0 * d : nullptr;
+            float *x_out = p < K - 1 ? P.pf_buf[par] + (size_t)c0 * d : P.x_last;
+            HeadReq hr;
+            hr.item = m - 1;
+            const bool last_chunk = c0 + m == n;
+            rc = enqueue_partition_step(c, p, bt, x_in, pbuf + c0, 0, x_out, last_chunk ? &hr : nullptr, P.stream);
+            if (rc != MDI_OK) return rc;
+        }
+        CU(cudaEventRecord(P.ev_pf_out[par], P.stream));
+        if (p > 0) { CU(cudaEventRecord(P.ev_pf_used[par], P.stream)); P.pf_used_valid[par] = true; }
+        P.pos_host[sample] += n;
+    }
+    CU(cudaEventRecord(c->ev_pf1, c->part[K - 1].stream));
+    CU(cudaGetLastError());
+    ++c->pf_count;
+    c->prefilled[sample] = 1;
+    c->gen_host[sample] = 1;
+    c->returned_host[sample] = 0;
+    ++c->st.tokens_generated;
+    return MDI_OK;
+}
+
+int mdi_prefill(mdi_ctx *c, int sample, const int32_t *prompt_host, int n) { return prefill_impl(c, sample, prompt_host, n, false); }
+int mdi_prefill_dev(mdi_ctx *c, int sample, const int32_t *prompt_dev, int n) { return prefill_impl(c, sample, prompt_dev, n, true); }
+
+int mdi_step(mdi_ctx *c, int p, int slot, const void *act_in, void *act_out) {
+    if (!c || !act_in || !act_out) return fail(c, MDI_ERR_ARG, "null argument");
+    if (p < 0 || p >= c->K || slot < 0 || slot >= c->S) return fail(c, MDI_ERR_ARG, "partition or slot out of range");
+    int rc = check_weights(c);
+    if (rc != MDI_OK) return rc;
+    CU(cudaSetDevice(c->dev));
+    Partition &P = c->part[p];
+    if (P.pos_host[slot] + 1 > c->s.n_ctx) return fail(c, MDI_ERR_CONTEXT, "slot %d is full (%d rows)", slot, P.pos_host[slot]);
+    if ((rc = ensure_pages(c, p, slot, P.pos_host[slot] + 1)) != MDI_OK) return rc;
+    Batch bt{};
+    bt.n = 1; bt.slot[0] = slot; bt.off[0] = 0; bt.adv[0] = 1;
+    HeadReq hr;
+    hr.item = 0; hr.update_state = false; hr.tok_out = (int *)act_out;
+    const bool last = p == c->K - 1;
+    rc = enqueue_partition_step(c, p, bt, (const float *)act_in, (const int *)act_in, 0, last ? P.x_last : (float *)act_out,
+                                last ? &hr : nullptr, P.stream);
+    if (rc != MDI_OK) return rc;
+    CU(cudaGetLastError());
+    ++P.pos_host[slot];
+    return MDI_OK;
+}
+
+// Enqueue ticks [t_begin, t_end) of the recurrent schedule.  The ring has K phase slots: at tick t
+// partition p serves phase (t - p) mod K, pass (t - p) / K; phases 0..G-1 carry the G sample groups and
+// the others are idle (fewer samples than partitions).  Handoffs whose producer lies before t_begin are
+// already ordered by the fork at the start of the segment.
+static int enqueue_ticks(mdi_ctx *c, int n_samples, int G, long t_begin, long t_end, long total_slots) {
+    const int K = c->K, d = c->s.d_model;
+    const bool cap = c->capturing;
+    cudaEvent_t fork = cap ? c->ev_fork_cap : c->ev_fork;
+    CU(cudaEventRecord(fork, c->main));
+    for (int p = 0; p < K; ++p) CU(cudaStreamWaitEvent(c->part[p].stream, fork, 0));
+    for (long t = t_begin; t < t_end; ++t)
+        for (int p = 0; p < K; ++p) {
+            const long v = t - p;
+            if (v < 0 || v >= total_slots) continue;
+            const int j = (int)(v % K);
+            if (j >= G) continue;
+            Partition &P = c->part[p];
+            const int prev = (p + K - 1) % K;
+            // producer of this step's input: partition p-1 one tick earlier (for p = 0: the last partition,
+            // which chose the token; none on a group's first pass of this call)
+            const bool has_producer = p > 0 || v >= K;
+            if (has_producer && t - 1 >= t_begin && K > 1)
+                CU(cudaStreamWaitEvent(P.stream, cap ? c->part[prev].ev_edge_cap[j] : c->part[prev].ev_edge[j], 0));
+            // the group's samples, in sub-batches of at most MAXB
+            std::vector<int> members;
+            for (int smp = j; smp < n_samples; smp += G) members.push_back(smp);
+            for (size_t first = 0; first < members.size(); first += MAXB) {
+                const int m = (int)std::min<size_t>(MAXB, members.size() - first);
+                Batch bt{};
+                bt.n = m;
+                for (int i = 0; i < m; ++i) { bt.slot[i] = members[first + i]; bt.off[i] = 0; bt.adv[i] = 1; }
+                const float *x_in = p > 0 ? c->part[p - 1].ring + ((size_t)j * c->gmax + first) * d : nullptr;
+                float *x_out = p < K - 1 ? P.ring + ((size_t)j * c->gmax + first) * d : P.x_last;
+                HeadReq hr;
+                int rc = enqueue_partition_step(c, p, bt, x_in, c->cur_tok, 1, x_out, &hr, P.stream);
+                if (rc != MDI_OK) return rc;
+            }
+            CU(cudaEventRecord(cap ? P.ev_edge_cap[j] : P.ev_edge[j], P.stream));
+        }
+    for (int p = 0; p < K; ++p) {
+        cudaEvent_t ej = cap ? c->part[p].ev_join_cap : c->part[p].ev_join;
+        CU(cudaEventRecord(ej, c->part[p].stream));
+        CU(cudaStreamWaitEvent(c->main, ej, 0));
+    }
+    return MDI_OK;
+}
+
+static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, bool on_device) {
+    if (!c || !out) return fail(c, MDI_ERR_ARG, "null argument");
+    if (n_samples < 1 || n_samples > c->S || n_new < 0) return fail(c, MDI_ERR_ARG, "bad n_samples or n_new_tokens");
+    int rc = check_weights(c);
+    if (rc != MDI_OK) return rc;
+    CU(cudaSetDevice(c->dev));
+    const int K = c->K, G = std::min(n_samples, K);
+    if ((n_samples + G - 1) / G > c->gmax) return fail(c, MDI_ERR_ARG, "group size exceeds what the context was created for");
+    const int pending = c->gen_host[0] - c->returned_host[0];
+    for (int smp = 0; smp < n_samples; ++smp) {
+        if (!c->prefilled[smp]) return fail(c, MDI_ERR_STATE, "sample %d has not been prefilled", smp);
+        if (c->gen_host[smp] - c->returned_host[smp] != pending) return fail(c, MDI_ERR_STATE, "samples are at different points of generation");
+    }
+    const int n_pass = std::max(0, n_new - pending);
+    for (int smp = 0; smp < n_samples; ++smp) {
+        if (c->part[0].pos_host[smp] + n_pass > c->s.n_ctx)
+            return fail(c, MDI_ERR_CONTEXT, "sample %d: %d cached + %d new positions exceed n_ctx %d", smp, c->part[0].pos_host[smp], n_pass, c->s.n_ctx);
+        if (c->gen_host[smp] + n_pass > c->s.n_ctx) return fail(c, MDI_ERR_CONTEXT, "token log full");
+    }
+    for (int p = 0; p < K; ++p)
+        for (int smp = 0; smp < n_samples; ++smp)
+            if ((rc = ensure_pages(c, p, smp, c->part[p].pos_host[smp] + n_pass)) != MDI_OK) return rc;
+
+    // everything enqueued so far (prefills, page tables) precedes the schedule
+    for (int p = 0; p < K; ++p) {
+        CU(cudaEventRecord(c->part[p].ev_join, c->part[p].stream));
+        CU(cudaStreamWaitEvent(c->main, c->part[p].ev_join, 0));
+    }
+    CU(cudaEventRecord(c->ev_t0, c->main));
+    const long total = (long)n_pass * K;        // phase slots per partition
+    const long t_total = total ? total + K - 1 : 0;
+    long t = 0;
+    if (t_total) {
+        const int R = c->rounds_per_graph;
+        const long W = R > 0 ? (long)R * K : 0;
+        const long t_steady = K > 1 ? K : 0; // first tick, multiple of K, from which every partition is in steady state
+        if (W > 0 && t_steady + 2 * W <= total) {
+            if ((rc = enqueue_ticks(c, n_samples, G, 0, t_steady, total)) != MDI_OK) return rc;
+            t = t_steady;
+            auto key = std::make_pair(n_samples, (int)W);
+            GraphEntry &ge = c->graphs[key];
+            if (!ge.exec) {
+                cudaGraph_t graph = nullptr;
+                CU(cudaStreamBeginCapture(c->main, cudaStreamCaptureModeThreadLocal));
+                c->capturing = true;
+                c->cap_launches = c->cap_steps = 0;
+                rc = enqueue_ticks(c, n_samples, G, t_steady, t_steady + W, 1L << 60);
+                c->capturing = false;
+                cudaError_t e = cudaStreamEndCapture(c->main, &graph);
+                if (rc != MDI_OK) { if (graph) cudaGraphDestroy(graph); c->graphs.erase(key); return rc; }
+                if (e != cudaSuccess) { c->graphs.erase(key); return fail(c, MDI_ERR_CUDA, "graph capture: %s", cudaGetErrorString(e)); }
+                e = cudaGraphInstantiate(&ge.exec, graph, 0);
+                cudaGraphDestroy(graph);
+                if (e != cudaSuccess) { c->graphs.erase(key); return fail(c, MDI_ERR_CUDA, "graph instantiate: %s", cudaGetErrorString(e)); }
+                ge.launches = c->cap_launches;
+                ge.steps = c->cap_steps;
+            }
+            while (t + W <= total) {
+                CU(cudaGraphLaunch(ge.exec, c->main));
+                c->st.kernel_launches += ge.launches;
+                c->st.stage_steps += ge.steps;
+                t += W;
+            }
+        }
+        if ((rc = enqueue_ticks(c, n_samples, G, t, t_total, total)) != MDI_OK) return rc;
+    }
+    CU(cudaEventRecord(c->ev_t1, c->main));
+    CU(cudaGetLastError());
+    // tokens: entries [returned, returned + n_new) of each sample's log
+    for (int smp = 0; smp < n_samples; ++smp) {
+        if (n_new)
+            CU(cudaMemcpyAsync(out + (size_t)smp * n_new, c->tok_log + (size_t)smp * c->s.n_ctx + c->returned_host[smp], (size_t)n_new * 4,
+                               on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, c->main));
+        for (int p = 0; p < K; ++p) c->part[p].pos_host[smp] += n_pass;
+        c->gen_host[smp] += n_pass;
+        c->returned_host[smp] += n_new;
+        c->st.tokens_generated += n_pass;
+    }
+    CU(cudaStreamSynchronize(c->main));
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->ev_t0, c->ev_t1) == cudaSuccess) c->st.last_generate_ms = ms;
+    if (c->pf_open) {
+        if (cudaEventElapsedTime(&ms, c->ev_pf0, c->ev_pf1) == cudaSuccess) c->st.last_prefill_ms = ms;
+        if (cudaEventElapsedTime(&ms, c->ev_pf0, c->ev_t1) == cudaSuccess) c->st.last_run_ms = ms;
+        c->pf_open = false;
+    }
+    return MDI_OK;
+}
+
+int mdi_generate(mdi_ctx *c, int n_samples, int n_new, int32_t *out_host) { return generate_impl(c, n_samples, n_new, out_host, false); }
+int mdi_generate_dev(mdi_ctx *c, int n_samples, int n_new, int32_t *out_dev) { return generate_impl(c, n_samples, n_new, out_dev, true); }
+
+int mdi_get_logits(mdi_ctx *c, int sample, float *out_host) {
+    if (!c || !out_host) return fail(c, MDI_ERR_ARG, "null argument");
+    if (sample < 0 || sample >= c->S) return fail(c, MDI_ERR_ARG, "sample out of range");
+    CU(cudaSetDevice(c->dev));
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemcpy(out_host, c->logits + (size_t)sample * c->s.vocab, (size_t)c->s.vocab * 4, cudaMemcpyDeviceToHost));
+    return MDI_OK;
+}
+
+int mdi_sync(mdi_ctx *c) {
+    if (!c) return MDI_ERR_ARG;
+    CU(cudaSetDevice(c->dev));
+    for (auto &P : c->part) CU(cudaStreamSynchronize(P.stream));
+    CU(cudaStreamSynchronize(c->main));
+    return MDI_OK;
+}
+
+int mdi_get_stats(mdi_ctx *c, mdi_stats *out) {
+    if (!c || !out) return fail(c, MDI_ERR_ARG, "null argument");
+    int rc = mdi_sync(c);
+    if (rc != MDI_OK) return rc;
+    if (c->pf_open) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->ev_pf0, c->ev_pf1) == cudaSuccess) c->st.last_prefill_ms = ms;
+    }
+    c->st.n_partitions = c->K;
+    c->st.n_samples = c->S;
+    c->st.n_groups = std::min(c->S, c->K);
+    for (int p = 0; p < c->K && p < 16; ++p) {
+        c->st.weight_bytes[p] = c->part[p].weight_bytes;
+        c->st.kv_pool_bytes[p] = (int64_t)c->part[p].kv_bytes;
+        c->st.kv_pages_in_use[p] = c->part[p].n_pages - (int64_t)c->part[p].free_pages.size();
+    }
+    *out = c->st;
+    return MDI_OK;
+}
+
+int64_t mdi_memory_bytes(mdi_ctx *c, int p) {
+    if (!c || p < 0 || p >= c->K) return MDI_ERR_ARG;
+    return c->part[p].weight_bytes + (int64_t)c->part[p].kv_bytes + c->part[p].buffer_bytes;
+}
+
+} // extern "C"
