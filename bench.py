@@ -171,8 +171,12 @@ def main():
     ap.add_argument("--workload", default="gpt2_small", choices=I.WORKLOAD_ORDER)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--rounds-per-graph", type=int, default=0)
+    ap.add_argument("--n-new", type=int, default=0, help="shorter generation (profiler captures only; not the headline)")
+    ap.add_argument("--n-prompt", type=int, default=0, help="shorter prompts (profiler captures only)")
     args = ap.parse_args()
     w = I.WORKLOADS[args.workload]
+    if args.n_new or args.n_prompt:
+        w = I.scaled(w, n_new=args.n_new or w.n_new, n_prompt=args.n_prompt or w.n_prompt)
     from paper_2505_18164_b200 import build
     build.build_inputs()
 
@@ -195,7 +199,7 @@ def main():
 
     s = w.shape
     S, P, N = w.n_samples, w.n_prompt, w.n_new
-    ctx = mdi.Context(s, list(w.part_bounds), S, kv_pool_tokens=S * (P + N), rounds_per_graph=args.rounds_per_graph)
+    ctx = mdi.Context(s, list(w.part_bounds), S, kv_pool_tokens=S * ((P + N + 15) // 16 * 16), rounds_per_graph=args.rounds_per_graph)
     weights = {}
     for name, a in I.iter_weights(s, w.weight_seed):
         ctx.load_weights(name, a)
