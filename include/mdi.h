@@ -67,7 +67,12 @@ typedef struct {
     int kv_pool_tokens;/* tokens of cache each partition's pool can hold over all samples
                           (default n_samples * n_ctx, rounded up to pages) */
     int attn_splits;   /* sequence splits of decode attention (default: chosen from n_ctx) */
-    int rounds_per_graph; /* rounds of the recurrent schedule captured per CUDA graph (default 16; <0: no graphs) */
+    int rounds_per_graph; /* stream scheduler: rounds of the recurrent schedule captured per CUDA graph
+                             (default 16; <0: no graphs) */
+    int scheduler;     /* how mdi_generate runs the recurrent pipeline.  0: the persistent kernel (one launch,
+                          one team of thread blocks per partition, flag handoff between teams) when the shape
+                          fits it (groups of at most 4 samples), else the stream scheduler; 1: always the
+                          stream scheduler (one stream per partition, event handoff); 2: persistent or fail */
 } mdi_options;
 
 typedef struct {
@@ -154,6 +159,14 @@ int mdi_reset_sample(mdi_ctx *ctx, int sample);
 int mdi_get_stats(mdi_ctx *ctx, mdi_stats *out);
 /* Device bytes held by one partition (parameters + key/value pool + buffers), cf. Tables I-II. */
 int64_t mdi_memory_bytes(mdi_ctx *ctx, int partition);
+/* Tracing aid (the paper times token arrival on the starter; here each partition's team of thread
+ * blocks times itself).  With MDI_PK_PROFILE set in the environment at mdi_create, the persistent kernel
+ * accumulates, per thread block, the nanoseconds spent in: [0] waiting for the input edge, [1] staging
+ * and normalising inputs, [2] streaming weight tiles, [3] team barriers, [4] attention, [5] choosing
+ * tokens, [6] producer warp waiting for a free ring slot, [7] producer warp total.  This call averages
+ * them over the partition's blocks for the last mdi_generate, in milliseconds, into out_ms[0..n).
+ * Returns the number of blocks of the partition (> 0) or a negative error (STATE when timing is off). */
+int mdi_get_partition_times(mdi_ctx *ctx, int partition, double *out_ms, int n);
 /* Wait for everything enqueued on the context's streams. */
 int mdi_sync(mdi_ctx *ctx);
 /* Text of the last error of this context (or of the last failed mdi_create if ctx is NULL). */

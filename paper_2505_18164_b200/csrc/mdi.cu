@@ -14,6 +14,7 @@
 #include <string>
 #include <vector>
 
+#include "persistent_decode.cuh"
 #include "step_kernels.cuh"
 
 using namespace mdi;
@@ -99,6 +100,18 @@ struct mdi_ctx {
     std::map<std::pair<int, int>, GraphEntry> graphs; // (n_samples, window ticks)
     bool capturing = false;
     int64_t cap_launches = 0, cap_steps = 0;
+    // persistent decode kernel
+    bool pk_ok = false, pk_prof_on = false, pk_tables_stale = true;
+    int pk_slots = 0, pk_xs_floats = 0, pk_nb = 1, n_sm = 0, scheduler = 0;
+    size_t pk_smem = 0;
+    std::vector<PkTeam> pk_teams_host;
+    std::vector<PkPhase> pk_phases_host;
+    std::vector<int> pk_phase_begin, pk_phase_count;
+    PkTeam *pk_teams = nullptr;
+    PkPhase *pk_phases = nullptr;
+    unsigned *pk_sync = nullptr; // [K][64]: word 0 team barrier, words 32.. output-edge flags
+    int *pk_err = nullptr;
+    unsigned long long *pk_prof = nullptr; // [n_sm][PK_PROF_N]
     mdi_stats st{};
     std::string err;
 };
@@ -354,6 +367,184 @@ int ensure_pages(mdi_ctx *c, int p, int slot, int rows) {
     return MDI_OK;
 }
 
+
+// ---- persistent decode kernel: tables and launch -----------------------------------------------------
+template <typename WT> cudaError_t pk_attr(size_t smem) {
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(k_persistent_decode<WT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(k_persistent_decode<WT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    return cudaFuncSetAttribute(k_persistent_decode<WT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+template <typename WT> const void *pk_func(int nb) {
+    return nb == 1 ? (const void *)k_persistent_decode<WT, 1> : nb == 2 ? (const void *)k_persistent_decode<WT, 2>
+                                                                        : (const void *)k_persistent_decode<WT, 4>;
+}
+
+// Phase list of every partition, team sizes (blocks per partition, in proportion to the bytes a step
+// streams), shared-memory budget.  Leaves pk_ok false when the shape does not fit this kernel
+// (groups of more than 4 samples, or too little shared memory for two ring slots).
+int pk_setup(mdi_ctx *c) {
+    const mdi_model_shape &s = c->s;
+    const int K = c->K, d = s.d_model, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim;
+    cudaDeviceProp prop;
+    CU(cudaGetDeviceProperties(&prop, c->dev));
+    c->n_sm = prop.multiProcessorCount;
+    if (c->scheduler == 1) return MDI_OK;
+    const bool want = c->scheduler == 2;
+    if (c->gmax > PK_MAXNB) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: at most %d samples per group", PK_MAXNB) : MDI_OK;
+    if (K > 32 || K > c->n_sm) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: too many partitions") : MDI_OK;
+    c->pk_nb = c->gmax <= 1 ? 1 : c->gmax <= 2 ? 2 : 4;
+    const int max_in = std::max(std::max(d, s.d_ff), qw);
+    c->pk_xs_floats = c->pk_nb * ((max_in + 255) & ~255);
+    const size_t misc = (size_t)(256 * 8 + 128 + 128 + 8 + 2 * PK_CWARPS * PK_MAXNB + 2 + PK_MAX_SLOTS) * 4 + 2 * PK_MAX_SLOTS * 8 + 128;
+    const size_t fixed = (size_t)c->pk_xs_floats * 4 + misc;
+    const size_t budget = (size_t)prop.sharedMemPerBlockOptin;
+    if (fixed + 2 * PK_SLOT_BYTES > budget) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: inputs do not fit in shared memory") : MDI_OK;
+    c->pk_slots = (int)std::min<size_t>(PK_MAX_SLOTS, (budget - fixed) / PK_SLOT_BYTES);
+    c->pk_smem = fixed + (size_t)c->pk_slots * PK_SLOT_BYTES;
+    CU(s.weight_dtype == MDI_DTYPE_F32 ? pk_attr<float>(c->pk_smem) : pk_attr<__nv_bfloat16>(c->pk_smem));
+
+    std::vector<PkPhase> &ph = c->pk_phases_host;
+    ph.clear();
+    c->pk_phase_begin.assign(K, 0);
+    c->pk_phase_count.assign(K, 0);
+    std::vector<double> bytes(K, 0.0);
+    const bool rope = s.arch == MDI_ARCH_LLAMA;
+    auto blocks16 = [](int n) { return (n + PK_SEGS - 1) / PK_SEGS; };
+    for (int p = 0; p < K; ++p) {
+        Partition &P = c->part[p];
+        c->pk_phase_begin[p] = (int)ph.size();
+        for (int l = P.lo; l < P.hi; ++l) {
+            PkPhase q{};
+            q.kind = PK_QKV; q.n_rows = qw + 2 * kw; q.in_dim = d; q.layer_local = l - P.lo; q.first_layer = l == P.lo;
+            q.n_blocks = rope ? (q.n_rows / 2 + 7) / 8 : blocks16(q.n_rows);
+            ph.push_back(q);
+            PkPhase a{}; a.kind = PK_ATTN; a.layer_local = l - P.lo; ph.push_back(a);
+            PkPhase o{}; o.kind = PK_OUT; o.n_rows = d; o.in_dim = qw; o.n_blocks = blocks16(d); o.layer_local = l - P.lo; o.first_layer = l == P.lo; ph.push_back(o);
+            PkPhase f{};
+            if (s.act == MDI_ACT_SWIGLU) { f.kind = PK_GATEUP; f.n_rows = s.d_ff; f.in_dim = d; f.n_blocks = (s.d_ff + 7) / 8; }
+            else { f.kind = PK_FC1; f.n_rows = s.d_ff; f.in_dim = d; f.n_blocks = blocks16(s.d_ff); }
+            f.layer_local = l - P.lo; ph.push_back(f);
+            PkPhase g{}; g.kind = PK_FC2; g.n_rows = d; g.in_dim = s.d_ff; g.n_blocks = blocks16(d); g.layer_local = l - P.lo; ph.push_back(g);
+            bytes[p] += (double)((size_t)(qw + 2 * kw) * d + (size_t)d * qw + (size_t)(s.act == MDI_ACT_SWIGLU ? 3 : 2) * s.d_ff * d) * c->esize;
+        }
+        if (p == K - 1) {
+            PkPhase h{}; h.kind = PK_HEAD; h.n_rows = s.vocab; h.in_dim = d; h.n_blocks = blocks16(s.vocab); ph.push_back(h);
+            bytes[p] += (double)s.vocab * d * c->esize;
+        }
+        c->pk_phase_count[p] = (int)ph.size() - c->pk_phase_begin[p];
+    }
+    // team sizes
+    std::vector<int> n_cta(K, 1);
+    const char *env = getenv("MDI_TEAM_CTAS");
+    bool from_env = false;
+    if (env) {
+        std::vector<int> v;
+        const char *q = env;
+        while (*q) { v.push_back(atoi(q)); while (*q && *q != ',') ++q; if (*q == ',') ++q; }
+        int tot = 0;
+        for (int x : v) tot += x;
+        if ((int)v.size() == K && tot <= c->n_sm && *std::min_element(v.begin(), v.end()) >= 1) { n_cta = v; from_env = true; }
+    }
+    if (!from_env) {
+        double tot = 0;
+        for (double b : bytes) tot += b;
+        int used = 0, big = 0;
+        for (int p = 0; p < K; ++p) {
+            n_cta[p] = std::max(1, (int)std::floor(c->n_sm * bytes[p] / tot));
+            used += n_cta[p];
+            if (bytes[p] > bytes[big]) big = p;
+        }
+        n_cta[big] += c->n_sm - used;
+        if (n_cta[big] < 1) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: not enough SMs") : MDI_OK;
+    }
+    c->pk_teams_host.assign(K, PkTeam{});
+    int first = 0, rcx;
+    if ((rcx = dalloc(c, &c->pk_sync, (size_t)K * 64)) != MDI_OK) return rcx;
+    if ((rcx = dalloc(c, &c->pk_err, 1)) != MDI_OK) return rcx;
+    if ((rcx = dalloc(c, &c->pk_prof, (size_t)c->n_sm * PK_PROF_N)) != MDI_OK) return rcx;
+    c->pk_prof_on = getenv("MDI_PK_PROFILE") != nullptr;
+    for (int p = 0; p < K; ++p) {
+        Partition &P = c->part[p];
+        PkTeam &T = c->pk_teams_host[p];
+        T.first_cta = first; T.n_cta = n_cta[p]; first += n_cta[p];
+        T.phase_begin = c->pk_phase_begin[p]; T.n_phases = c->pk_phase_count[p];
+        T.is_first = p == 0; T.is_last = p == K - 1;
+        T.n_split = std::max(1, std::min(16, n_cta[p] / (c->pk_nb * s.n_head)));
+        T.kv = kv_view(c, P);
+        T.qbuf = P.qbuf; T.part = P.part; T.hbuf = P.hbuf; T.x_embed = P.x_embed; T.x_last = P.x_last;
+        T.ring_in = p > 0 ? c->part[p - 1].ring : nullptr;
+        T.ring_out = p < K - 1 ? P.ring : nullptr;
+        T.pos = P.pos_dev;
+        T.bar = c->pk_sync + (size_t)p * 64;
+        T.flag_out = c->pk_sync + (size_t)p * 64 + 32;
+        T.flag_in = c->pk_sync + (size_t)((p + K - 1) % K) * 64 + 32;
+    }
+    if ((rcx = dalloc(c, &c->pk_teams, (size_t)K)) != MDI_OK) return rcx;
+    if ((rcx = dalloc(c, &c->pk_phases, ph.size())) != MDI_OK) return rcx;
+    CU(cudaMemcpy(c->pk_teams, c->pk_teams_host.data(), sizeof(PkTeam) * K, cudaMemcpyHostToDevice));
+    c->pk_ok = true;
+    return MDI_OK;
+}
+
+// Weight pointers are known once the tensors are loaded: (re)write the device phase table when they changed.
+int pk_fill_phases(mdi_ctx *c) {
+    if (!c->pk_tables_stale) return MDI_OK;
+    const mdi_model_shape &s = c->s;
+    std::vector<PkPhase> &ph = c->pk_phases_host;
+    for (int p = 0; p < c->K; ++p) {
+        Partition &P = c->part[p];
+        for (int i = 0; i < c->pk_phase_count[p]; ++i) {
+            PkPhase &q = ph[c->pk_phase_begin[p] + i];
+            if (q.kind == PK_HEAD) {
+                q.W = s.tied_lm_head ? c->wte : c->lm_head; q.gamma = c->lnfg; q.beta = c->lnfb;
+                continue;
+            }
+            const LayerW &L = c->layer[P.lo + q.layer_local];
+            switch (q.kind) {
+                case PK_QKV: q.W = L.wqkv; q.bias = L.bqkv; q.gamma = L.ln1g; q.beta = L.ln1b; break;
+                case PK_OUT: q.W = L.wo; q.bias = L.bo; break;
+                case PK_FC1: q.W = L.w1; q.bias = L.b1; q.gamma = L.ln2g; q.beta = L.ln2b; break;
+                case PK_GATEUP: q.W = L.wgate; q.W2 = L.wup; q.gamma = L.ln2g; q.beta = L.ln2b; break;
+                case PK_FC2: q.W = s.act == MDI_ACT_SWIGLU ? L.wdown : L.w2; q.bias = L.b2; break;
+                default: break;
+            }
+        }
+    }
+    CU(cudaMemcpy(c->pk_phases, ph.data(), sizeof(PkPhase) * ph.size(), cudaMemcpyHostToDevice));
+    c->pk_tables_stale = false;
+    return MDI_OK;
+}
+
+// One cooperative launch that runs n_pass passes of the recurrent pipeline for samples 0..n_samples-1.
+int pk_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
+    const mdi_model_shape &s = c->s;
+    int rc = pk_fill_phases(c);
+    if (rc != MDI_OK) return rc;
+    CU(cudaMemsetAsync(c->pk_sync, 0, (size_t)c->K * 64 * sizeof(unsigned), c->main));
+    CU(cudaMemsetAsync(c->pk_err, 0, sizeof(int), c->main));
+    if (c->pk_prof_on) CU(cudaMemsetAsync(c->pk_prof, 0, (size_t)c->n_sm * PK_PROF_N * 8, c->main));
+    PkParams P{};
+    P.d = s.d_model; P.n_head = s.n_head; P.n_kv_head = s.n_kv_head; P.head_dim = s.head_dim; P.d_ff = s.d_ff; P.vocab = s.vocab;
+    P.norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS; P.act = s.act == MDI_ACT_GELU_ERF; P.rope = s.arch == MDI_ARCH_LLAMA;
+    P.K = c->K; P.G = G; P.n_samples = n_samples; P.gmax = c->gmax; P.n_pass = n_pass; P.n_slots_ring = c->pk_slots; P.xs_floats = c->pk_xs_floats;
+    P.eps = s.norm_eps; P.scale = 1.0f / std::sqrt((float)s.head_dim);
+    P.teams = c->pk_teams; P.phases = c->pk_phases; P.wte = c->wte; P.wpe = c->wpe; P.rope_cos = c->rope_cos; P.rope_sin = c->rope_sin;
+    P.logits = c->logits; P.head_pv = c->head_pv; P.head_pi = c->head_pi; P.cur_tok = c->cur_tok; P.tok_log = c->tok_log;
+    P.gen_count = c->gen_count; P.teacher = c->teacher; P.n_teacher = c->n_teacher; P.log_stride = s.n_ctx; P.err = c->pk_err;
+    P.prof = c->pk_prof_on ? c->pk_prof : nullptr;
+    int grid = 0;
+    for (auto &T : c->pk_teams_host) grid += T.n_cta;
+    const int nb = (n_samples + G - 1) / G;
+    const int tnb = nb <= 1 ? 1 : nb <= 2 ? 2 : 4;
+    const void *fn = s.weight_dtype == MDI_DTYPE_F32 ? pk_func<float>(tnb) : pk_func<__nv_bfloat16>(tnb);
+    void *args[] = {&P};
+    CU(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(PK_THREADS), args, c->pk_smem, c->main));
+    ++c->st.kernel_launches;
+    c->st.stage_steps += (int64_t)c->K * n_pass * G;
+    return MDI_OK;
+}
+
 } // namespace
 
 // ====================================================================================================
@@ -382,7 +573,7 @@ void mdi_destroy(mdi_ctx *c) {
         if (P.stream) cudaStreamDestroy(P.stream);
     }
     void *ptrs[] = {c->rope_cos, c->rope_sin, c->logits, c->head_pv, c->head_pi, c->head_ticket, c->cur_tok, c->tok_log,
-                    c->gen_count, c->teacher, c->n_teacher, c->prompt_buf};
+                    c->gen_count, c->teacher, c->n_teacher, c->prompt_buf, c->pk_teams, c->pk_phases, c->pk_sync, c->pk_err, c->pk_prof};
     for (void *q : ptrs) if (q) cudaFree(q);
     cudaEvent_t evs[] = {c->ev_fork, c->ev_fork_cap, c->ev_t0, c->ev_t1, c->ev_pf0, c->ev_pf1};
     for (auto e : evs) if (e) cudaEventDestroy(e);
@@ -437,6 +628,8 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     c->page_elems = (size_t)2 * s.n_kv_head * c->page_tokens * s.head_dim;
     c->n_split = c->o.attn_splits > 0 ? c->o.attn_splits : std::max(1, std::min(16, s.n_ctx / 128));
     c->rounds_per_graph = c->o.rounds_per_graph != 0 ? c->o.rounds_per_graph : 16;
+    c->scheduler = c->o.scheduler;
+    if (c->scheduler < 0 || c->scheduler > 2) return bail(fail(c, MDI_ERR_ARG, "scheduler must be 0, 1 or 2"));
     const int G = std::min(n_samples, K);
     c->gmax = (n_samples + G - 1) / G;
     const long pool_tokens = c->o.kv_pool_tokens > 0 ? c->o.kv_pool_tokens : (long)n_samples * s.n_ctx;
@@ -524,7 +717,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
         TRY(dalloc(c, &P.qbuf, (size_t)MAXB * qw, &P.buffer_bytes));
         TRY(dalloc(c, &P.obuf, (size_t)MAXB * qw, &P.buffer_bytes));
         TRY(dalloc(c, &P.hbuf, (size_t)MAXB * F, &P.buffer_bytes));
-        TRY(dalloc(c, &P.part, (size_t)MAXB * s.n_head * c->n_split * (s.head_dim + 2), &P.buffer_bytes));
+        TRY(dalloc(c, &P.part, (size_t)MAXB * s.n_head * std::max(c->n_split, 16) * (s.head_dim + 2), &P.buffer_bytes));
         TRY(dalloc(c, &P.attn_ticket, (size_t)MAXB * s.n_head, &P.buffer_bytes));
         TRY(dalloc(c, &P.x_last, (size_t)std::max(MAXB, c->gmax) * d, &P.buffer_bytes));
         if (p < K - 1) {
@@ -551,8 +744,8 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     c->head_grid = (head_units + LIN_WARPS - 1) / LIN_WARPS;
     int64_t *acc = &c->part[K - 1].buffer_bytes;
     TRY(dalloc(c, &c->logits, (size_t)n_samples * V, acc));
-    TRY(dalloc(c, &c->head_pv, (size_t)MAXB * c->head_grid, acc));
-    TRY(dalloc(c, &c->head_pi, (size_t)MAXB * c->head_grid, acc));
+    TRY(dalloc(c, &c->head_pv, (size_t)MAXB * std::max(c->head_grid, 1024), acc));
+    TRY(dalloc(c, &c->head_pi, (size_t)MAXB * std::max(c->head_grid, 1024), acc));
     TRY(dalloc(c, &c->head_ticket, 1, acc));
     TRY(dalloc(c, &c->cur_tok, (size_t)n_samples));
     TRY(dalloc(c, &c->gen_count, (size_t)n_samples));
@@ -563,6 +756,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     c->gen_host.assign(n_samples, 0);
     c->returned_host.assign(n_samples, 0);
     c->prefilled.assign(n_samples, 0);
+    TRY(pk_setup(c));
     CUB(cudaDeviceSynchronize());
 #undef TRY
 #undef CUB
@@ -591,6 +785,7 @@ int mdi_load_weights(mdi_ctx *c, const char *name, const void *host, size_t nbyt
         CU(cudaMemcpy(*t.vec, f.data(), t.elems * 4, cudaMemcpyHostToDevice));
     }
     if (!t.loaded) { t.loaded = true; ++c->n_loaded; }
+    c->pk_tables_stale = true;
     return MDI_OK;
 }
 
@@ -782,7 +977,11 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
     const long total = (long)n_pass * K;        // phase slots per partition
     const long t_total = total ? total + K - 1 : 0;
     long t = 0;
-    if (t_total) {
+    const bool use_pk = c->pk_ok && c->scheduler != 1 && (n_samples + G - 1) / G <= PK_MAXNB;
+    if (c->scheduler == 2 && !use_pk) return fail(c, MDI_ERR_SHAPE, "persistent scheduler unavailable for this call");
+    if (t_total && use_pk) {
+        if ((rc = pk_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
+    } else if (t_total) {
         const int R = c->rounds_per_graph;
         const long W = R > 0 ? (long)R * K : 0;
         const long t_steady = K > 1 ? K : 0; // first tick, multiple of K, from which every partition is in steady state
@@ -829,6 +1028,11 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
         c->st.tokens_generated += n_pass;
     }
     CU(cudaStreamSynchronize(c->main));
+    if (t_total && use_pk) {
+        int kerr = 0;
+        CU(cudaMemcpy(&kerr, c->pk_err, sizeof(int), cudaMemcpyDeviceToHost));
+        if (kerr) return fail(c, MDI_ERR_TIMEOUT, "persistent decode kernel gave up waiting (code %d: 1 edge flag, 2 team barrier, 3 weight tile, 4 ring slot)", kerr);
+    }
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, c->ev_t0, c->ev_t1) == cudaSuccess) c->st.last_generate_ms = ms;
     if (c->pf_open) {
@@ -877,6 +1081,23 @@ int mdi_get_stats(mdi_ctx *c, mdi_stats *out) {
     }
     *out = c->st;
     return MDI_OK;
+}
+
+int mdi_get_partition_times(mdi_ctx *c, int p, double *out_ms, int n) {
+    if (!c || !out_ms) return fail(c, MDI_ERR_ARG, "null argument");
+    if (p < 0 || p >= c->K || n < 1) return fail(c, MDI_ERR_ARG, "partition out of range");
+    if (!c->pk_ok || !c->pk_prof_on) return fail(c, MDI_ERR_STATE, "in-kernel timing is off (set MDI_PK_PROFILE=1 before mdi_create; persistent scheduler only)");
+    CU(cudaSetDevice(c->dev));
+    CU(cudaDeviceSynchronize());
+    const PkTeam &T = c->pk_teams_host[p];
+    std::vector<unsigned long long> h((size_t)T.n_cta * PK_PROF_N);
+    CU(cudaMemcpy(h.data(), c->pk_prof + (size_t)T.first_cta * PK_PROF_N, h.size() * 8, cudaMemcpyDeviceToHost));
+    for (int i = 0; i < n; ++i) {
+        double acc = 0;
+        for (int k = 0; k < T.n_cta && i < PK_PROF_N; ++k) acc += (double)h[(size_t)k * PK_PROF_N + i];
+        out_ms[i] = acc / T.n_cta * 1e-6;
+    }
+    return T.n_cta;
 }
 
 int64_t mdi_memory_bytes(mdi_ctx *c, int p) {

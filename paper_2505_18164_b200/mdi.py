@@ -22,7 +22,7 @@ _ERR_NAMES = {ERR_ARG: "MDI_ERR_ARG", ERR_SHAPE: "MDI_ERR_SHAPE", ERR_OOM: "MDI_
 
 EXPORTS = ["mdi_create", "mdi_destroy", "mdi_load_weights", "mdi_prefill", "mdi_prefill_dev", "mdi_step",
            "mdi_generate", "mdi_generate_dev", "mdi_get_logits", "mdi_set_teacher_tokens", "mdi_reset_sample",
-           "mdi_get_stats", "mdi_memory_bytes", "mdi_sync", "mdi_last_error"]
+           "mdi_get_stats", "mdi_get_partition_times", "mdi_memory_bytes", "mdi_sync", "mdi_last_error"]
 
 
 class MdiError(RuntimeError):
@@ -40,7 +40,7 @@ class ModelShape(ctypes.Structure):
 
 class Options(ctypes.Structure):
     _fields_ = [("page_tokens", ctypes.c_int), ("kv_pool_tokens", ctypes.c_int), ("attn_splits", ctypes.c_int),
-                ("rounds_per_graph", ctypes.c_int)]
+                ("rounds_per_graph", ctypes.c_int), ("scheduler", ctypes.c_int)]
 
 
 class Stats(ctypes.Structure):
@@ -77,6 +77,7 @@ def lib():
         L.mdi_set_teacher_tokens.argtypes = [vp, ci, vp, ci]
         L.mdi_reset_sample.argtypes = [vp, ci]
         L.mdi_get_stats.argtypes = [vp, ctypes.POINTER(Stats)]
+        L.mdi_get_partition_times.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_double), ci]
         L.mdi_memory_bytes.argtypes = [vp, ci]
         L.mdi_memory_bytes.restype = ctypes.c_int64
         L.mdi_sync.argtypes = [vp]
@@ -101,14 +102,14 @@ class Context:
     """One model on one GPU: mdi_create ... mdi_destroy."""
 
     def __init__(self, shape, part_bounds: Sequence[int], n_samples: int, page_tokens: int = 0,
-                 kv_pool_tokens: int = 0, attn_splits: int = 0, rounds_per_graph: int = 0):
+                 kv_pool_tokens: int = 0, attn_splits: int = 0, rounds_per_graph: int = 0, scheduler: int = 0):
         self._h = None
         self.shape = shape
         self.K = len(part_bounds) - 1
         self.n_samples = n_samples
         cs = ModelShape(**{n: getattr(shape, n) for n, _ in ModelShape._fields_})
         bounds = (ctypes.c_int * len(part_bounds))(*part_bounds)
-        opts = Options(page_tokens, kv_pool_tokens, attn_splits, rounds_per_graph)
+        opts = Options(page_tokens, kv_pool_tokens, attn_splits, rounds_per_graph, scheduler)
         h = ctypes.c_void_p()
         rc = lib().mdi_create(ctypes.byref(cs), bounds, self.K, n_samples, ctypes.byref(opts), ctypes.byref(h))
         if rc != MDI_OK:
@@ -120,9 +121,9 @@ class Context:
             raise MdiError(rc, (lib().mdi_last_error(self._h) or b"").decode())
 
     def close(self):
-        if self._h:
-            lib().mdi_destroy(self._h)
-            self._h = None
+        if self._h and _lib is not None:
+            _lib.mdi_destroy(self._h)
+        self._h = None
 
     __del__ = close
 
@@ -176,6 +177,14 @@ class Context:
         st = Stats()
         self._check(lib().mdi_get_stats(self._h, ctypes.byref(st)))
         return st
+
+    def partition_times(self, partition: int):
+        """(blocks in the partition's team, [8] mean milliseconds per category) of the last generate."""
+        out = (ctypes.c_double * 8)()
+        rc = lib().mdi_get_partition_times(self._h, partition, out, 8)
+        if rc < 0:
+            self._check(rc)
+        return rc, list(out)
 
     def memory_bytes(self, partition: int) -> int:
         return lib().mdi_memory_bytes(self._h, partition)

@@ -70,16 +70,19 @@ CASES = [
     ("llama", I.DT_BF16, 2, 256, 2, 1, 300, 40, [0, 2], 11, 3, 10, {}),         # one partition, group > 8 items
     ("gpt", I.DT_F32, 2, 64, 4, None, 50, 32, [0, 1, 2], 3, 10, 22, {}),        # prompt + new == n_ctx exactly
     ("gpt", I.DT_BF16, 4, 64, 2, None, 97, 64, [0, 1, 2, 3, 4], 1, 4, 9, {}),   # one sample, four partitions
+    ("gpt", I.DT_BF16, 2, 256, 4, None, 2100, 48, [0, 1, 2], 4, 5, 8, {}),      # d_ff 1024+: several tiles per warp, 2 per group
+    ("gpt", I.DT_BF16, 4, 64, 2, None, 97, 64, [0, 1, 2, 3, 4], 1, 4, 9, {}),   # one sample, four partitions
 ]
 
 
+@pytest.mark.parametrize("scheduler", [0, 1], ids=["persistent", "streams"])
 @pytest.mark.parametrize("arch,dtype,L,d,H,n_kv,V,C,bounds,S,P,N,opts", CASES)
-def test_small_shapes_match_oracle(arch, dtype, L, d, H, n_kv, V, C, bounds, S, P, N, opts):
+def test_small_shapes_match_oracle(arch, dtype, L, d, H, n_kv, V, C, bounds, S, P, N, opts, scheduler):
     shape = tiny_shape(arch, dtype, L=L, d=d, H=H, V=V, C=C, n_kv=n_kv)
     orc, w = make_oracle(shape, seed=3, std=0.08 if dtype == I.DT_F32 else 0.04)
     prompts = I.make_prompts(V, S, P, seed=5)
     toks, lgs, margins = oracle_reference(orc, prompts, N)
-    ctx = _ctx(shape, bounds, S, w, **opts)
+    ctx = _ctx(shape, bounds, S, w, scheduler=scheduler, **opts)
     _check_teacher_forced_stepwise(ctx, shape, prompts, toks, lgs, margins, N)
     _check_free_running(ctx, shape, prompts, toks, margins, N)
     ctx.close()
@@ -106,14 +109,14 @@ def test_results_do_not_depend_on_partitioning_or_grouping():
         ctx.close()
 
 
-def test_graph_windows_equal_eager_schedule():
-    """A run long enough for the captured steady-state windows gives the same tokens as eager launches."""
+def test_schedulers_agree():
+    """Eager stream scheduler, captured steady-state windows and the persistent kernel give the same tokens."""
     shape = tiny_shape("gpt", I.DT_F32, L=3, d=64, H=4, V=97, C=128)
     orc, w = make_oracle(shape, seed=11, std=0.08)
     prompts = I.make_prompts(97, 3, 4, seed=2)
     outs = []
-    for rpg in (-1, 2, 5):
-        ctx = _ctx(shape, [0, 1, 2, 3], 3, w, rounds_per_graph=rpg)
+    for rpg, sched in ((-1, 1), (2, 1), (5, 1), (0, 2)):
+        ctx = _ctx(shape, [0, 1, 2, 3], 3, w, rounds_per_graph=rpg, scheduler=sched)
         for s in range(3):
             ctx.prefill(s, prompts[s])
         a = ctx.generate(3, 50)
@@ -122,7 +125,7 @@ def test_graph_windows_equal_eager_schedule():
         st = ctx.stats()
         assert st.kernel_launches > 0 and st.stage_steps > 0
         ctx.close()
-    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+    assert all(np.array_equal(outs[0], o) for o in outs[1:])
     toks, _, margins = oracle_reference(orc, prompts, 90)
     for s in range(3):
         low = np.nonzero(margins[s] <= 2e-4)[0]
