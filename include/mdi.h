@@ -163,7 +163,8 @@ int64_t mdi_memory_bytes(mdi_ctx *ctx, int partition);
  * blocks times itself).  With MDI_PK_PROFILE set in the environment at mdi_create, the persistent kernel
  * accumulates, per thread block, the nanoseconds spent in: [0] waiting for the input edge, [1] staging
  * and normalising inputs, [2] streaming weight tiles, [3] team barriers, [4] attention, [5] choosing
- * tokens, [6] producer warp waiting for a free ring slot, [7] producer warp total.  This call averages
+ * tokens, [6] producer warp waiting for a free ring slot, [7] producer warp total, and within [2]:
+ * [8] waiting for a tile to land, [9] multiply-accumulate, [10] reduction and epilogue.  This call averages
  * them over the partition's blocks for the last mdi_generate, in milliseconds, into out_ms[0..n).
  * Returns the number of blocks of the partition (> 0) or a negative error (STATE when timing is off). */
 int mdi_get_partition_times(mdi_ctx *ctx, int partition, double *out_ms, int n);

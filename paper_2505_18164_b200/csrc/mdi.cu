@@ -396,7 +396,8 @@ int pk_setup(mdi_ctx *c) {
     c->pk_nb = c->gmax <= 1 ? 1 : c->gmax <= 2 ? 2 : 4;
     const int max_in = std::max(std::max(d, s.d_ff), qw);
     c->pk_xs_floats = c->pk_nb * ((max_in + 255) & ~255);
-    const size_t misc = (size_t)(256 * 8 + 128 + 128 + 8 + 2 * PK_CWARPS * PK_MAXNB + 2 + PK_MAX_SLOTS) * 4 + 2 * PK_MAX_SLOTS * 8 + 128;
+    const size_t misc = (size_t)(256 * 8 + 128 + 128 + 16 + 2 * PK_CWARPS * PK_MAXNB + 2 + PK_MAX_SLOTS) * 4 + 2 * PK_MAX_SLOTS * 8 +
+                        PK_SMEM_PHASES * sizeof(PkPhase) + 128;
     const size_t fixed = (size_t)c->pk_xs_floats * 4 + misc;
     const size_t budget = (size_t)prop.sharedMemPerBlockOptin;
     if (fixed + 2 * PK_SLOT_BYTES > budget) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: inputs do not fit in shared memory") : MDI_OK;

@@ -19,6 +19,8 @@
 // word is set, the thread stops waiting for good, and the kernel runs to its end without further
 // waits; the host then reports MDI_ERR_TIMEOUT.  Nothing traps.
 #pragma once
+#include <type_traits>
+
 #include "step_kernels.cuh"
 
 namespace mdi {
@@ -30,11 +32,12 @@ constexpr int PK_SEGS = 16;
 constexpr int PK_SLOT_BYTES = 32768;
 constexpr int PK_MAX_SLOTS = 6;
 constexpr int PK_MAXNB = 4;
+constexpr int PK_SMEM_PHASES = 48; // phase descriptors of a team kept in shared memory (more: read from global memory)
 constexpr unsigned long long PK_WAIT_NS = 2000000000ull; // 2 s
 
 enum PkKind { PK_QKV = 0, PK_ATTN = 1, PK_OUT = 2, PK_FC1 = 3, PK_GATEUP = 4, PK_FC2 = 5, PK_HEAD = 6 };
 enum PkProf { PF_FLAG = 0, PF_PROLOGUE = 1, PF_TILES = 2, PF_BARRIER = 3, PF_ATTN = 4, PF_HEADFIN = 5, PF_PROD_WAIT = 6,
-              PF_PROD_TOTAL = 7, PK_PROF_N = 8 };
+              PF_PROD_TOTAL = 7, PF_TWAIT = 8, PF_TCOMP = 9, PF_TEPI = 10, PK_PROF_N = 12 };
 enum PkErr { PKE_FLAG = 1, PKE_BARRIER = 2, PKE_FULL = 3, PKE_EMPTY = 4 };
 
 struct PkPhase {
@@ -181,6 +184,17 @@ __device__ __forceinline__ float cblock_sum(float v, float *red) { // over the 2
     return t;
 }
 
+__device__ __forceinline__ void cblock_sum2(float &a, float &b, float *red /* [2 * PK_CWARPS] */) {
+    a = warp_sum(a);
+    b = warp_sum(b);
+    consumer_bar();
+    if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = a; red[PK_CWARPS + (threadIdx.x >> 5)] = b; }
+    consumer_bar();
+    a = b = 0.f;
+#pragma unroll
+    for (int w = 0; w < PK_CWARPS; ++w) { a += red[w]; b += red[PK_CWARPS + w]; }
+}
+
 template <typename WT, int NB>
 __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkParams P) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -192,12 +206,13 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
     float *att_o = xs + P.xs_floats;          // [256 * 8]
     float *att_m = att_o + 256 * 8;           // [128]
     float *att_l = att_m + 128;               // [128]
-    float *red = att_l + 128;                 // [8]
-    float *hbest_v = red + 8;                 // [8][PK_MAXNB]
+    float *red = att_l + 128;                 // [16]
+    float *hbest_v = red + 16;                // [8][PK_MAXNB]
     int *hbest_i = reinterpret_cast<int *>(hbest_v + PK_CWARPS * PK_MAXNB);
     int *s_dead = hbest_i + PK_CWARPS * PK_MAXNB;  // [2]
     volatile int *s_cons = s_dead + 2;        // [PK_MAX_SLOTS] tiles consumed so far from each ring slot
     uint64_t *bars = reinterpret_cast<uint64_t *>(s_dead + 2 + PK_MAX_SLOTS); // [2 * n_slots]; 8-byte aligned (xs_floats is even)
+    PkPhase *s_ph = reinterpret_cast<PkPhase *>(bars + 2 * PK_MAX_SLOTS);     // [PK_SMEM_PHASES]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int p = 0;
@@ -216,11 +231,16 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
         for (int s = 0; s < PK_MAX_SLOTS; ++s) s_cons[s] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    const bool ph_in_smem = T.n_phases <= PK_SMEM_PHASES;
+    if (ph_in_smem)
+        for (int i = tid; i < T.n_phases * (int)(sizeof(PkPhase) / 8); i += PK_THREADS)
+            reinterpret_cast<unsigned long long *>(s_ph)[i] = reinterpret_cast<const unsigned long long *>(P.phases + T.phase_begin)[i];
+    const PkPhase *phases = ph_in_smem ? s_ph : P.phases + T.phase_begin;
     __syncthreads();
     bool dead = false;
     const long total_slots = (long)P.n_pass * K;
     const bool prof_on = P.prof != nullptr && lane == 0 && (warp == 0 || warp == PK_CWARPS);
-    unsigned long long pf[PK_PROF_N] = {0, 0, 0, 0, 0, 0, 0, 0}, pf_t = prof_on ? pk_now() : 0;
+    unsigned long long pf[PK_PROF_N] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, pf_t = prof_on ? pk_now() : 0;
     auto lap = [&](int cat) { if (prof_on) { const unsigned long long n = pk_now(); pf[cat] += n - pf_t; pf_t = n; } };
 
     if (warp == PK_CWARPS) {
@@ -231,7 +251,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
         for (long v = 0; v < total_slots && !dead; ++v) {
             if ((int)(v % K) >= G) continue;
             for (int pi = 0; pi < T.n_phases && !dead; ++pi) {
-                const PkPhase ph = P.phases[T.phase_begin + pi];
+                const PkPhase ph = phases[pi];
                 if (ph.kind == PK_ATTN) continue;
                 const bool whole = ph.in_dim <= KC && ph.kind != PK_GATEUP && !(ph.kind == PK_QKV && P.rope);
                 const int b0 = (int)((long)cta * ph.n_blocks / T.n_cta), b1 = (int)((long)(cta + 1) * ph.n_blocks / T.n_cta);
@@ -326,7 +346,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
         float *x_out = T.is_last ? T.x_last : T.ring_out + (size_t)j * P.gmax * d;
 
         for (int pi = 0; pi < T.n_phases; ++pi) {
-            const PkPhase ph = P.phases[T.phase_begin + pi];
+            const PkPhase ph = phases[pi];
             const int Kd = ph.in_dim, Kpad = (Kd + 255) & ~255;
             if (ph.kind == PK_ATTN) {
                 // ---------------- attention over the cache: items (item, head, split) dealt to the team's blocks
@@ -402,44 +422,59 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
             for (int b = 0; b < NB; ++b) {
                 const bool live = b < nb;
                 const int slot = slots[b];
-                float s = 0.f;
-                for (int i = tid; i < Kd; i += PK_CTHREADS) {
-                    float xv = 0.f;
-                    if (live) {
-                        if (ph.kind == PK_QKV && ph.first_layer && T.is_first) {
-                            int tok = __ldcg(P.cur_tok + slot);
-                            tok = min(max(tok, 0), P.vocab - 1);
-                            xv = wt_to_f<WT>(reinterpret_cast<const WT *>(P.wte)[(size_t)tok * d + i]);
-                            if (P.wpe) xv += wt_to_f<WT>(reinterpret_cast<const WT *>(P.wpe)[(size_t)pos[b] * d + i]);
-                            if (cta == 0) T.x_embed[(size_t)b * d + i] = xv;
-                        } else if (ph.kind == PK_QKV) {
-                            xv = __ldcg((ph.first_layer ? x_in : x_out) + (size_t)b * d + i);
-                        } else if (ph.kind == PK_OUT) {
-                            // merge the attention splits of this element's head
-                            const int h = i / hd, e = i - h * hd;
-                            const float *pb = T.part + ((size_t)b * P.n_head + h) * T.n_split * (hd + 2);
-                            float M = -INFINITY, L = 0.f, O = 0.f;
+                // the loads of a batch of elements are all issued before any of them is used (one round trip to L2
+                // per batch instead of one per element)
+                int tok = 0;
+                const bool embed = ph.kind == PK_QKV && ph.first_layer && T.is_first;
+                if (embed && live) tok = min(max(__ldcg(P.cur_tok + slot), 0), P.vocab - 1);
+                auto fetch = [&](int i) -> float {
+                    if (embed) {
+                        float xv = wt_to_f<WT>(reinterpret_cast<const WT *>(P.wte)[(size_t)tok * d + i]);
+                        if (P.wpe) xv += wt_to_f<WT>(reinterpret_cast<const WT *>(P.wpe)[(size_t)pos[b] * d + i]);
+                        return xv;
+                    }
+                    if (ph.kind == PK_QKV) return __ldcg((ph.first_layer ? x_in : x_out) + (size_t)b * d + i);
+                    if (ph.kind == PK_OUT) {
+                        // merge the attention splits of this element's head
+                        const int h = i / hd, e = i - h * hd;
+                        const float *pb = T.part + ((size_t)b * P.n_head + h) * T.n_split * (hd + 2);
+                        float M = -INFINITY, L = 0.f, O = 0.f;
 #pragma unroll 4
-                            for (int s2 = 0; s2 < T.n_split; ++s2) {
-                                const float ms = __ldcg(pb + (size_t)s2 * (hd + 2)), ls = __ldcg(pb + (size_t)s2 * (hd + 2) + 1),
-                                            os = __ldcg(pb + (size_t)s2 * (hd + 2) + 2 + e);
-                                if (ms != -INFINITY) {
-                                    const float mn = fmaxf(M, ms), c0 = expf(M - mn), c1 = expf(ms - mn);
-                                    L = L * c0 + ls * c1;
-                                    O = O * c0 + os * c1;
-                                    M = mn;
-                                }
+                        for (int s2 = 0; s2 < T.n_split; ++s2) {
+                            const float ms = __ldcg(pb + (size_t)s2 * (hd + 2)), ls = __ldcg(pb + (size_t)s2 * (hd + 2) + 1),
+                                        os = __ldcg(pb + (size_t)s2 * (hd + 2) + 2 + e);
+                            if (ms != -INFINITY) {
+                                const float mn = fmaxf(M, ms), c0 = expf(M - mn), c1 = expf(ms - mn);
+                                L = L * c0 + ls * c1;
+                                O = O * c0 + os * c1;
+                                M = mn;
                             }
-                            xv = O / L;
-                        } else if (ph.kind == PK_FC2) {
-                            xv = __ldcg(T.hbuf + (size_t)b * Kd + i);
-                        } else { // FC1, GATEUP, HEAD: the block's current activation
-                            xv = __ldcg(x_out + (size_t)b * d + i);
+                        }
+                        return O / L;
+                    }
+                    if (ph.kind == PK_FC2) return __ldcg(T.hbuf + (size_t)b * Kd + i);
+                    return __ldcg(x_out + (size_t)b * d + i); // FC1, GATEUP, HEAD: the block's current activation
+                };
+                constexpr int SU = 8;
+                float s = 0.f;
+                for (int i0 = tid; i0 < Kd; i0 += PK_CTHREADS * SU) {
+                    float v[SU];
+#pragma unroll
+                    for (int u = 0; u < SU; ++u) {
+                        const int i = i0 + u * PK_CTHREADS;
+                        v[u] = (live && i < Kd) ? fetch(i) : 0.f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < SU; ++u) {
+                        const int i = i0 + u * PK_CTHREADS;
+                        if (i < Kd) {
+                            xs[b * Kpad + xs_perm<ES>(i)] = v[u];
+                            if (embed && live && cta == 0) T.x_embed[(size_t)b * d + i] = v[u];
+                            s += v[u];
                         }
                     }
-                    xs[b * Kpad + xs_perm<ES>(i)] = xv;
-                    s += xv;
                 }
+                (void)s;
                 if (ph.gamma) {
                     // gains and offsets do not depend on the activations: fetch them while the statistics reduce
                     constexpr int PRE = 8;
@@ -453,11 +488,16 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                             bp[u] = (i < Kd && ph.beta) ? ph.beta[i] : 0.f;
                         }
                     }
-                    float mean = 0.f;
-                    if (P.norm == NORM_LAYER) mean = cblock_sum(s, red) / (float)Kd;
-                    float ss = 0.f;
-                    for (int i = tid; i < Kd; i += PK_CTHREADS) { const float c = xs[b * Kpad + xs_perm<ES>(i)] - mean; ss += c * c; }
-                    const float rstd = rsqrtf(cblock_sum(ss, red) / (float)Kd + P.eps);
+                    // one reduction for both moments; the variance is taken about a pilot value (the item's first
+                    // element) so that it does not cancel when the mean is large
+                    consumer_bar(); // the pilot element was staged by another thread
+                    const float pilot = P.norm == NORM_LAYER ? xs[b * Kpad] : 0.f;
+                    float s1 = 0.f, s2 = 0.f;
+                    for (int i = tid; i < Kd; i += PK_CTHREADS) { const float c = xs[b * Kpad + xs_perm<ES>(i)] - pilot; s1 += c; s2 += c * c; }
+                    cblock_sum2(s1, s2, red);
+                    const float dm = P.norm == NORM_LAYER ? s1 / (float)Kd : 0.f;
+                    const float mean = pilot + dm;
+                    const float rstd = rsqrtf(fmaxf(s2 / (float)Kd - dm * dm, 0.f) + P.eps);
                     if (pre) {
 #pragma unroll
                         for (int u = 0; u < PRE; ++u) {
@@ -476,14 +516,18 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
             consumer_bar();
             lap(PF_PROLOGUE);
 
-            // ---------------- stream the weight tiles: consumer warp w owns row blocks b0+w, b0+w+8, ...
+            // ---------------- stream the weight tiles.  Two ways to split the work, chosen per phase:
+            //  ROWS = 2: all 8 consumer warps share every tile, warp w taking the partner segments w and w+8
+            //            (lowest latency when this block has only a few tiles in the phase);
+            //  ROWS = 16: a warp owns whole tiles (row blocks b0+w, b0+w+8, ...), so up to 8 tiles are in work
+            //            at once (the long output-layer phase).
+            // Either way the totals end up one row per even lane: lane 2i finishes the warp's i-th row.
             const int b0 = (int)((long)cta * ph.n_blocks / T.n_cta), b1 = (int)((long)(cta + 1) * ph.n_blocks / T.n_cta);
             const int n_chunks = (Kd + KC - 1) / KC;
             float best_v[NB];
             int best_i[NB];
 #pragma unroll
             for (int b = 0; b < NB; ++b) { best_v[b] = -INFINITY; best_i[b] = 0x7fffffff; }
-            const int seg = lane >> 1; // the row this lane finishes after the transpose-reduce
             size_t page_off[NB];
 #pragma unroll
             for (int b = 0; b < NB; ++b)
@@ -491,138 +535,162 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                                   ? (size_t)T.kv.page_table[((size_t)slots[b] * T.kv.n_layers_local + ph.layer_local) * T.kv.pages_per_seq + (pos[b] >> T.kv.page_shift)] * T.kv.page_elems
                                   : 0;
             const float *xres = (ph.kind == PK_OUT && ph.first_layer) ? x_in : x_out;
-            for (int blk = b0 + warp; blk < b1; blk += PK_CWARPS) {
-                // everything the epilogue needs besides the dot products is requested before waiting for the tile
-                // and not touched until the epilogue, so the loads stay in flight during the wait
-                bool sec;
-                const int row = pk_seg_row(ph, P.rope, hd, blk, seg, sec);
-                const bool rv = row < ph.n_rows;
-                float eb = 0.f, xr[NB], rc[NB], rs[NB];
+
+            auto run_tiles = [&](auto rows_c) {
+                constexpr int ROWS = decltype(rows_c)::value;
+                constexpr bool SHARED = ROWS == 2;            // tile shared by all warps
+                constexpr int KSB = SHARED ? 4 : 1;           // k-steps whose loads are issued together
+                constexpr int RB = (ROWS == 16 && NB > 2) ? 8 : ROWS; // rows whose loads are issued together
+                const int my_i = lane >> 1;                   // which of the warp's rows this lane finishes
+                const int seg = SHARED ? warp + 8 * (my_i & 1) : my_i;
+                const bool fin = (lane & 1) == 0 && my_i < ROWS;
+                for (int blk = SHARED ? b0 : b0 + warp; blk < b1; blk += SHARED ? 1 : PK_CWARPS) {
+                    // everything the epilogue needs besides the dot products is requested before waiting for the tile
+                    // and not touched until the epilogue, so the loads stay in flight during the wait
+                    bool sec;
+                    const int row = pk_seg_row(ph, P.rope, hd, blk, seg, sec);
+                    const bool rv = fin && row < ph.n_rows;
+                    float eb = 0.f, xr[NB], rc[NB], rs[NB];
 #pragma unroll
-                for (int b = 0; b < NB; ++b) { xr[b] = 0.f; rc[b] = 1.f; rs[b] = 0.f; }
-                if (rv) {
-                    if (ph.kind != PK_GATEUP && ph.bias) eb = ph.bias[row];
-#pragma unroll
-                    for (int b = 0; b < NB; ++b) {
-                        if (b < nb && (ph.kind == PK_OUT || ph.kind == PK_FC2)) xr[b] = __ldcg(xres + (size_t)b * d + row);
-                        if (b < nb && ph.kind == PK_QKV && P.rope && row < qw + kw) {
-                            const int i = (row % hd) & ((hd >> 1) - 1);
-                            rc[b] = P.rope_cos[(size_t)pos[b] * (hd >> 1) + i];
-                            rs[b] = P.rope_sin[(size_t)pos[b] * (hd >> 1) + i];
-                        }
-                    }
-                }
-                float acc[PK_SEGS][NB];
-#pragma unroll
-                for (int r2 = 0; r2 < PK_SEGS; ++r2)
-#pragma unroll
-                    for (int b = 0; b < NB; ++b) acc[r2][b] = 0.f;
-                const long seq0 = tile_seq + (long)(blk - b0) * n_chunks;
-                for (int c = 0; c < n_chunks; ++c) {
-                    const long seq = seq0 + c;
-                    const int slot = (int)(seq % NS), lap_no = (int)(seq / NS);
-                    const int kc0 = c * KC, kc_len = min(KC, Kd - kc0);
-                    // a parity test is only meaningful once every earlier tile of this slot has been consumed
-                    // (warps run ahead of one another); then wait for this tile's bytes to land
-                    pk_wait([&] { return s_cons[slot] >= lap_no; }, P.err, PKE_FULL, dead);
-                    wait_mbar(full_base + 8 * slot, (uint32_t)(lap_no & 1), P.err, PKE_FULL, dead);
-                    const unsigned char *tb = ring_mem + (size_t)slot * PK_SLOT_BYTES;
-                    for (int k = lane * VEC; k < kc_len; k += 32 * VEC) {
-                        float xv[NB][VEC];
+                    for (int b = 0; b < NB; ++b) { xr[b] = 0.f; rc[b] = 1.f; rs[b] = 0.f; }
+                    if (rv) {
+                        if (ph.kind != PK_GATEUP && ph.bias) eb = ph.bias[row];
 #pragma unroll
                         for (int b = 0; b < NB; ++b) {
-                            // 2-byte weights: column kc0+k starts this lane's 8-column run of its 256-column group
-                            const float *xrow = xs + b * Kpad + (ES == 2 ? ((kc0 + k) & ~255) + lane * 4 : kc0 + k);
-#pragma unroll
-                            for (int q = 0; q < VEC / 4; ++q) {
-                                const float4 x4 = *reinterpret_cast<const float4 *>(xrow + q * 128);
-                                xv[b][4 * q + 0] = x4.x; xv[b][4 * q + 1] = x4.y; xv[b][4 * q + 2] = x4.z; xv[b][4 * q + 3] = x4.w;
-                            }
-                        }
-                        // all loads of a batch of rows are issued before their (independent) FMA chains
-                        constexpr int RB = NB <= 2 ? 16 : 8;
-#pragma unroll
-                        for (int rb = 0; rb < PK_SEGS; rb += RB) {
-                            uint4 raw[RB];
-#pragma unroll
-                            for (int r2 = 0; r2 < RB; ++r2)
-                                raw[r2] = *reinterpret_cast<const uint4 *>(tb + ((size_t)(rb + r2) * kc_len + k) * ES);
-#pragma unroll
-                            for (int r2 = 0; r2 < RB; ++r2) {
-                                float f[VEC];
-                                pk_unpack<ES>(raw[r2], f);
-#pragma unroll
-                                for (int b = 0; b < NB; ++b)
-#pragma unroll
-                                    for (int e = 0; e < VEC; ++e) acc[rb + r2][b] = fmaf(f[e], xv[b][e], acc[rb + r2][b]);
+                            if (b < nb && (ph.kind == PK_OUT || ph.kind == PK_FC2)) xr[b] = __ldcg(xres + (size_t)b * d + row);
+                            if (b < nb && ph.kind == PK_QKV && P.rope && row < qw + kw) {
+                                const int i = (row % hd) & ((hd >> 1) - 1);
+                                rc[b] = P.rope_cos[(size_t)pos[b] * (hd >> 1) + i];
+                                rs[b] = P.rope_sin[(size_t)pos[b] * (hd >> 1) + i];
                             }
                         }
                     }
-                    __syncwarp();
-                    if (lane == 0) { s_cons[slot] = lap_no + 1; mbar_arrive(empty_base + 8 * slot); }
-                }
-                // transpose-reduce: 16 partial sums per lane -> the total of row (lane >> 1) in lanes 2i and 2i+1
-                float tot[NB];
+                    float acc[ROWS][NB][2];
 #pragma unroll
-                for (int b = 0; b < NB; ++b) {
-                    float v8[8], v4[4], v2[2];
+                    for (int r2 = 0; r2 < ROWS; ++r2)
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const bool up = lane & 16;
-                        const float send = up ? acc[i][b] : acc[i + 8][b], keep = up ? acc[i + 8][b] : acc[i][b];
-                        v8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+                        for (int b = 0; b < NB; ++b) acc[r2][b][0] = acc[r2][b][1] = 0.f;
+                    const long seq0 = tile_seq + (long)(blk - b0) * n_chunks;
+                    for (int c = 0; c < n_chunks; ++c) {
+                        const long seq = seq0 + c;
+                        const int slot = (int)(seq % NS), lap_no = (int)(seq / NS);
+                        const int kc0 = c * KC, kc_len = min(KC, Kd - kc0);
+                        // a parity test is only meaningful once every earlier tile of this slot has been consumed
+                        // (warps run ahead of one another); then wait for this tile's bytes to land
+                        lap(PF_TILES);
+                        pk_wait([&] { return s_cons[slot] >= lap_no; }, P.err, PKE_FULL, dead);
+                        wait_mbar(full_base + 8 * slot, (uint32_t)(lap_no & 1), P.err, PKE_FULL, dead);
+                        lap(PF_TWAIT);
+                        const unsigned char *tb = ring_mem + (size_t)slot * PK_SLOT_BYTES;
+                        for (int k0 = lane * VEC; k0 < kc_len; k0 += 32 * VEC * KSB) {
+#pragma unroll
+                            for (int rb = 0; rb < ROWS; rb += RB) {
+                                uint4 raw[KSB][RB];
+#pragma unroll
+                                for (int ks = 0; ks < KSB; ++ks)
+#pragma unroll
+                                    for (int r2 = 0; r2 < RB; ++r2) {
+                                        const int k = k0 + ks * 32 * VEC;
+                                        const int sg = SHARED ? warp + 8 * r2 : rb + r2;
+                                        raw[ks][r2] = k < kc_len ? *reinterpret_cast<const uint4 *>(tb + ((size_t)sg * kc_len + k) * ES)
+                                                                 : make_uint4(0u, 0u, 0u, 0u);
+                                    }
+#pragma unroll
+                                for (int ks = 0; ks < KSB; ++ks) {
+                                    const int k = min(k0 + ks * 32 * VEC, kc_len - VEC);
+                                    float xv[NB][VEC];
+#pragma unroll
+                                    for (int b = 0; b < NB; ++b) {
+                                        // 2-byte weights: column kc0+k starts this lane's 8-column run of its 256-column group
+                                        const float *xrow = xs + b * Kpad + (ES == 2 ? ((kc0 + k) & ~255) + lane * 4 : kc0 + k);
+#pragma unroll
+                                        for (int q = 0; q < VEC / 4; ++q) {
+                                            const float4 x4 = *reinterpret_cast<const float4 *>(xrow + q * 128);
+                                            xv[b][4 * q + 0] = x4.x; xv[b][4 * q + 1] = x4.y; xv[b][4 * q + 2] = x4.z; xv[b][4 * q + 3] = x4.w;
+                                        }
+                                    }
+#pragma unroll
+                                    for (int r2 = 0; r2 < RB; ++r2) {
+                                        float f[VEC];
+                                        pk_unpack<ES>(raw[ks][r2], f);
+#pragma unroll
+                                        for (int b = 0; b < NB; ++b)
+#pragma unroll
+                                            for (int e = 0; e < VEC; ++e) acc[rb + r2][b][e & 1] = fmaf(f[e], xv[b][e], acc[rb + r2][b][e & 1]);
+                                    }
+                                }
+                            }
+                        }
+                        if constexpr (SHARED) consumer_bar(); else __syncwarp();
+                        if (lane == 0 && (!SHARED || warp == 0)) { s_cons[slot] = lap_no + 1; mbar_arrive(empty_base + 8 * slot); }
+                        lap(PF_TCOMP);
                     }
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const bool up = lane & 8;
-                        const float send = up ? v8[i] : v8[i + 4], keep = up ? v8[i + 4] : v8[i];
-                        v4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-                    }
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        const bool up = lane & 4;
-                        const float send = up ? v4[i] : v4[i + 2], keep = up ? v4[i + 2] : v4[i];
-                        v2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-                    }
-                    {
-                        const bool up = lane & 2;
-                        const float send = up ? v2[0] : v2[1], keep = up ? v2[1] : v2[0];
-                        tot[b] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-                    }
-                    tot[b] += __shfl_xor_sync(0xffffffffu, tot[b], 1);
-                    tot[b] += eb + xr[b];
-                }
-                // partner segment (seg ^ 8): the other half of a rotary pair, or the "up" row of a gate row
-                float oth[NB];
-#pragma unroll
-                for (int b = 0; b < NB; ++b) oth[b] = __shfl_xor_sync(0xffffffffu, tot[b], 16);
-                if (rv && (lane & 1) == 0) {
+                    // reduce across lanes: lane 2i (and 2i+1) ends with the total of the warp's i-th row
+                    float tot[NB], oth[NB];
 #pragma unroll
                     for (int b = 0; b < NB; ++b) {
-                        if (b >= nb) break;
-                        float y = tot[b];
-                        if (ph.kind == PK_QKV) {
-                            if (P.rope && row < qw + kw) y = seg < 8 ? y * rc[b] - oth[b] * rs[b] : y * rc[b] + oth[b] * rs[b];
-                            if (row < qw) T.qbuf[(size_t)b * qw + row] = y;
-                            else {
-                                const int rk = row - qw, which = rk >= kw, rl = rk - which * kw;
-                                WT *dst = reinterpret_cast<WT *>(T.kv.pool) + page_off[b] +
-                                          ((size_t)(which * T.kv.n_kv_head + rl / hd) * T.kv.page_tokens + (pos[b] & (T.kv.page_tokens - 1))) * hd + rl % hd;
-                                kv_store<WT>(dst, y);
+                        if constexpr (SHARED) {
+                            float ta = acc[0][b][0] + acc[0][b][1], tb2 = acc[1][b][0] + acc[1][b][1];
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) { ta += __shfl_xor_sync(0xffffffffu, ta, o); tb2 += __shfl_xor_sync(0xffffffffu, tb2, o); }
+                            tot[b] = (my_i & 1) ? tb2 : ta;
+                        } else {
+                            float v8[8], v4[4], v2[2];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const bool up = lane & 16;
+                                const float lo8 = acc[i % ROWS][b][0] + acc[i % ROWS][b][1], hi8 = acc[(i + 8) % ROWS][b][0] + acc[(i + 8) % ROWS][b][1];
+                                v8[i] = (up ? hi8 : lo8) + __shfl_xor_sync(0xffffffffu, up ? lo8 : hi8, 16);
                             }
-                        } else if (ph.kind == PK_FC1) {
-                            T.hbuf[(size_t)b * ph.n_rows + row] = P.act == 0 ? gelu_tanh_f(y) : gelu_erf_f(y);
-                        } else if (ph.kind == PK_GATEUP) {
-                            if (seg < 8) T.hbuf[(size_t)b * ph.n_rows + row] = silu_f(y) * oth[b];
-                        } else if (ph.kind == PK_OUT || ph.kind == PK_FC2) {
-                            x_out[(size_t)b * d + row] = y;
-                        } else { // PK_HEAD
-                            P.logits[(size_t)slots[b] * ph.n_rows + row] = y;
-                            if (y > best_v[b] || (y == best_v[b] && row < best_i[b])) { best_v[b] = y; best_i[b] = row; }
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const bool up = lane & 8;
+                                v4[i] = (up ? v8[i + 4] : v8[i]) + __shfl_xor_sync(0xffffffffu, up ? v8[i] : v8[i + 4], 8);
+                            }
+#pragma unroll
+                            for (int i = 0; i < 2; ++i) {
+                                const bool up = lane & 4;
+                                v2[i] = (up ? v4[i + 2] : v4[i]) + __shfl_xor_sync(0xffffffffu, up ? v4[i] : v4[i + 2], 4);
+                            }
+                            const bool up = lane & 2;
+                            tot[b] = (up ? v2[1] : v2[0]) + __shfl_xor_sync(0xffffffffu, up ? v2[0] : v2[1], 2);
+                            tot[b] += __shfl_xor_sync(0xffffffffu, tot[b], 1);
+                        }
+                        tot[b] += eb + xr[b];
+                        // partner row (segment ^ 8): the other half of a rotary pair, or the "up" row of a gate row
+                        oth[b] = __shfl_xor_sync(0xffffffffu, tot[b], SHARED ? 2 : 16);
+                    }
+                    if (rv) {
+#pragma unroll
+                        for (int b = 0; b < NB; ++b) {
+                            if (b >= nb) break;
+                            float y = tot[b];
+                            if (ph.kind == PK_QKV) {
+                                if (P.rope && row < qw + kw) y = seg < 8 ? y * rc[b] - oth[b] * rs[b] : y * rc[b] + oth[b] * rs[b];
+                                if (row < qw) T.qbuf[(size_t)b * qw + row] = y;
+                                else {
+                                    const int rk = row - qw, which = rk >= kw, rl = rk - which * kw;
+                                    WT *dst = reinterpret_cast<WT *>(T.kv.pool) + page_off[b] +
+                                              ((size_t)(which * T.kv.n_kv_head + rl / hd) * T.kv.page_tokens + (pos[b] & (T.kv.page_tokens - 1))) * hd + rl % hd;
+                                    kv_store<WT>(dst, y);
+                                }
+                            } else if (ph.kind == PK_FC1) {
+                                T.hbuf[(size_t)b * ph.n_rows + row] = P.act == 0 ? gelu_tanh_f(y) : gelu_erf_f(y);
+                            } else if (ph.kind == PK_GATEUP) {
+                                if (seg < 8) T.hbuf[(size_t)b * ph.n_rows + row] = silu_f(y) * oth[b];
+                            } else if (ph.kind == PK_OUT || ph.kind == PK_FC2) {
+                                x_out[(size_t)b * d + row] = y;
+                            } else { // PK_HEAD
+                                P.logits[(size_t)slots[b] * ph.n_rows + row] = y;
+                                if (y > best_v[b] || (y == best_v[b] && row < best_i[b])) { best_v[b] = y; best_i[b] = row; }
+                            }
                         }
                     }
+                    lap(PF_TEPI);
                 }
-            }
+            };
+            if (b1 - b0 >= 6) run_tiles(std::integral_constant<int, 16>{});
+            else run_tiles(std::integral_constant<int, 2>{});
             tile_seq += (long)(b1 - b0) * n_chunks;
             lap(PF_TILES);
 
@@ -696,7 +764,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
     if (cta == 0)
         for (int s = tid; s < P.n_samples; s += PK_CTHREADS) T.pos[s] += P.n_pass;
     if (prof_on)
-        for (int i = 0; i < PF_PROD_WAIT; ++i) P.prof[(size_t)blockIdx.x * PK_PROF_N + i] = pf[i];
+        for (int i = 0; i < PK_PROF_N; ++i)
+            if (i != PF_PROD_WAIT && i != PF_PROD_TOTAL) P.prof[(size_t)blockIdx.x * PK_PROF_N + i] = pf[i];
 }
 
 } // namespace mdi

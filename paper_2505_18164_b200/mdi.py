@@ -179,9 +179,9 @@ class Context:
         return st
 
     def partition_times(self, partition: int):
-        """(blocks in the partition's team, [8] mean milliseconds per category) of the last generate."""
-        out = (ctypes.c_double * 8)()
-        rc = lib().mdi_get_partition_times(self._h, partition, out, 8)
+        """(blocks in the partition's team, [12] mean milliseconds per category) of the last generate."""
+        out = (ctypes.c_double * 12)()
+        rc = lib().mdi_get_partition_times(self._h, partition, out, 12)
         if rc < 0:
             self._check(rc)
         return rc, list(out)
