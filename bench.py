@@ -121,7 +121,7 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def cpu_baseline(w: I.Workload, weights, n_new_sample: int = 24):
+def cpu_baseline(w: I.Workload, weights, n_new_sample: int = 256):
     """The CPU checker, as it stands, on a bounded sample of the workload: all samples, full prompts,
     the first n_new_sample of the new tokens, scheduled by its own recurrent-pipeline simulation."""
     from oracle import mdi_oracle as O

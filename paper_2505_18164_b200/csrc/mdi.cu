@@ -471,7 +471,7 @@ int pk_setup(mdi_ctx *c) {
         T.first_cta = first; T.n_cta = n_cta[p]; first += n_cta[p];
         T.phase_begin = c->pk_phase_begin[p]; T.n_phases = c->pk_phase_count[p];
         T.is_first = p == 0; T.is_last = p == K - 1;
-        T.n_split = std::max(1, std::min(16, n_cta[p] / (c->pk_nb * s.n_head)));
+        T.n_split = std::max(1, std::min(4, n_cta[p] / (c->pk_nb * s.n_head)));
         T.kv = kv_view(c, P);
         T.qbuf = P.qbuf; T.part = P.part; T.hbuf = P.hbuf; T.x_embed = P.x_embed; T.x_last = P.x_last;
         T.ring_in = p > 0 ? c->part[p - 1].ring : nullptr;

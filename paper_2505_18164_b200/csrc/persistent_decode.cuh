@@ -113,28 +113,63 @@ __device__ __forceinline__ unsigned long long pk_now() {
     return t;
 }
 
-// Bounded wait: gives up after PK_WAIT_NS of wall time, records why in *err and marks the thread `dead`;
-// `dead` is sticky, so after a failure (its own or one it sees in *err) a thread never waits again.
-template <typename Probe> __device__ __forceinline__ void pk_wait(Probe ready, int *err, int code, bool &dead) {
-    if (dead) return;
+// Bounded waits: the first probe is inline; the polling loop lives out of line (one copy, keeps the kernel's
+// instruction footprint small).  A wait gives up after PK_WAIT_NS of wall time, records why in *err and marks
+// the thread `dead`; `dead` is sticky, so after a failure (its own or one it sees in *err) a thread never waits again.
+enum PkWaitKind { PKW_GLOBAL_GE = 0, PKW_MBAR = 1, PKW_SMEM_GE = 2 };
+__device__ __forceinline__ bool pk_probe(int kind, const void *p, uint32_t a) {
+    if (kind == PKW_GLOBAL_GE) return ld_acquire(reinterpret_cast<const unsigned *>(p)) >= a;
+    if (kind == PKW_MBAR) return mbar_try_wait((uint32_t)(uintptr_t)p, a);
+    return *reinterpret_cast<const volatile int *>(p) >= (int)a;
+}
+__device__ __noinline__ bool pk_wait_slow(int kind, const void *p, uint32_t a, int *err, int code) {
     unsigned long long t0 = 0;
     for (unsigned it = 0;; ++it) {
-        if (ready()) return;
+        if (pk_probe(kind, p, a)) return false;
         if ((it & 63u) == 63u) {
-            if (*(volatile int *)err) { dead = true; return; }
+            if (*(volatile int *)err) return true;
             const unsigned long long now = pk_now();
             if (t0 == 0) t0 = now;
             else if (now - t0 > PK_WAIT_NS) break;
         }
     }
     atomicCAS(err, 0, code);
-    dead = true;
+    return true;
 }
 __device__ __forceinline__ void wait_ge(const unsigned *p, unsigned target, int *err, int code, bool &dead) {
-    pk_wait([&] { return ld_acquire(p) >= target; }, err, code, dead);
+    if (dead || pk_probe(PKW_GLOBAL_GE, p, target)) return;
+    dead = pk_wait_slow(PKW_GLOBAL_GE, p, target, err, code);
 }
 __device__ __forceinline__ void wait_mbar(uint32_t bar, uint32_t parity, int *err, int code, bool &dead) {
-    pk_wait([&] { return mbar_try_wait(bar, parity); }, err, code, dead);
+    if (dead || pk_probe(PKW_MBAR, (const void *)(uintptr_t)bar, parity)) return;
+    dead = pk_wait_slow(PKW_MBAR, (const void *)(uintptr_t)bar, parity, err, code);
+}
+__device__ __forceinline__ void wait_smem_ge(const volatile int *p, int target, int *err, int code, bool &dead) {
+    if (dead || *p >= target) return;
+    dead = pk_wait_slow(PKW_SMEM_GE, (const void *)p, (uint32_t)target, err, code);
+}
+__device__ __noinline__ void pk_lap(unsigned long long *pf, unsigned long long *t, int cat) {
+    const unsigned long long n = pk_now();
+    pf[cat] += n - *t;
+    *t = n;
+}
+__device__ __noinline__ float pk_act(float y, int act) { return act == 0 ? gelu_tanh_f(y) : gelu_erf_f(y); }
+__device__ __noinline__ float pk_silu(float y) { return silu_f(y); }
+// Merge of the attention splits for element e of one (item, head): partials are (max, sum, o[head_dim]) per split.
+__device__ __noinline__ float pk_merge_splits(const float *pb, int n_split, int hd, int e) {
+    float M = -INFINITY, L = 0.f, O = 0.f;
+#pragma unroll 4
+    for (int s2 = 0; s2 < n_split; ++s2) {
+        const float ms = __ldcg(pb + (size_t)s2 * (hd + 2)), ls = __ldcg(pb + (size_t)s2 * (hd + 2) + 1),
+                    os = __ldcg(pb + (size_t)s2 * (hd + 2) + 2 + e);
+        if (ms != -INFINITY) {
+            const float mn = fmaxf(M, ms), c0 = expf(M - mn), c1 = expf(ms - mn);
+            L = L * c0 + ls * c1;
+            O = O * c0 + os * c1;
+            M = mn;
+        }
+    }
+    return O / L;
 }
 
 // Which matrix row sits in segment i of row block blk.  Segments i and i+8 are partners: the two halves
@@ -241,7 +276,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
     const long total_slots = (long)P.n_pass * K;
     const bool prof_on = P.prof != nullptr && lane == 0 && (warp == 0 || warp == PK_CWARPS);
     unsigned long long pf[PK_PROF_N] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, pf_t = prof_on ? pk_now() : 0;
-    auto lap = [&](int cat) { if (prof_on) { const unsigned long long n = pk_now(); pf[cat] += n - pf_t; pf_t = n; } };
+    auto lap = [&](int cat) { if (prof_on) pk_lap(pf, &pf_t, cat); };
 
     if (warp == PK_CWARPS) {
         // =========================== producer ===========================
@@ -422,55 +457,42 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
             for (int b = 0; b < NB; ++b) {
                 const bool live = b < nb;
                 const int slot = slots[b];
-                // the loads of a batch of elements are all issued before any of them is used (one round trip to L2
-                // per batch instead of one per element)
-                int tok = 0;
-                const bool embed = ph.kind == PK_QKV && ph.first_layer && T.is_first;
-                if (embed && live) tok = min(max(__ldcg(P.cur_tok + slot), 0), P.vocab - 1);
-                auto fetch = [&](int i) -> float {
-                    if (embed) {
-                        float xv = wt_to_f<WT>(reinterpret_cast<const WT *>(P.wte)[(size_t)tok * d + i]);
-                        if (P.wpe) xv += wt_to_f<WT>(reinterpret_cast<const WT *>(P.wpe)[(size_t)pos[b] * d + i]);
-                        return xv;
-                    }
-                    if (ph.kind == PK_QKV) return __ldcg((ph.first_layer ? x_in : x_out) + (size_t)b * d + i);
-                    if (ph.kind == PK_OUT) {
-                        // merge the attention splits of this element's head
-                        const int h = i / hd, e = i - h * hd;
-                        const float *pb = T.part + ((size_t)b * P.n_head + h) * T.n_split * (hd + 2);
-                        float M = -INFINITY, L = 0.f, O = 0.f;
-#pragma unroll 4
-                        for (int s2 = 0; s2 < T.n_split; ++s2) {
-                            const float ms = __ldcg(pb + (size_t)s2 * (hd + 2)), ls = __ldcg(pb + (size_t)s2 * (hd + 2) + 1),
-                                        os = __ldcg(pb + (size_t)s2 * (hd + 2) + 2 + e);
-                            if (ms != -INFINITY) {
-                                const float mn = fmaxf(M, ms), c0 = expf(M - mn), c1 = expf(ms - mn);
-                                L = L * c0 + ls * c1;
-                                O = O * c0 + os * c1;
-                                M = mn;
-                            }
-                        }
-                        return O / L;
-                    }
-                    if (ph.kind == PK_FC2) return __ldcg(T.hbuf + (size_t)b * Kd + i);
-                    return __ldcg(x_out + (size_t)b * d + i); // FC1, GATEUP, HEAD: the block's current activation
-                };
-                constexpr int SU = 8;
+                // Source of the staged row: a plain fp32 vector for most phases (loads issued in batches of 8 per
+                // thread so that a batch costs one round trip to L2); the embedding and the split merge have
+                // their own short loops.
                 float s = 0.f;
-                for (int i0 = tid; i0 < Kd; i0 += PK_CTHREADS * SU) {
-                    float v[SU];
-#pragma unroll
-                    for (int u = 0; u < SU; ++u) {
-                        const int i = i0 + u * PK_CTHREADS;
-                        v[u] = (live && i < Kd) ? fetch(i) : 0.f;
+                if (ph.kind == PK_QKV && ph.first_layer && T.is_first) {
+                    const int tok = live ? min(max(__ldcg(P.cur_tok + slot), 0), P.vocab - 1) : 0;
+                    const WT *te = reinterpret_cast<const WT *>(P.wte) + (size_t)tok * d;
+                    const WT *pe = P.wpe ? reinterpret_cast<const WT *>(P.wpe) + (size_t)pos[b] * d : nullptr;
+                    for (int i = tid; i < Kd; i += PK_CTHREADS) {
+                        float xv = 0.f;
+                        if (live) { xv = wt_to_f<WT>(te[i]); if (pe) xv += wt_to_f<WT>(pe[i]); }
+                        xs[b * Kpad + xs_perm<ES>(i)] = xv;
+                        if (live && cta == 0) T.x_embed[(size_t)b * d + i] = xv;
                     }
+                } else if (ph.kind == PK_OUT) {
+                    for (int i = tid; i < Kd; i += PK_CTHREADS) {
+                        const int h = i / hd;
+                        xs[b * Kpad + xs_perm<ES>(i)] =
+                            live ? pk_merge_splits(T.part + ((size_t)b * P.n_head + h) * T.n_split * (hd + 2), T.n_split, hd, i - h * hd) : 0.f;
+                    }
+                } else {
+                    const float *src = ph.kind == PK_QKV ? (ph.first_layer ? x_in : x_out) + (size_t)b * d
+                                       : ph.kind == PK_FC2 ? T.hbuf + (size_t)b * Kd
+                                                           : x_out + (size_t)b * d;
+                    constexpr int SU = 8;
+                    for (int i0 = tid; i0 < Kd; i0 += PK_CTHREADS * SU) {
+                        float v[SU];
 #pragma unroll
-                    for (int u = 0; u < SU; ++u) {
-                        const int i = i0 + u * PK_CTHREADS;
-                        if (i < Kd) {
-                            xs[b * Kpad + xs_perm<ES>(i)] = v[u];
-                            if (embed && live && cta == 0) T.x_embed[(size_t)b * d + i] = v[u];
-                            s += v[u];
+                        for (int u = 0; u < SU; ++u) {
+                            const int i = i0 + u * PK_CTHREADS;
+                            v[u] = (live && i < Kd) ? __ldcg(src + i) : 0.f;
+                        }
+#pragma unroll
+                        for (int u = 0; u < SU; ++u) {
+                            const int i = i0 + u * PK_CTHREADS;
+                            if (i < Kd) xs[b * Kpad + xs_perm<ES>(i)] = v[u];
                         }
                     }
                 }
@@ -578,7 +600,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                         // a parity test is only meaningful once every earlier tile of this slot has been consumed
                         // (warps run ahead of one another); then wait for this tile's bytes to land
                         lap(PF_TILES);
-                        pk_wait([&] { return s_cons[slot] >= lap_no; }, P.err, PKE_FULL, dead);
+                        wait_smem_ge(s_cons + slot, lap_no, P.err, PKE_FULL, dead);
                         wait_mbar(full_base + 8 * slot, (uint32_t)(lap_no & 1), P.err, PKE_FULL, dead);
                         lap(PF_TWAIT);
                         const unsigned char *tb = ring_mem + (size_t)slot * PK_SLOT_BYTES;
@@ -675,9 +697,9 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                                     kv_store<WT>(dst, y);
                                 }
                             } else if (ph.kind == PK_FC1) {
-                                T.hbuf[(size_t)b * ph.n_rows + row] = P.act == 0 ? gelu_tanh_f(y) : gelu_erf_f(y);
+                                T.hbuf[(size_t)b * ph.n_rows + row] = pk_act(y, P.act);
                             } else if (ph.kind == PK_GATEUP) {
-                                if (seg < 8) T.hbuf[(size_t)b * ph.n_rows + row] = silu_f(y) * oth[b];
+                                if (seg < 8) T.hbuf[(size_t)b * ph.n_rows + row] = pk_silu(y) * oth[b];
                             } else if (ph.kind == PK_OUT || ph.kind == PK_FC2) {
                                 x_out[(size_t)b * d + row] = y;
                             } else { // PK_HEAD
