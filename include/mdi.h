@@ -170,7 +170,29 @@ int64_t mdi_memory_bytes(mdi_ctx *ctx, int partition);
 int mdi_get_partition_times(mdi_ctx *ctx, int partition, double *out_ms, int n);
 /* Wait for everything enqueued on the context's streams. */
 int mdi_sync(mdi_ctx *ctx);
-/* Text of the last error of this context (or of the last failed mdi_create if ctx is NULL). */
+/* Greedy token choice for callers that must not allocate.  (The paper has no counterpart: this is a
+ * convenience of this library, not part of the method.)
+ * Some users of the library cannot call cudaMalloc where they pick tokens: a serving loop that has
+ * given the whole device to its own memory pool, a latency-critical section that cannot afford the
+ * device synchronisation an allocation or a free may bring, or code that runs where another component
+ * owns the allocator.  They already hold the logits; this call returns, per row, the index of the largest
+ * value (the lowest index on ties, like the output layer of mdi_generate) and allocates nothing: its
+ * working memory is a fixed array inside the library (about 128 KB on every GPU that loads the library,
+ * held until the process exits).
+ *   logits_dev: [n_rows][n_cols] fp32, row-major, device memory of the current device (read only);
+ *   out_dev:    [n_rows] int32, device memory; stream: a cudaStream_t (NULL = default stream).
+ * Limits: n_rows <= 64 and n_cols <= 262144; larger sizes return MDI_ERR_SHAPE and touch nothing.
+ * The work is enqueued on `stream`; the result is there once the stream has reached it.
+ * The first call on each device looks up the array's device address (one extra runtime query): make
+ * that first call outside any stream capture.  All calls on a device share the one array, which keeps
+ * what the previous call left in it (the call clears the counters it needs): two calls that overlap on
+ * the GPU - different streams without an ordering between them - race on it and give wrong tokens, so
+ * order them (same stream, or events).  Errors: ARG (null pointer, non-positive size), SHAPE, CUDA; the
+ * text is available from mdi_last_error(NULL). */
+int mdi_greedy_argmax_static(const float *logits_dev, int n_rows, int n_cols, int32_t *out_dev, void *stream);
+
+/* Text of the last error of this context; with ctx NULL, of the last failed call that takes no context
+ * (mdi_create, mdi_greedy_argmax_static). */
 const char *mdi_last_error(mdi_ctx *ctx);
 
 #ifdef __cplusplus

@@ -548,6 +548,9 @@ int pk_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
 
 } // namespace
 
+// Used by entry points that take no context (other files of the library): text for mdi_last_error(NULL).
+void mdi_internal_set_error(const char *text) { g_create_error = text ? text : ""; }
+
 // ====================================================================================================
 extern "C" {
 

@@ -22,7 +22,7 @@ _ERR_NAMES = {ERR_ARG: "MDI_ERR_ARG", ERR_SHAPE: "MDI_ERR_SHAPE", ERR_OOM: "MDI_
 
 EXPORTS = ["mdi_create", "mdi_destroy", "mdi_load_weights", "mdi_prefill", "mdi_prefill_dev", "mdi_step",
            "mdi_generate", "mdi_generate_dev", "mdi_get_logits", "mdi_set_teacher_tokens", "mdi_reset_sample",
-           "mdi_get_stats", "mdi_get_partition_times", "mdi_memory_bytes", "mdi_sync", "mdi_last_error"]
+           "mdi_get_stats", "mdi_get_partition_times", "mdi_memory_bytes", "mdi_sync", "mdi_last_error", "mdi_greedy_argmax_static"]
 
 
 class MdiError(RuntimeError):
@@ -81,6 +81,7 @@ def lib():
         L.mdi_memory_bytes.argtypes = [vp, ci]
         L.mdi_memory_bytes.restype = ctypes.c_int64
         L.mdi_sync.argtypes = [vp]
+        L.mdi_greedy_argmax_static.argtypes = [vp, ci, ci, vp, vp]
         L.mdi_last_error.argtypes = [vp]
         L.mdi_last_error.restype = ctypes.c_char_p
         _lib = L
@@ -96,6 +97,14 @@ def _ptr(x) -> int:
     if isinstance(x, np.ndarray):
         return x.ctypes.data
     return x.data_ptr()
+
+
+def greedy_argmax_static(logits_dev, n_rows: int, n_cols: int, out_dev, stream: int = 0):
+    """mdi_greedy_argmax_static: per-row argmax of device logits without any allocation (see mdi.h).
+    ``logits_dev`` / ``out_dev``: device tensors or raw addresses; ``stream``: a cudaStream_t value."""
+    rc = lib().mdi_greedy_argmax_static(_ptr(logits_dev), n_rows, n_cols, _ptr(out_dev), stream)
+    if rc != MDI_OK:
+        raise MdiError(rc, (lib().mdi_last_error(None) or b"").decode())
 
 
 class Context:
