@@ -63,11 +63,12 @@ def decode_bytes(w: I.Workload, n_samples: int) -> dict:
     G = min(n_samples, w.n_partitions)
     per_pass_w = G * (block + head) * bpe
     kvw = s.n_kv_head * s.head_dim
+    kv_bpe = 4                                       # the cache holds fp32 (library default)
     n_pass = w.n_new - 1
     kv = 0
     for i in range(n_pass):
         t = w.n_prompt + i                       # rows cached before this pass
-        kv += n_samples * s.n_layer * (2 * (t + 1) * kvw + 2 * kvw) * bpe
+        kv += n_samples * s.n_layer * (2 * (t + 1) * kvw + 2 * kvw) * kv_bpe
     return {"weights": per_pass_w * n_pass, "kv": kv, "total": per_pass_w * n_pass + kv, "passes": n_pass,
             "per_pass_weights": per_pass_w}
 

@@ -53,8 +53,8 @@ typedef struct {
     int arch;         /* MDI_ARCH_GPT: LayerNorm, learned positions, biases, GELU MLP;
                          MDI_ARCH_LLAMA: RMSNorm, rotary positions (split-halves pairing), SwiGLU, no biases */
     int n_layer, d_model, n_head, head_dim, n_kv_head, d_ff, vocab, n_ctx;
-    int weight_dtype; /* MDI_DTYPE_*: element type of every tensor given to mdi_load_weights; the
-                         key/value cache uses the same type; activations and accumulation are fp32 */
+    int weight_dtype; /* MDI_DTYPE_*: element type of every tensor given to mdi_load_weights; activations,
+                         accumulation and (by default) the key/value cache are fp32 */
     int tied_lm_head; /* 1: the output projection reuses "wte" */
     int has_bias;     /* 1: linear layers carry biases (GPT) */
     int act;          /* MDI_ACT_* */
@@ -69,6 +69,9 @@ typedef struct {
     int attn_splits;   /* sequence splits of decode attention (default: chosen from n_ctx) */
     int rounds_per_graph; /* stream scheduler: rounds of the recurrent schedule captured per CUDA graph
                              (default 16; <0: no graphs) */
+    int kv_cache_bf16; /* 0 (default): the key/value cache holds fp32; 1: with bf16 weights, hold bf16 instead - half the
+                          cache bytes, at about 2e-3 relative error per block on the activations (measured), which on a
+                          32-block model exceeds a 3e-2 absolute logit tolerance */
     int scheduler;     /* how mdi_generate runs the recurrent pipeline.  0: the persistent kernel (one launch,
                           one team of thread blocks per partition, flag handoff between teams) when the shape
                           fits it (groups of at most 4 samples), else the stream scheduler; 1: always the

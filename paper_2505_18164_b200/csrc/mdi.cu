@@ -75,7 +75,8 @@ struct mdi_ctx {
     mdi_options o{};
     int K = 0, S = 0, dev = 0;
     int page_tokens = 16, page_shift = 4, pages_per_seq = 0, n_split = 1, gmax = 1, rounds_per_graph = 16;
-    size_t page_elems = 0, esize = 2;
+    size_t page_elems = 0, esize = 2, kv_esize = 4;
+    bool kv_f32 = true;
     std::vector<Partition> part;
     std::vector<LayerW> layer;
     void *wte = nullptr, *wpe = nullptr, *lm_head = nullptr;
@@ -151,11 +152,17 @@ inline void count_launch(mdi_ctx *c) {
 // ---- kernel dispatch ------------------------------------------------------------------------------
 constexpr size_t LIN_SMEM_MAX = 200 * 1024;
 
+// The key/value cache is fp32 unless the context asked for a cache in the (2-byte) weight type.
+bool g_kv_f32_dispatch = true;
 template <int NB, typename WT, int MODE> void lin_launch(const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st) {
-    k_linear<NB, WT, MODE><<<grid, LIN_THREADS, smem, st>>>(a, bt);
+    if (MODE == LIN_QKV && g_kv_f32_dispatch) k_linear<NB, WT, MODE, float><<<grid, LIN_THREADS, smem, st>>>(a, bt);
+    else k_linear<NB, WT, MODE><<<grid, LIN_THREADS, smem, st>>>(a, bt);
 }
 template <int NB, typename WT, int MODE> cudaError_t lin_attr() {
-    return cudaFuncSetAttribute(k_linear<NB, WT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LIN_SMEM_MAX);
+    cudaError_t e = cudaFuncSetAttribute(k_linear<NB, WT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LIN_SMEM_MAX);
+    if (e == cudaSuccess && MODE == LIN_QKV)
+        e = cudaFuncSetAttribute(k_linear<NB, WT, MODE, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LIN_SMEM_MAX);
+    return e;
 }
 template <typename WT, int MODE> void lin_nb(int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st) {
     switch (nb) {
@@ -219,6 +226,7 @@ int linear(mdi_ctx *c, int mode, LinArgs a, const Batch &bt, cudaStream_t st) {
         if (a.x_res) b.x_res = a.x_res + (size_t)first * a.n_rows;
         if (a.x_out) b.x_out = a.x_out + (size_t)first * a.n_rows;
         const size_t smem = (size_t)nb * a.in_dim * 4;
+        g_kv_f32_dispatch = c->kv_f32;
         if (f32) lin_mode<float>(mode, nb, b, sb, grid, smem, st);
         else lin_mode<__nv_bfloat16>(mode, nb, b, sb, grid, smem, st);
         count_launch(c);
@@ -291,7 +299,7 @@ int enqueue_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in
             a.layer_local = l - P.lo; a.n_head = s.n_head; a.n_split = c->n_split; a.pos = P.pos_dev;
             a.scale = 1.0f / std::sqrt((float)s.head_dim);
             dim3 g(s.n_head, c->n_split, bt.n);
-            if (f32) attn_hd<float>(s.head_dim, a, bt, g, st); else attn_hd<__nv_bfloat16>(s.head_dim, a, bt, g, st);
+            if (c->kv_f32) attn_hd<float>(s.head_dim, a, bt, g, st); else attn_hd<__nv_bfloat16>(s.head_dim, a, bt, g, st);
             count_launch(c);
         }
         {   // output projection + residual
@@ -369,15 +377,19 @@ int ensure_pages(mdi_ctx *c, int p, int slot, int rows) {
 
 
 // ---- persistent decode kernel: tables and launch -----------------------------------------------------
-template <typename WT> cudaError_t pk_attr(size_t smem) {
+template <typename WT, typename KT> cudaError_t pk_attr(size_t smem) {
     cudaError_t e;
-    if ((e = cudaFuncSetAttribute(k_persistent_decode<WT, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(k_persistent_decode<WT, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    return cudaFuncSetAttribute(k_persistent_decode<WT, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if ((e = cudaFuncSetAttribute(k_persistent_decode<WT, 1, KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(k_persistent_decode<WT, 2, KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    return cudaFuncSetAttribute(k_persistent_decode<WT, 4, KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
-template <typename WT> const void *pk_func(int nb) {
-    return nb == 1 ? (const void *)k_persistent_decode<WT, 1> : nb == 2 ? (const void *)k_persistent_decode<WT, 2>
-                                                                        : (const void *)k_persistent_decode<WT, 4>;
+template <typename WT, typename KT> const void *pk_func(int nb) {
+    return nb == 1 ? (const void *)k_persistent_decode<WT, 1, KT> : nb == 2 ? (const void *)k_persistent_decode<WT, 2, KT>
+                                                                            : (const void *)k_persistent_decode<WT, 4, KT>;
+}
+const void *pk_func_for(const mdi_ctx *c, int nb) {
+    if (c->s.weight_dtype == MDI_DTYPE_F32) return pk_func<float, float>(nb);
+    return c->kv_f32 ? pk_func<__nv_bfloat16, float>(nb) : pk_func<__nv_bfloat16, __nv_bfloat16>(nb);
 }
 
 // Phase list of every partition, team sizes (blocks per partition, in proportion to the bytes a step
@@ -403,7 +415,13 @@ int pk_setup(mdi_ctx *c) {
     if (fixed + 2 * PK_SLOT_BYTES > budget) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: inputs do not fit in shared memory") : MDI_OK;
     c->pk_slots = (int)std::min<size_t>(PK_MAX_SLOTS, (budget - fixed) / PK_SLOT_BYTES);
     c->pk_smem = fixed + (size_t)c->pk_slots * PK_SLOT_BYTES;
-    CU(s.weight_dtype == MDI_DTYPE_F32 ? pk_attr<float>(c->pk_smem) : pk_attr<__nv_bfloat16>(c->pk_smem));
+    {
+        cudaError_t ea;
+        if (s.weight_dtype == MDI_DTYPE_F32) ea = pk_attr<float, float>(c->pk_smem);
+        else if (c->kv_f32) ea = pk_attr<__nv_bfloat16, float>(c->pk_smem);
+        else ea = pk_attr<__nv_bfloat16, __nv_bfloat16>(c->pk_smem);
+        CU(ea);
+    }
 
     std::vector<PkPhase> &ph = c->pk_phases_host;
     ph.clear();
@@ -538,7 +556,7 @@ int pk_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     for (auto &T : c->pk_teams_host) grid += T.n_cta;
     const int nb = (n_samples + G - 1) / G;
     const int tnb = nb <= 1 ? 1 : nb <= 2 ? 2 : 4;
-    const void *fn = s.weight_dtype == MDI_DTYPE_F32 ? pk_func<float>(tnb) : pk_func<__nv_bfloat16>(tnb);
+    const void *fn = pk_func_for(c, tnb);
     void *args[] = {&P};
     CU(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(PK_THREADS), args, c->pk_smem, c->main));
     ++c->st.kernel_launches;
@@ -629,6 +647,8 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     while ((1 << c->page_shift) < c->page_tokens) ++c->page_shift;
     c->pages_per_seq = (s.n_ctx + c->page_tokens - 1) / c->page_tokens;
     c->esize = s.weight_dtype == MDI_DTYPE_F32 ? 4 : 2;
+    c->kv_f32 = !(c->o.kv_cache_bf16 && s.weight_dtype == MDI_DTYPE_BF16);
+    c->kv_esize = c->kv_f32 ? 4 : 2;
     c->page_elems = (size_t)2 * s.n_kv_head * c->page_tokens * s.head_dim;
     c->n_split = c->o.attn_splits > 0 ? c->o.attn_splits : std::max(1, std::min(16, s.n_ctx / 128));
     c->rounds_per_graph = c->o.rounds_per_graph != 0 ? c->o.rounds_per_graph : 16;
@@ -707,7 +727,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
         CUB(cudaStreamCreateWithFlags(&P.stream, cudaStreamNonBlocking));
         const long pages_per_layer = (pool_tokens + c->page_tokens - 1) / c->page_tokens;
         P.n_pages = (int)(pages_per_layer * Lp);
-        P.kv_bytes = (size_t)P.n_pages * c->page_elems * c->esize;
+        P.kv_bytes = (size_t)P.n_pages * c->page_elems * c->kv_esize;
         CUB(cudaMalloc(&P.kv_pool, std::max<size_t>(P.kv_bytes, 16)));
         CUB(cudaMemset(P.kv_pool, 0, std::max<size_t>(P.kv_bytes, 16)));
         P.free_pages.resize(P.n_pages);

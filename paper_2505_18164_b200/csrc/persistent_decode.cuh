@@ -230,7 +230,7 @@ __device__ __forceinline__ void cblock_sum2(float &a, float &b, float *red /* [2
     for (int w = 0; w < PK_CWARPS; ++w) { a += red[w]; b += red[PK_CWARPS + w]; }
 }
 
-template <typename WT, int NB>
+template <typename WT, int NB, typename KT>
 __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkParams P) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int ES = sizeof(WT);
@@ -385,7 +385,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
             const int Kd = ph.in_dim, Kpad = (Kd + 255) & ~255;
             if (ph.kind == PK_ATTN) {
                 // ---------------- attention over the cache: items (item, head, split) dealt to the team's blocks
-                constexpr int EPL = VEC;
+                constexpr int EPL = 16 / (int)sizeof(KT);
                 const int LPR = hd / EPL, RPW = 32 / LPR, NG = PK_CWARPS * RPW;
                 const int sub = lane % LPR, grp = lane / LPR;
                 const int n_items = nb * P.n_head * T.n_split;
@@ -406,12 +406,12 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                         for (int j0 = lo + warp * RPW; j0 < hi; j0 += NG) {
                             const int jr = j0 + grp;
                             const bool live = jr < hi;
-                            const WT *kp = kv_addr<WT>(T.kv, slot, ph.layer_local, 0, kvh, live ? jr : lo, sub * EPL);
-                            const WT *vp = kp + (size_t)T.kv.n_kv_head * T.kv.page_tokens * hd;
+                            const KT *kp = kv_addr<KT>(T.kv, slot, ph.layer_local, 0, kvh, live ? jr : lo, sub * EPL);
+                            const KT *vp = kp + (size_t)T.kv.n_kv_head * T.kv.page_tokens * hd;
                             float kf[EPL], vf[EPL];
                             const uint4 kk = __ldcg(reinterpret_cast<const uint4 *>(kp)), vv = __ldcg(reinterpret_cast<const uint4 *>(vp));
-                            pk_unpack<ES>(kk, kf);
-                            pk_unpack<ES>(vv, vf);
+                            pk_unpack<(int)sizeof(KT)>(kk, kf);
+                            pk_unpack<(int)sizeof(KT)>(vv, vf);
                             float s = 0.f;
 #pragma unroll
                             for (int e = 0; e < EPL; ++e) s = fmaf(q[e], kf[e], s);
@@ -692,9 +692,9 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                                 if (row < qw) T.qbuf[(size_t)b * qw + row] = y;
                                 else {
                                     const int rk = row - qw, which = rk >= kw, rl = rk - which * kw;
-                                    WT *dst = reinterpret_cast<WT *>(T.kv.pool) + page_off[b] +
+                                    KT *dst = reinterpret_cast<KT *>(T.kv.pool) + page_off[b] +
                                               ((size_t)(which * T.kv.n_kv_head + rl / hd) * T.kv.page_tokens + (pos[b] & (T.kv.page_tokens - 1))) * hd + rl % hd;
-                                    kv_store<WT>(dst, y);
+                                    kv_store<KT>(dst, y);
                                 }
                             } else if (ph.kind == PK_FC1) {
                                 T.hbuf[(size_t)b * ph.n_rows + row] = pk_act(y, P.act);

@@ -158,7 +158,7 @@ __global__ void k_embed(const WT *wte, const WT *wpe, int d, int vocab, const in
 // ---- weight-streaming linear layer ------------------------------------------------------------
 // Each warp owns one unit of two weight rows and streams them once with 16-byte loads; the NB
 // input vectors sit in shared memory as fp32 (normalised in the prologue where asked).
-template <int NB, typename WT, int MODE>
+template <int NB, typename WT, int MODE, typename KT = WT>
 __global__ void __launch_bounds__(LIN_THREADS) k_linear(const LinArgs a, const Batch bt) {
     extern __shared__ __align__(16) float xs[]; // [NB][in_dim]
     __shared__ float red[LIN_WARPS];
@@ -285,7 +285,7 @@ __global__ void __launch_bounds__(LIN_THREADS) k_linear(const LinArgs a, const B
                     const int rk = r - a.q_rows;
                     const int which = rk >= a.kv_rows;
                     const int rl = rk - which * a.kv_rows;
-                    kv_store<WT>(kv_addr<WT>(a.kv, slot, a.layer_local, which, rl / hd, p, rl % hd), yy[j]);
+                    kv_store<KT>(kv_addr<KT>(a.kv, slot, a.layer_local, which, rl / hd, p, rl % hd), yy[j]);
                 }
             }
         }
