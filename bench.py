@@ -163,6 +163,21 @@ def run_reference(args, w: I.Workload):
         "gpu_launches": 0}))
 
 
+def max_over_ranks(values, world: int, device: str = "cpu"):
+    """Per-rank totals -> the slowest rank's (replicas run independently; the job is as slow as its slowest)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def aggregate_tokens_per_s(world: int, n_samples: int, n_new: int, steps: int, total_ms: float) -> float:
+    """Whole-job throughput: every rank generated n_samples * n_new tokens per step."""
+    return world * n_samples * n_new * steps / (total_ms * 1e-3)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -263,18 +278,15 @@ def main():
     barrier()
     assert np.array_equal(out_np, tokens_dev), "host and device entry points disagree"
 
-    tot_ms = torch.tensor([sum(run_ms), sum(e2e_s) * 1e3], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(tot_ms, op=dist.ReduceOp.MAX)
-    tot_run_ms, tot_e2e_ms = (float(v) for v in tot_ms.cpu())
+    tot_run_ms, tot_e2e_ms = max_over_ranks([sum(run_ms), sum(e2e_s) * 1e3], world, "cuda")
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
         db = decode_bytes(w, S)
         gen_avg_ms = sum(gen_ms) / len(gen_ms)
         achieved = db["total"] / (gen_avg_ms * 1e-3) / 1e9
-        value = world * S * N * args.steps / (tot_run_ms * 1e-3)
-        e2e_value = world * S * N * args.steps / (tot_e2e_ms * 1e-3)
+        value = aggregate_tokens_per_s(world, S, N, args.steps, tot_run_ms)
+        e2e_value = aggregate_tokens_per_s(world, S, N, args.steps, tot_e2e_ms)
         launches = int(st1.kernel_launches - st0.kernel_launches)
         line = {
             "metric": "generated tokens/s (all in-flight samples)", "value": value, "unit": "tokens/s",
