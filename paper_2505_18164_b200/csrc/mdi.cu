@@ -466,16 +466,30 @@ int pk_setup(mdi_ctx *c) {
         if ((int)v.size() == K && tot <= c->n_sm && *std::min_element(v.begin(), v.end()) >= 1) { n_cta = v; from_env = true; }
     }
     if (!from_env) {
+        // Proportional to the bytes a step streams, then rounded down to a size that deals the row blocks of
+        // the d_model-row matrices (and the attention items) out evenly - uneven shares make every phase wait
+        // for the blocks with one more tile - unless that would give up more than 30% of the share.
+        const int unit = (blocks16(d) % 2 == 0) ? blocks16(d) / 2 : blocks16(d);
+        auto even_size = [&](int share) {
+            int best = share;
+            if (share >= unit) best = share / unit * unit;
+            else
+                for (int k = 2; k <= unit; ++k)
+                    if (unit % k == 0 && unit / k <= share) { best = unit / k; break; }
+            return best * 10 >= share * 7 ? best : share;
+        };
         double tot = 0;
         for (double b : bytes) tot += b;
         int used = 0, big = 0;
-        for (int p = 0; p < K; ++p) {
-            n_cta[p] = std::max(1, (int)std::floor(c->n_sm * bytes[p] / tot));
-            used += n_cta[p];
+        for (int p = 0; p < K; ++p)
             if (bytes[p] > bytes[big]) big = p;
+        for (int p = 0; p < K; ++p) {
+            if (p == big) continue;
+            n_cta[p] = even_size(std::max(1, (int)std::floor(c->n_sm * bytes[p] / tot)));
+            used += n_cta[p];
         }
-        n_cta[big] += c->n_sm - used;
-        if (n_cta[big] < 1) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: not enough SMs") : MDI_OK;
+        if (c->n_sm - used < 1) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: not enough SMs") : MDI_OK;
+        n_cta[big] = even_size(c->n_sm - used);
     }
     c->pk_teams_host.assign(K, PkTeam{});
     int first = 0, rcx;

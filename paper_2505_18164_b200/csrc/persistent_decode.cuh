@@ -457,6 +457,56 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
             for (int b = 0; b < NB; ++b) {
                 const bool live = b < nb;
                 const int slot = slots[b];
+                // Common case (the source is a plain fp32 vector of at most 4096 elements: every phase but the
+                // embedding and the split merge): float4 loads, the values stay in registers through the norm
+                // statistics, and shared memory is written once.
+                const bool plain = !(ph.kind == PK_QKV && ph.first_layer && T.is_first) && ph.kind != PK_OUT;
+                if (plain && Kd <= 4 * 4 * PK_CTHREADS) {
+                    const float *src = ph.kind == PK_QKV ? (ph.first_layer ? x_in : x_out) + (size_t)b * d
+                                       : ph.kind == PK_FC2 ? T.hbuf + (size_t)b * Kd
+                                                           : x_out + (size_t)b * d;
+                    const float4 *src4 = reinterpret_cast<const float4 *>(src);
+                    const int n4 = Kd >> 2;
+                    float4 v[4], g4[4], o4[4];
+                    const bool layer_norm = ph.gamma && P.norm == NORM_LAYER;
+                    const float pilot = (live && layer_norm) ? __ldcg(src) : 0.f;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int i4 = tid + u * PK_CTHREADS;
+                        const bool in = i4 < n4;
+                        v[u] = (live && in) ? __ldcg(src4 + i4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        g4[u] = (ph.gamma && in) ? reinterpret_cast<const float4 *>(ph.gamma)[i4] : make_float4(0.f, 0.f, 0.f, 0.f);
+                        o4[u] = (ph.gamma && ph.beta && in) ? reinterpret_cast<const float4 *>(ph.beta)[i4] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    if (ph.gamma) {
+                        // one reduction for both moments, taken about a pilot value (the row's first element) so that
+                        // the variance does not cancel when the mean is large
+                        float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (tid + u * PK_CTHREADS < n4) {
+                                const float c0 = v[u].x - pilot, c1 = v[u].y - pilot, c2 = v[u].z - pilot, c3 = v[u].w - pilot;
+                                s1 += (c0 + c1) + (c2 + c3);
+                                s2 += (c0 * c0 + c1 * c1) + (c2 * c2 + c3 * c3);
+                            }
+                        cblock_sum2(s1, s2, red);
+                        const float dm = layer_norm ? s1 / (float)Kd : 0.f, mean = pilot + dm;
+                        const float rstd = rsqrtf(fmaxf(s2 / (float)Kd - dm * dm, 0.f) + P.eps);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            v[u].x = (v[u].x - mean) * rstd * g4[u].x + o4[u].x;
+                            v[u].y = (v[u].y - mean) * rstd * g4[u].y + o4[u].y;
+                            v[u].z = (v[u].z - mean) * rstd * g4[u].z + o4[u].z;
+                            v[u].w = (v[u].w - mean) * rstd * g4[u].w + o4[u].w;
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int i4 = tid + u * PK_CTHREADS;
+                        if (i4 < n4) *reinterpret_cast<float4 *>(xs + b * Kpad + xs_perm<ES>(4 * i4)) = v[u];
+                    }
+                    continue;
+                }
                 // Source of the staged row: a plain fp32 vector for most phases (loads issued in batches of 8 per
                 // thread so that a batch costs one round trip to L2); the embedding and the split merge have
                 // their own short loops.
