@@ -472,6 +472,7 @@ int pk_setup(mdi_ctx *c) {
         const int unit = (blocks16(d) % 2 == 0) ? blocks16(d) / 2 : blocks16(d);
         auto even_size = [&](int share) {
             int best = share;
+            if ((share + 1) % unit == 0 || (unit % (share + 1) == 0)) return share + 1; // one block short of an even size
             if (share >= unit) best = share / unit * unit;
             else
                 for (int k = 2; k <= unit; ++k)
