@@ -72,6 +72,9 @@ typedef struct {
     int kv_cache_bf16; /* 0 (default): the key/value cache holds fp32; 1: with bf16 weights, hold bf16 instead - half the
                           cache bytes, at about 2e-3 relative error per block on the activations (measured), which on a
                           32-block model exceeds a 3e-2 absolute logit tolerance */
+    int prefill_mode;  /* first visits (whole prompt): 0 (default) tensor-core GEMMs (tcgen05, bf16 x bf16 -> fp32, inputs split
+                          into two bf16 planes) when the weights are bf16, else the CUDA-core step kernels in chunks of 8
+                          positions; 1: always the CUDA-core kernels */
     int scheduler;     /* how mdi_generate runs the recurrent pipeline.  0: the persistent kernel (one launch,
                           one team of thread blocks per partition, flag handoff between teams) when the shape
                           fits it (groups of at most 4 samples), else the stream scheduler; 1: always the

@@ -12,10 +12,13 @@
 #include <cstring>
 #include <map>
 #include <string>
+#include <tuple>
 #include <vector>
 
 #include "persistent_decode.cuh"
+#include "prefill_kernels.cuh"
 #include "step_kernels.cuh"
+#include "tc_gemm.cuh"
 
 using namespace mdi;
 
@@ -60,6 +63,9 @@ struct Partition {
     cudaEvent_t ev_pf_out[2] = {nullptr, nullptr}, ev_pf_used[2] = {nullptr, nullptr};
     bool pf_used_valid[2] = {false, false};
     cudaEvent_t ev_join = nullptr, ev_join_cap = nullptr;
+    // tensor-core first visit: inputs as bf16 hi/lo planes, fp32 intermediates, for up to PF_CHUNK positions
+    uint16_t *pf_hi = nullptr, *pf_lo = nullptr;
+    float *pf_qkv = nullptr, *pf_q = nullptr, *pf_o = nullptr, *pf_h = nullptr, *pf_u = nullptr, *pf_xa = nullptr, *pf_xb = nullptr;
     int64_t weight_bytes = 0, buffer_bytes = 0;
 };
 
@@ -101,6 +107,10 @@ struct mdi_ctx {
     std::map<std::pair<int, int>, GraphEntry> graphs; // (n_samples, window ticks)
     bool capturing = false;
     int64_t cap_launches = 0, cap_steps = 0;
+    // tensor-core first visit
+    bool pf_tc = false;
+    int *tg_err = nullptr;
+    std::map<std::tuple<const void *, uint64_t, uint64_t, uint32_t>, CUtensorMap> tmaps;
     // persistent decode kernel
     bool pk_ok = false, pk_prof_on = false, pk_tables_stale = true;
     int pk_slots = 0, pk_xs_floats = 0, pk_nb = 1, n_sm = 0, scheduler = 0;
@@ -263,6 +273,22 @@ struct HeadReq {
     int *tok_out = nullptr;
 };
 
+// Output layers for the items of hb (final norm, vocabulary projection, greedy argmax); x_rows: [hb.n][d].
+int enqueue_head(mdi_ctx *c, const Batch &hb, const float *x_rows, const HeadReq &head, cudaStream_t st) {
+    const mdi_model_shape &s = c->s;
+    LinArgs a{};
+    a.W = s.tied_lm_head ? c->wte : c->lm_head; a.n_rows = s.vocab; a.in_dim = s.d_model;
+    a.x_in = x_rows;
+    a.norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS; a.gamma = c->lnfg; a.beta = c->lnfb; a.eps = s.norm_eps;
+    a.logits = c->logits; a.part_val = c->head_pv; a.part_idx = c->head_pi; a.ticket = c->head_ticket;
+    a.tok_out = head.tok_out; a.log_stride = s.n_ctx;
+    if (head.update_state) {
+        a.cur_tok = c->cur_tok; a.tok_log = c->tok_log; a.gen_count = c->gen_count;
+        a.teacher = c->teacher; a.n_teacher = c->n_teacher;
+    }
+    return linear(c, LIN_HEAD, a, hb, st);
+}
+
 // All kernels of one visit of a batch of items to partition p.
 //   x_in:  [n][d] input activations (ignored for p == 0, which embeds tokens from tok_src)
 //   x_out: [n][d] where the partition's output activations are written
@@ -328,21 +354,151 @@ int enqueue_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in
         }
     }
     if (head && p == c->K - 1) {
-        Batch hb = head->item < 0 ? bt : slice(bt, head->item, 1);
-        LinArgs a{};
-        a.W = s.tied_lm_head ? c->wte : c->lm_head; a.n_rows = s.vocab; a.in_dim = d;
-        a.x_in = head->item < 0 ? x_out : x_out + (size_t)head->item * d;
-        a.norm = norm; a.gamma = c->lnfg; a.beta = c->lnfb; a.eps = s.norm_eps;
-        a.logits = c->logits; a.part_val = c->head_pv; a.part_idx = c->head_pi; a.ticket = c->head_ticket;
-        a.tok_out = head->tok_out; a.log_stride = s.n_ctx;
-        if (head->update_state) {
-            a.cur_tok = c->cur_tok; a.tok_log = c->tok_log; a.gen_count = c->gen_count;
-            a.teacher = c->teacher; a.n_teacher = c->n_teacher;
-        }
-        int rc = linear(c, LIN_HEAD, a, hb, st);
+        const Batch hb = head->item < 0 ? bt : slice(bt, head->item, 1);
+        const int rc = enqueue_head(c, hb, head->item < 0 ? x_out : x_out + (size_t)head->item * d, *head, st);
         if (rc != MDI_OK) return rc;
     }
     if (c->capturing) ++c->cap_steps; else ++c->st.stage_steps;
+    return MDI_OK;
+}
+
+
+// ---- first visit on tensor cores (bf16 weights): GEMMs of tc_gemm.cuh + helpers of prefill_kernels.cuh ----
+constexpr int PF_CHUNK = 128; // positions per pass through a partition (one tile of positions per GEMM block)
+
+int pf_setup(mdi_ctx *c) {
+    const mdi_model_shape &s = c->s;
+    c->pf_tc = s.weight_dtype == MDI_DTYPE_BF16 && c->o.prefill_mode != 1;
+    if (!c->pf_tc) return MDI_OK;
+    CU(cudaFuncSetAttribute(k_tc_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TG_SMEM));
+    const int d = s.d_model, F = s.d_ff, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim;
+    const size_t maxk = (size_t)std::max(std::max(d, F), qw);
+    int rc;
+    if ((rc = dalloc(c, &c->tg_err, 1)) != MDI_OK) return rc;
+    for (auto &P : c->part) {
+        if ((rc = dalloc(c, &P.pf_hi, PF_CHUNK * maxk, &P.buffer_bytes)) != MDI_OK) return rc;
+        if ((rc = dalloc(c, &P.pf_lo, PF_CHUNK * maxk, &P.buffer_bytes)) != MDI_OK) return rc;
+        if ((rc = dalloc(c, &P.pf_qkv, (size_t)PF_CHUNK * (qw + 2 * kw), &P.buffer_bytes)) != MDI_OK) return rc;
+        if ((rc = dalloc(c, &P.pf_q, (size_t)PF_CHUNK * qw, &P.buffer_bytes)) != MDI_OK) return rc;
+        if ((rc = dalloc(c, &P.pf_o, (size_t)PF_CHUNK * qw, &P.buffer_bytes)) != MDI_OK) return rc;
+        if ((rc = dalloc(c, &P.pf_h, (size_t)PF_CHUNK * F, &P.buffer_bytes)) != MDI_OK) return rc;
+        if (s.act == MDI_ACT_SWIGLU && (rc = dalloc(c, &P.pf_u, (size_t)PF_CHUNK * F, &P.buffer_bytes)) != MDI_OK) return rc;
+        if ((rc = dalloc(c, &P.pf_xa, (size_t)PF_CHUNK * d, &P.buffer_bytes)) != MDI_OK) return rc;
+        if ((rc = dalloc(c, &P.pf_xb, (size_t)PF_CHUNK * d, &P.buffer_bytes)) != MDI_OK) return rc;
+    }
+    return MDI_OK;
+}
+
+// Tensor maps are cached by (base address, rows, columns, box rows): weights never move, scratch neither.
+int pf_map(mdi_ctx *c, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows, const CUtensorMap **out) {
+    auto key = std::make_tuple(base, rows, cols, box_rows);
+    auto it = c->tmaps.find(key);
+    if (it == c->tmaps.end()) {
+        CUtensorMap m;
+        const CUresult r = tg_make_map(&m, base, rows, cols, box_rows);
+        if (r != CUDA_SUCCESS) return fail(c, MDI_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) for a %llu x %llu matrix", (int)r,
+                                           (unsigned long long)rows, (unsigned long long)cols);
+        it = c->tmaps.emplace(key, m).first;
+    }
+    *out = &it->second;
+    return MDI_OK;
+}
+
+// y[t][r] = act(W[r][:] . x[t][:] + bias[r] + resid[t][r]) for T positions whose inputs sit in P.pf_hi / P.pf_lo.
+int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, const float *bias, const float *resid, int act,
+            float *y, cudaStream_t st) {
+    const int n_tile = T <= 16 ? 16 : T <= 32 ? 32 : T <= 64 ? 64 : 128;
+    const CUtensorMap *mw, *mhi, *mlo;
+    int rc;
+    if ((rc = pf_map(c, W, (uint64_t)n_rows, (uint64_t)K, TG_BM, &mw)) != MDI_OK) return rc;
+    if ((rc = pf_map(c, P.pf_hi, PF_CHUNK, (uint64_t)K, (uint32_t)n_tile, &mhi)) != MDI_OK) return rc;
+    if ((rc = pf_map(c, P.pf_lo, PF_CHUNK, (uint64_t)K, (uint32_t)n_tile, &mlo)) != MDI_OK) return rc;
+    TgArgs a{};
+    a.n_rows = n_rows; a.K = K; a.T = T; a.n_tile = n_tile; a.bias = bias; a.resid = resid; a.act = act; a.y = y; a.ldy = n_rows;
+    a.err = c->tg_err;
+    k_tc_gemm<<<dim3((n_rows + TG_BM - 1) / TG_BM, (T + n_tile - 1) / n_tile), TG_THREADS, TG_SMEM, st>>>(*mw, *mhi, *mlo, a);
+    count_launch(c);
+    return MDI_OK;
+}
+
+template <typename KT> void pf_attn_hd(int hd, dim3 g, cudaStream_t st, const float *q, float *o, const KvView &kv, int ll, int n_head,
+                                       const int *pos, int slot, float scale) {
+    switch (hd) {
+        case 16: k_pf_attn<KT, 16><<<g, ATT_THREADS, 0, st>>>(q, o, kv, ll, n_head, pos, slot, scale); break;
+        case 32: k_pf_attn<KT, 32><<<g, ATT_THREADS, 0, st>>>(q, o, kv, ll, n_head, pos, slot, scale); break;
+        case 64: k_pf_attn<KT, 64><<<g, ATT_THREADS, 0, st>>>(q, o, kv, ll, n_head, pos, slot, scale); break;
+        default: k_pf_attn<KT, 128><<<g, ATT_THREADS, 0, st>>>(q, o, kv, ll, n_head, pos, slot, scale); break;
+    }
+}
+
+// T (<= PF_CHUNK) new positions of one slot through partition p.  x_in: [T][d] (ignored for p == 0, which embeds
+// tok_dev[0..T)); x_out: [T][d].  Cache rows pos .. pos+T-1 are written and pos advances by T at the end.
+int pf_partition_chunk(mdi_ctx *c, int p, int slot, const int *tok_dev, int T, const float *x_in, float *x_out, cudaStream_t st) {
+    Partition &P = c->part[p];
+    const mdi_model_shape &s = c->s;
+    const int d = s.d_model, F = s.d_ff, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim;
+    const int norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS;
+    const KvView kv = kv_view(c, P);
+    const float scale = 1.0f / std::sqrt((float)s.head_dim);
+    __nv_bfloat16 *hi = (__nv_bfloat16 *)P.pf_hi, *lo = (__nv_bfloat16 *)P.pf_lo;
+    int rc;
+    if (p == 0) {
+        k_pf_embed<__nv_bfloat16><<<T, 256, 0, st>>>((const __nv_bfloat16 *)c->wte, (const __nv_bfloat16 *)c->wpe, d, s.vocab, tok_dev,
+                                                    P.pos_dev, slot, P.pf_xa);
+        count_launch(c);
+        x_in = P.pf_xa;
+    }
+    for (int l = P.lo; l < P.hi; ++l) {
+        const LayerW &L = c->layer[l];
+        const float *xin_l = l == P.lo ? x_in : x_out;
+        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(xin_l, d, norm, L.ln1g, L.ln1b, s.norm_eps, hi, lo);
+        count_launch(c);
+        if ((rc = pf_gemm(c, P, L.wqkv, qw + 2 * kw, d, T, L.bqkv, nullptr, TG_NONE, P.pf_qkv, st)) != MDI_OK) return rc;
+        if (c->kv_f32)
+            k_pf_rope_append<float><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, s.arch == MDI_ARCH_LLAMA, c->rope_cos, c->rope_sin, kv,
+                                                       l - P.lo, P.pos_dev, slot, P.pf_q);
+        else
+            k_pf_rope_append<__nv_bfloat16><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, s.arch == MDI_ARCH_LLAMA, c->rope_cos,
+                                                               c->rope_sin, kv, l - P.lo, P.pos_dev, slot, P.pf_q);
+        count_launch(c);
+        if (c->kv_f32) pf_attn_hd<float>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, P.pf_o, kv, l - P.lo, s.n_head, P.pos_dev, slot, scale);
+        else pf_attn_hd<__nv_bfloat16>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, P.pf_o, kv, l - P.lo, s.n_head, P.pos_dev, slot, scale);
+        count_launch(c);
+        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.pf_o, qw, NORM_NONE, nullptr, nullptr, 0.f, hi, lo);
+        count_launch(c);
+        if ((rc = pf_gemm(c, P, L.wo, d, qw, T, L.bo, xin_l, TG_NONE, x_out, st)) != MDI_OK) return rc;
+        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(x_out, d, norm, L.ln2g, L.ln2b, s.norm_eps, hi, lo);
+        count_launch(c);
+        if (s.act == MDI_ACT_SWIGLU) {
+            if ((rc = pf_gemm(c, P, L.wgate, F, d, T, nullptr, nullptr, TG_NONE, P.pf_h, st)) != MDI_OK) return rc;
+            if ((rc = pf_gemm(c, P, L.wup, F, d, T, nullptr, nullptr, TG_NONE, P.pf_u, st)) != MDI_OK) return rc;
+            k_pf_swiglu_split<<<T, 256, 0, st>>>(P.pf_h, P.pf_u, F, hi, lo);
+            count_launch(c);
+            if ((rc = pf_gemm(c, P, L.wdown, d, F, T, nullptr, x_out, TG_NONE, x_out, st)) != MDI_OK) return rc;
+        } else {
+            if ((rc = pf_gemm(c, P, L.w1, F, d, T, L.b1, nullptr, s.act == MDI_ACT_GELU_ERF ? TG_GELU_ERF : TG_GELU_TANH, P.pf_h, st)) != MDI_OK)
+                return rc;
+            k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo);
+            count_launch(c);
+            if ((rc = pf_gemm(c, P, L.w2, d, F, T, L.b2, x_out, TG_NONE, x_out, st)) != MDI_OK) return rc;
+        }
+    }
+    k_pf_advance<<<1, 32, 0, st>>>(P.pos_dev, slot, T);
+    count_launch(c);
+    ++c->st.stage_steps;
+    return MDI_OK;
+}
+
+// Did a tensor-core first visit give up on one of its bounded waits?  (Synchronises the partition streams.)
+int pf_check(mdi_ctx *c) {
+    if (!c->pf_tc) return MDI_OK;
+    for (auto &P : c->part) CU(cudaStreamSynchronize(P.stream));
+    int e = 0;
+    CU(cudaMemcpy(&e, c->tg_err, sizeof(int), cudaMemcpyDeviceToHost));
+    if (e) {
+        CU(cudaMemset(c->tg_err, 0, sizeof(int)));
+        return fail(c, MDI_ERR_TIMEOUT, "a tensor-core first-visit kernel gave up waiting for its operands");
+    }
     return MDI_OK;
 }
 
@@ -600,7 +756,7 @@ void mdi_destroy(mdi_ctx *c) {
     }
     for (auto &P : c->part) {
         void *ptrs[] = {P.kv_pool, P.pt_dev, P.pos_dev, P.x_embed, P.qbuf, P.obuf, P.hbuf, P.part, P.x_last, P.attn_ticket,
-                        P.ring, P.pf_buf[0], P.pf_buf[1]};
+                        P.ring, P.pf_buf[0], P.pf_buf[1], P.pf_hi, P.pf_lo, P.pf_qkv, P.pf_q, P.pf_o, P.pf_h, P.pf_u, P.pf_xa, P.pf_xb};
         for (void *q : ptrs) if (q) cudaFree(q);
         for (auto e : P.ev_edge) cudaEventDestroy(e);
         for (auto e : P.ev_edge_cap) cudaEventDestroy(e);
@@ -610,7 +766,7 @@ void mdi_destroy(mdi_ctx *c) {
         if (P.stream) cudaStreamDestroy(P.stream);
     }
     void *ptrs[] = {c->rope_cos, c->rope_sin, c->logits, c->head_pv, c->head_pi, c->head_ticket, c->cur_tok, c->tok_log,
-                    c->gen_count, c->teacher, c->n_teacher, c->prompt_buf, c->pk_teams, c->pk_phases, c->pk_sync, c->pk_err, c->pk_prof};
+                    c->gen_count, c->teacher, c->n_teacher, c->prompt_buf, c->pk_teams, c->pk_phases, c->pk_sync, c->pk_err, c->pk_prof, c->tg_err};
     for (void *q : ptrs) if (q) cudaFree(q);
     cudaEvent_t evs[] = {c->ev_fork, c->ev_fork_cap, c->ev_t0, c->ev_t1, c->ev_pf0, c->ev_pf1};
     for (auto e : evs) if (e) cudaEventDestroy(e);
@@ -667,6 +823,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     c->page_elems = (size_t)2 * s.n_kv_head * c->page_tokens * s.head_dim;
     c->n_split = c->o.attn_splits > 0 ? c->o.attn_splits : std::max(1, std::min(16, s.n_ctx / 128));
     c->rounds_per_graph = c->o.rounds_per_graph != 0 ? c->o.rounds_per_graph : 16;
+    if (c->o.prefill_mode < 0 || c->o.prefill_mode > 1) return bail(fail(c, MDI_ERR_ARG, "prefill_mode must be 0 or 1"));
     c->scheduler = c->o.scheduler;
     if (c->scheduler < 0 || c->scheduler > 2) return bail(fail(c, MDI_ERR_ARG, "scheduler must be 0, 1 or 2"));
     const int G = std::min(n_samples, K);
@@ -796,6 +953,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     c->returned_host.assign(n_samples, 0);
     c->prefilled.assign(n_samples, 0);
     TRY(pk_setup(c));
+    TRY(pf_setup(c));
     CUB(cudaDeviceSynchronize());
 #undef TRY
 #undef CUB
@@ -885,7 +1043,19 @@ static int prefill_impl(mdi_ctx *c, int sample, const int32_t *prompt, int n, bo
         Partition &P = c->part[p];
         if (p > 0) CU(cudaStreamWaitEvent(P.stream, c->part[p - 1].ev_pf_out[par], 0));
         if (p < K - 1 && c->part[p + 1].pf_used_valid[par]) CU(cudaStreamWaitEvent(P.stream, c->part[p + 1].ev_pf_used[par], 0));
-        for (int c0 = 0; c0 < n; c0 += MAXB) {
+        for (int c0 = 0; c->pf_tc && c0 < n; c0 += PF_CHUNK) {
+            const int m = std::min(PF_CHUNK, n - c0);
+            const float *x_in = p > 0 ? c->part[p - 1].pf_buf[par] + (size_t)c0 * d : nullptr;
+            float *x_out = p < K - 1 ? P.pf_buf[par] + (size_t)c0 * d : P.pf_xb;
+            if ((rc = pf_partition_chunk(c, p, sample, pbuf + c0, m, x_in, x_out, P.stream)) != MDI_OK) return rc;
+            if (p == K - 1 && c0 + m == n) {
+                Batch hb{};
+                hb.n = 1; hb.slot[0] = sample;
+                HeadReq hr;
+                if ((rc = enqueue_head(c, hb, x_out + (size_t)(m - 1) * d, hr, P.stream)) != MDI_OK) return rc;
+            }
+        }
+        for (int c0 = 0; !c->pf_tc && c0 < n; c0 += MAXB) {
             const int m = std::min(MAXB, n - c0);
             Batch bt{};
             bt.n = m;
@@ -1013,6 +1183,7 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
         CU(cudaStreamWaitEvent(c->main, c->part[p].ev_join, 0));
     }
     CU(cudaEventRecord(c->ev_t0, c->main));
+    if ((rc = pf_check(c)) != MDI_OK) return rc;
     const long total = (long)n_pass * K;        // phase slots per partition
     const long t_total = total ? total + K - 1 : 0;
     long t = 0;

@@ -1,0 +1,153 @@
+// Helper kernels of the tensor-core first visit (whole prompt through a partition): everything around
+// the GEMMs of tc_gemm.cuh.  Activations are fp32 [position][feature]; the GEMM inputs are written as two
+// bf16 planes (hi, lo) with x = hi + lo to about 16 mantissa bits, so that the tensor cores lose nothing
+// that matters against the fp32 CUDA-core path.
+#pragma once
+#include "step_kernels.cuh"
+
+namespace mdi {
+
+constexpr int PF_THREADS = 256;
+
+__device__ __forceinline__ void pf_split_store(__nv_bfloat16 *hi, __nv_bfloat16 *lo, size_t i, float v) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    hi[i] = h;
+    lo[i] = __float2bfloat16_rn(v - __bfloat162float(h));
+}
+
+// x[t][:] = wte[tok[t]][:] (+ wpe[pos0 + t][:]);  grid (T)
+template <typename WT>
+__global__ void k_pf_embed(const WT *wte, const WT *wpe, int d, int vocab, const int *tok, const int *pos, int slot, float *x) {
+    const int t = blockIdx.x;
+    const int id = min(max(tok[t], 0), vocab - 1);
+    const int p = pos[slot] + t;
+    for (int e = threadIdx.x; e < d; e += blockDim.x) {
+        float v = __bfloat162float(wte[(size_t)id * d + e]);
+        if (wpe) v += __bfloat162float(wpe[(size_t)p * d + e]);
+        x[(size_t)t * d + e] = v;
+    }
+}
+
+// Row-wise LayerNorm / RMSNorm (or plain copy when gamma is null) followed by the hi/lo split.  grid (T)
+__global__ void __launch_bounds__(PF_THREADS) k_pf_norm_split(const float *x, int n, int norm, const float *gamma, const float *beta,
+                                                               float eps, __nv_bfloat16 *hi, __nv_bfloat16 *lo) {
+    __shared__ float red[2 * PF_THREADS / 32];
+    const int t = blockIdx.x, tid = threadIdx.x;
+    const float *row = x + (size_t)t * n;
+    float mean = 0.f, rstd = 1.f;
+    if (gamma) {
+        const float pilot = norm == NORM_LAYER ? row[0] : 0.f;
+        float s1 = 0.f, s2 = 0.f;
+        for (int i = tid; i < n; i += PF_THREADS) { const float c = row[i] - pilot; s1 += c; s2 += c * c; }
+        s1 = warp_sum(s1);
+        s2 = warp_sum(s2);
+        if ((tid & 31) == 0) { red[tid >> 5] = s1; red[PF_THREADS / 32 + (tid >> 5)] = s2; }
+        __syncthreads();
+        s1 = s2 = 0.f;
+        for (int w = 0; w < PF_THREADS / 32; ++w) { s1 += red[w]; s2 += red[PF_THREADS / 32 + w]; }
+        const float dm = norm == NORM_LAYER ? s1 / (float)n : 0.f;
+        mean = pilot + dm;
+        rstd = rsqrtf(fmaxf(s2 / (float)n - dm * dm, 0.f) + eps);
+    }
+    for (int i = tid; i < n; i += PF_THREADS) {
+        float v = row[i];
+        if (gamma) { v = (v - mean) * rstd * gamma[i]; if (beta) v += beta[i]; }
+        pf_split_store(hi, lo, (size_t)t * n + i, v);
+    }
+}
+
+// h = SiLU(g) * u, split.  grid (T)
+__global__ void k_pf_swiglu_split(const float *g, const float *u, int n, __nv_bfloat16 *hi, __nv_bfloat16 *lo) {
+    const int t = blockIdx.x;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const size_t k = (size_t)t * n + i;
+        pf_split_store(hi, lo, k, silu_f(g[k]) * u[k]);
+    }
+}
+
+// qkv[t][q | k | v] (bias already added) -> q[t][:] (rotated) and the cache rows pos0 + t (k rotated).  grid (T)
+template <typename KT>
+__global__ void k_pf_rope_append(const float *qkv, int q_rows, int kv_rows, int hd, int rope, const float *rope_cos,
+                                 const float *rope_sin, KvView kv, int layer_local, const int *pos, int slot, float *q_out) {
+    const int t = blockIdx.x, p = pos[slot] + t, half = hd >> 1, rows = q_rows + 2 * kv_rows;
+    const float *src = qkv + (size_t)t * rows;
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+        float y = src[r];
+        if (rope && r < q_rows + kv_rows) {
+            const int e = r % hd, i = e % half;
+            const float c = rope_cos[(size_t)p * half + i], s = rope_sin[(size_t)p * half + i];
+            y = e < half ? y * c - src[r + half] * s : y * c + src[r - half] * s;
+        }
+        if (r < q_rows) q_out[(size_t)t * q_rows + r] = y;
+        else {
+            const int rk = r - q_rows, which = rk >= kv_rows, rl = rk - which * kv_rows;
+            kv_store<KT>(kv_addr<KT>(kv, slot, layer_local, which, rl / hd, p, rl % hd), y);
+        }
+    }
+}
+
+// Causal attention of the T new positions over the slot's cache (rows 0 .. pos0 + t for position t).
+// grid (n_head, T); same row-sharing scheme as k_attn_decode, no sequence split.
+template <typename KT, int HD>
+__global__ void __launch_bounds__(ATT_THREADS) k_pf_attn(const float *q, float *o, KvView kv, int layer_local, int n_head,
+                                                          const int *pos, int slot, float scale) {
+    constexpr int EPL = 16 / sizeof(KT), LPR = HD / EPL, RPW = 32 / LPR, NG = ATT_WARPS * RPW;
+    __shared__ float sm_m[NG], sm_l[NG];
+    __shared__ float sm_o[NG][HD];
+    const int h = blockIdx.x, t = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, grp = lane / LPR;
+    const int n_keys = pos[slot] + t + 1;
+    const int kvh = h / (n_head / kv.n_kv_head);
+    float qv[EPL], ov[EPL];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) { qv[e] = q[((size_t)t * n_head + h) * HD + sub * EPL + e] * scale; ov[e] = 0.f; }
+    float m = -INFINITY, l = 0.f;
+    for (int j0 = warp * RPW; j0 < n_keys; j0 += NG) {
+        const int j = j0 + grp;
+        const bool live = j < n_keys;
+        const KT *kp = kv_addr<KT>(kv, slot, layer_local, 0, kvh, live ? j : 0, sub * EPL);
+        const KT *vp = kp + (size_t)kv.n_kv_head * kv.page_tokens * HD;
+        WVec<KT> kk, vv;
+        kk.load(kp);
+        vv.load(vp);
+        float kf[EPL], vf[EPL];
+        kk.unpack(kf);
+        vv.unpack(vf);
+        float s = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) s = fmaf(qv[e], kf[e], s);
+#pragma unroll
+        for (int w = LPR / 2; w > 0; w >>= 1) s += __shfl_xor_sync(0xffffffffu, s, w);
+        if (live) {
+            const float mn = fmaxf(m, s), corr = expf(m - mn), pr = expf(s - mn);
+            l = l * corr + pr;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) ov[e] = ov[e] * corr + pr * vf[e];
+            m = mn;
+        }
+    }
+    const int g = warp * RPW + grp;
+    if (sub == 0) { sm_m[g] = m; sm_l[g] = l; }
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) sm_o[g][sub * EPL + e] = ov[e];
+    __syncthreads();
+    if (tid < HD) {
+        float M = -INFINITY;
+#pragma unroll
+        for (int g2 = 0; g2 < NG; ++g2) M = fmaxf(M, sm_m[g2]);
+        float L = 0.f, O = 0.f;
+#pragma unroll
+        for (int g2 = 0; g2 < NG; ++g2) {
+            const float w = sm_m[g2] == -INFINITY ? 0.f : expf(sm_m[g2] - M);
+            L += sm_l[g2] * w;
+            O += sm_o[g2][tid] * w;
+        }
+        o[((size_t)t * n_head + h) * HD + tid] = O / L;
+    }
+}
+
+__global__ void k_pf_advance(int *pos, int slot, int by) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) pos[slot] += by;
+}
+
+} // namespace mdi
