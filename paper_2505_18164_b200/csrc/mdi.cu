@@ -289,6 +289,8 @@ int enqueue_head(mdi_ctx *c, const Batch &hb, const float *x_rows, const HeadReq
     return linear(c, LIN_HEAD, a, hb, st);
 }
 
+int tc_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in, float *x_out, cudaStream_t st);
+
 // All kernels of one visit of a batch of items to partition p.
 //   x_in:  [n][d] input activations (ignored for p == 0, which embeds tokens from tok_src)
 //   x_out: [n][d] where the partition's output activations are written
@@ -307,7 +309,13 @@ int enqueue_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in
         x_in = P.x_embed;
     }
     const KvView kv = kv_view(c, P);
-    for (int l = P.lo; l < P.hi; ++l) {
+    // groups of more than 4 items with bf16 weights: the linear layers run on the tensor cores
+    const bool tc = c->pf_tc && bt.n > 4;
+    if (tc) {
+        const int rc = tc_partition_step(c, p, bt, x_in, x_out, st);
+        if (rc != MDI_OK) return rc;
+    }
+    for (int l = P.lo; l < P.hi && !tc; ++l) {
         const LayerW &L = c->layer[l];
         const float *xin_l = l == P.lo ? x_in : x_out;
         int rc;
@@ -486,6 +494,62 @@ int pf_partition_chunk(mdi_ctx *c, int p, int slot, const int *tok_dev, int T, c
     k_pf_advance<<<1, 32, 0, st>>>(P.pos_dev, slot, T);
     count_launch(c);
     ++c->st.stage_steps;
+    return MDI_OK;
+}
+
+// A group's decode step (5..8 items of different slots, one new position each) with the linear layers on the
+// tensor cores: the weights of the partition are streamed once by TMA for the whole group.
+int tc_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in, float *x_out, cudaStream_t st) {
+    Partition &P = c->part[p];
+    const mdi_model_shape &s = c->s;
+    const int d = s.d_model, F = s.d_ff, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim, T = bt.n;
+    const int norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS;
+    const KvView kv = kv_view(c, P);
+    __nv_bfloat16 *hi = (__nv_bfloat16 *)P.pf_hi, *lo = (__nv_bfloat16 *)P.pf_lo;
+    int rc;
+    for (int l = P.lo; l < P.hi; ++l) {
+        const LayerW &L = c->layer[l];
+        const float *xin_l = l == P.lo ? x_in : x_out;
+        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(xin_l, d, norm, L.ln1g, L.ln1b, s.norm_eps, hi, lo);
+        count_launch(c);
+        if ((rc = pf_gemm(c, P, L.wqkv, qw + 2 * kw, d, T, L.bqkv, nullptr, TG_NONE, P.pf_qkv, st)) != MDI_OK) return rc;
+        if (c->kv_f32)
+            k_bt_rope_append<float><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, s.arch == MDI_ARCH_LLAMA, c->rope_cos, c->rope_sin, kv,
+                                                       l - P.lo, P.pos_dev, bt, P.qbuf);
+        else
+            k_bt_rope_append<__nv_bfloat16><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, s.arch == MDI_ARCH_LLAMA, c->rope_cos,
+                                                               c->rope_sin, kv, l - P.lo, P.pos_dev, bt, P.qbuf);
+        count_launch(c);
+        {
+            AttnArgs a{};
+            a.q = P.qbuf; a.o = P.obuf; a.part = P.part; a.ticket = P.attn_ticket; a.kv = kv;
+            a.layer_local = l - P.lo; a.n_head = s.n_head; a.n_split = c->n_split; a.pos = P.pos_dev;
+            a.scale = 1.0f / std::sqrt((float)s.head_dim);
+            dim3 g(s.n_head, c->n_split, bt.n);
+            if (c->kv_f32) attn_hd<float>(s.head_dim, a, bt, g, st); else attn_hd<__nv_bfloat16>(s.head_dim, a, bt, g, st);
+            count_launch(c);
+        }
+        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.obuf, qw, NORM_NONE, nullptr, nullptr, 0.f, hi, lo);
+        count_launch(c);
+        if ((rc = pf_gemm(c, P, L.wo, d, qw, T, L.bo, xin_l, TG_NONE, x_out, st)) != MDI_OK) return rc;
+        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(x_out, d, norm, L.ln2g, L.ln2b, s.norm_eps, hi, lo);
+        count_launch(c);
+        if (s.act == MDI_ACT_SWIGLU) {
+            if ((rc = pf_gemm(c, P, L.wgate, F, d, T, nullptr, nullptr, TG_NONE, P.pf_h, st)) != MDI_OK) return rc;
+            if ((rc = pf_gemm(c, P, L.wup, F, d, T, nullptr, nullptr, TG_NONE, P.pf_u, st)) != MDI_OK) return rc;
+            k_pf_swiglu_split<<<T, 256, 0, st>>>(P.pf_h, P.pf_u, F, hi, lo);
+            count_launch(c);
+            if ((rc = pf_gemm(c, P, L.wdown, d, F, T, nullptr, x_out, TG_NONE, x_out, st)) != MDI_OK) return rc;
+        } else {
+            if ((rc = pf_gemm(c, P, L.w1, F, d, T, L.b1, nullptr, s.act == MDI_ACT_GELU_ERF ? TG_GELU_ERF : TG_GELU_TANH, P.pf_h, st)) != MDI_OK)
+                return rc;
+            k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo);
+            count_launch(c);
+            if ((rc = pf_gemm(c, P, L.w2, d, F, T, L.b2, x_out, TG_NONE, x_out, st)) != MDI_OK) return rc;
+        }
+    }
+    k_bt_advance<<<1, 32, 0, st>>>(P.pos_dev, bt);
+    count_launch(c);
     return MDI_OK;
 }
 

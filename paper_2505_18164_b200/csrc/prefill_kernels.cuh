@@ -146,6 +146,33 @@ __global__ void __launch_bounds__(ATT_THREADS) k_pf_attn(const float *q, float *
     }
 }
 
+// The same for a batch of items of different slots (a group's decode step): item i sits at pos[slot_i] + off_i.
+// grid (n items)
+template <typename KT>
+__global__ void k_bt_rope_append(const float *qkv, int q_rows, int kv_rows, int hd, int rope, const float *rope_cos,
+                                 const float *rope_sin, KvView kv, int layer_local, const int *pos, Batch bt, float *q_out) {
+    const int t = blockIdx.x, slot = bt.slot[t], p = pos[slot] + bt.off[t], half = hd >> 1, rows = q_rows + 2 * kv_rows;
+    const float *src = qkv + (size_t)t * rows;
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+        float y = src[r];
+        if (rope && r < q_rows + kv_rows) {
+            const int e = r % hd, i = e % half;
+            const float c = rope_cos[(size_t)p * half + i], s = rope_sin[(size_t)p * half + i];
+            y = e < half ? y * c - src[r + half] * s : y * c + src[r - half] * s;
+        }
+        if (r < q_rows) q_out[(size_t)t * q_rows + r] = y;
+        else {
+            const int rk = r - q_rows, which = rk >= kv_rows, rl = rk - which * kv_rows;
+            kv_store<KT>(kv_addr<KT>(kv, slot, layer_local, which, rl / hd, p, rl % hd), y);
+        }
+    }
+}
+
+__global__ void k_bt_advance(int *pos, Batch bt) {
+    const int i = threadIdx.x;
+    if (blockIdx.x == 0 && i < bt.n && bt.adv[i]) pos[bt.slot[i]] += bt.adv[i];
+}
+
 __global__ void k_pf_advance(int *pos, int slot, int by) {
     if (threadIdx.x == 0 && blockIdx.x == 0) pos[slot] += by;
 }

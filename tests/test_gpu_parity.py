@@ -71,6 +71,7 @@ CASES = [
     ("llama", I.DT_BF16, 4, 64, 4, None, 101, 64, [0, 2, 3, 4], 3, 6, 20, dict(page_tokens=4, attn_splits=2, kv_cache_bf16=1)),
     ("llama", I.DT_F32, 2, 128, 4, 2, 67, 48, [0, 1, 2], 4, 11, 14, dict(attn_splits=3)),
     ("llama", I.DT_BF16, 2, 256, 2, 1, 300, 40, [0, 2], 11, 3, 10, {}),         # one partition, group > 8 items
+    ("llama", I.DT_BF16, 2, 256, 2, 1, 300, 40, [0, 2], 11, 3, 10, dict(prefill_mode=1)),   # the same on the CUDA-core kernels
     ("llama", I.DT_BF16, 2, 256, 2, 1, 300, 200, [0, 1, 2], 2, 150, 6, {}),     # prompt longer than one prefill chunk
     ("llama", I.DT_BF16, 2, 256, 2, 1, 300, 40, [0, 2], 3, 9, 6, dict(prefill_mode=1)),
     ("gpt", I.DT_F32, 2, 64, 4, None, 50, 32, [0, 1, 2], 3, 10, 22, {}),        # prompt + new == n_ctx exactly
