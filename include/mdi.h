@@ -75,6 +75,9 @@ typedef struct {
     int prefill_mode;  /* first visits (whole prompt): 0 (default) tensor-core GEMMs (tcgen05, bf16 x bf16 -> fp32, inputs split
                           into two bf16 planes) when the weights are bf16, else the CUDA-core step kernels in chunks of 8
                           positions; 1: always the CUDA-core kernels */
+    int tc_min_group;  /* decode steps of groups with at least this many samples run their linear layers as tensor-core
+                          GEMMs (bf16 weights, prefill_mode 0; such calls use the stream scheduler).  0 (default): 5,
+                          or 1 when the matrices of one block hold 48 MB or more */
     int scheduler;     /* how mdi_generate runs the recurrent pipeline.  0: the persistent kernel (one launch,
                           one team of thread blocks per partition, flag handoff between teams) when the shape
                           fits it (groups of at most 4 samples), else the stream scheduler; 1: always the

@@ -109,6 +109,7 @@ struct mdi_ctx {
     int64_t cap_launches = 0, cap_steps = 0;
     // tensor-core first visit
     bool pf_tc = false;
+    int tc_min_group = 5; // groups with at least this many samples run their linear layers on the tensor cores
     int *tg_err = nullptr;
     std::map<std::tuple<const void *, uint64_t, uint64_t, uint32_t>, CUtensorMap> tmaps;
     // persistent decode kernel
@@ -310,7 +311,7 @@ int enqueue_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in
     }
     const KvView kv = kv_view(c, P);
     // groups of more than 4 items with bf16 weights: the linear layers run on the tensor cores
-    const bool tc = c->pf_tc && bt.n > 4;
+    const bool tc = c->pf_tc && bt.n >= c->tc_min_group;
     if (tc) {
         const int rc = tc_partition_step(c, p, bt, x_in, x_out, st);
         if (rc != MDI_OK) return rc;
@@ -377,6 +378,14 @@ constexpr int PF_CHUNK = 128; // positions per pass through a partition (one til
 int pf_setup(mdi_ctx *c) {
     const mdi_model_shape &s = c->s;
     c->pf_tc = s.weight_dtype == MDI_DTYPE_BF16 && c->o.prefill_mode != 1;
+    // Which decode steps use the tensor-core linear layers (stream scheduler): by default groups of 5 or more
+    // samples, and every group when one block's matrices are 48 MB or more (then a step moves enough bytes per
+    // kernel for launches not to matter, and TMA-fed GEMM tiles stream faster than the CUDA-core tiles).
+    {
+        const int d = s.d_model, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim;
+        const double layer_bytes = 2.0 * ((double)(qw + 2 * kw) * d + (double)d * qw + (double)(s.act == MDI_ACT_SWIGLU ? 3 : 2) * s.d_ff * d);
+        c->tc_min_group = c->o.tc_min_group > 0 ? c->o.tc_min_group : (layer_bytes >= 48e6 ? 1 : 5);
+    }
     if (!c->pf_tc) return MDI_OK;
     CU(cudaFuncSetAttribute(k_tc_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TG_SMEM));
     const int d = s.d_model, F = s.d_ff, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim;
@@ -1251,7 +1260,8 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
     const long total = (long)n_pass * K;        // phase slots per partition
     const long t_total = total ? total + K - 1 : 0;
     long t = 0;
-    const bool use_pk = c->pk_ok && c->scheduler != 1 && (n_samples + G - 1) / G <= PK_MAXNB;
+    const bool use_pk = c->pk_ok && c->scheduler != 1 && (n_samples + G - 1) / G <= PK_MAXNB &&
+                        !(c->pf_tc && (n_samples + G - 1) / G >= c->tc_min_group);
     if (c->scheduler == 2 && !use_pk) return fail(c, MDI_ERR_SHAPE, "persistent scheduler unavailable for this call");
     if (t_total && use_pk) {
         if ((rc = pk_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;

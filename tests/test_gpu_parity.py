@@ -76,8 +76,10 @@ CASES = [
     ("llama", I.DT_BF16, 2, 256, 2, 1, 300, 40, [0, 2], 3, 9, 6, dict(prefill_mode=1)),
     ("gpt", I.DT_F32, 2, 64, 4, None, 50, 32, [0, 1, 2], 3, 10, 22, {}),        # prompt + new == n_ctx exactly
     ("gpt", I.DT_BF16, 4, 64, 2, None, 97, 64, [0, 1, 2, 3, 4], 1, 4, 9, {}),   # one sample, four partitions
+    ("gpt", I.DT_BF16, 3, 128, 2, None, 131, 96, [0, 1, 2, 3], 5, 6, 12, dict(tc_min_group=1, attn_splits=2)),  # small groups on tensor cores
     ("gpt", I.DT_BF16, 2, 256, 4, None, 2100, 48, [0, 1, 2], 4, 5, 8, {}),      # d_ff 1024+: several tiles per warp, 2 per group
     ("gpt", I.DT_BF16, 4, 64, 2, None, 97, 64, [0, 1, 2, 3, 4], 1, 4, 9, {}),   # one sample, four partitions
+    ("gpt", I.DT_BF16, 3, 128, 2, None, 131, 96, [0, 1, 2, 3], 5, 6, 12, dict(tc_min_group=1, attn_splits=2)),  # small groups on tensor cores
 ]
 
 
