@@ -65,7 +65,8 @@ struct Partition {
     cudaEvent_t ev_join = nullptr, ev_join_cap = nullptr;
     // tensor-core first visit: inputs as bf16 hi/lo planes, fp32 intermediates, for up to PF_CHUNK positions
     uint16_t *pf_hi = nullptr, *pf_lo = nullptr;
-    float *pf_qkv = nullptr, *pf_q = nullptr, *pf_o = nullptr, *pf_h = nullptr, *pf_u = nullptr, *pf_xa = nullptr, *pf_xb = nullptr;
+    float *pf_qkv = nullptr, *pf_q = nullptr, *pf_o = nullptr, *pf_h = nullptr, *pf_u = nullptr, *pf_xa = nullptr, *pf_xb = nullptr,
+          *pf_part = nullptr; // split-K partial sums [PF_SPLIT_MAX][PF_CHUNK][d_model]
     int64_t weight_bytes = 0, buffer_bytes = 0;
 };
 
@@ -374,6 +375,7 @@ int enqueue_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in
 
 // ---- first visit on tensor cores (bf16 weights): GEMMs of tc_gemm.cuh + helpers of prefill_kernels.cuh ----
 constexpr int PF_CHUNK = 128; // positions per pass through a partition (one tile of positions per GEMM block)
+constexpr int PF_SPLIT_MAX = 8; // K splits of the GEMMs with few row tiles (output projection, MLP down)
 
 int pf_setup(mdi_ctx *c) {
     const mdi_model_shape &s = c->s;
@@ -402,6 +404,7 @@ int pf_setup(mdi_ctx *c) {
         if (s.act == MDI_ACT_SWIGLU && (rc = dalloc(c, &P.pf_u, (size_t)PF_CHUNK * F, &P.buffer_bytes)) != MDI_OK) return rc;
         if ((rc = dalloc(c, &P.pf_xa, (size_t)PF_CHUNK * d, &P.buffer_bytes)) != MDI_OK) return rc;
         if ((rc = dalloc(c, &P.pf_xb, (size_t)PF_CHUNK * d, &P.buffer_bytes)) != MDI_OK) return rc;
+        if ((rc = dalloc(c, &P.pf_part, (size_t)PF_SPLIT_MAX * PF_CHUNK * d, &P.buffer_bytes)) != MDI_OK) return rc;
     }
     return MDI_OK;
 }
@@ -430,11 +433,20 @@ int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, c
     if ((rc = pf_map(c, W, (uint64_t)n_rows, (uint64_t)K, TG_BM, &mw)) != MDI_OK) return rc;
     if ((rc = pf_map(c, P.pf_hi, PF_CHUNK, (uint64_t)K, (uint32_t)n_tile, &mhi)) != MDI_OK) return rc;
     if ((rc = pf_map(c, P.pf_lo, PF_CHUNK, (uint64_t)K, (uint32_t)n_tile, &mlo)) != MDI_OK) return rc;
+    // matrices with few 128-row tiles (d_model outputs) would leave most SMs idle: split the reduction over
+    // several blocks and add the partial sums up in a fixed order afterwards
+    const int grid_x = (n_rows + TG_BM - 1) / TG_BM, n_kb = (K + TG_BK - 1) / TG_BK;
+    int splits = 1;
+    if (n_rows == c->s.d_model && grid_x < 32) splits = std::max(1, std::min(std::min(PF_SPLIT_MAX, c->n_sm / grid_x), n_kb / 8));
     TgArgs a{};
     a.n_rows = n_rows; a.K = K; a.T = T; a.n_tile = n_tile; a.bias = bias; a.resid = resid; a.act = act; a.y = y; a.ldy = n_rows;
-    a.err = c->tg_err;
-    k_tc_gemm<<<dim3((n_rows + TG_BM - 1) / TG_BM, (T + n_tile - 1) / n_tile), TG_THREADS, TG_SMEM, st>>>(*mw, *mhi, *mlo, a);
+    a.err = c->tg_err; a.partial = P.pf_part;
+    k_tc_gemm<<<dim3(grid_x, (T + n_tile - 1) / n_tile, splits), TG_THREADS, TG_SMEM, st>>>(*mw, *mhi, *mlo, a);
     count_launch(c);
+    if (splits > 1) {
+        k_pf_reduce<<<T, 256, 0, st>>>(P.pf_part, splits, T, n_rows, bias, resid, y);
+        count_launch(c);
+    }
     return MDI_OK;
 }
 
@@ -829,7 +841,7 @@ void mdi_destroy(mdi_ctx *c) {
     }
     for (auto &P : c->part) {
         void *ptrs[] = {P.kv_pool, P.pt_dev, P.pos_dev, P.x_embed, P.qbuf, P.obuf, P.hbuf, P.part, P.x_last, P.attn_ticket,
-                        P.ring, P.pf_buf[0], P.pf_buf[1], P.pf_hi, P.pf_lo, P.pf_qkv, P.pf_q, P.pf_o, P.pf_h, P.pf_u, P.pf_xa, P.pf_xb};
+                        P.ring, P.pf_buf[0], P.pf_buf[1], P.pf_hi, P.pf_lo, P.pf_qkv, P.pf_q, P.pf_o, P.pf_h, P.pf_u, P.pf_xa, P.pf_xb, P.pf_part};
         for (void *q : ptrs) if (q) cudaFree(q);
         for (auto e : P.ev_edge) cudaEventDestroy(e);
         for (auto e : P.ev_edge_cap) cudaEventDestroy(e);

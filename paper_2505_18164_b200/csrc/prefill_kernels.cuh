@@ -168,6 +168,17 @@ __global__ void k_bt_rope_append(const float *qkv, int q_rows, int kv_rows, int 
     }
 }
 
+// y[t][i] = sum_z partial[z][t][i] + bias[i] + resid[t][i]  (fixed summation order).  grid (T)
+__global__ void k_pf_reduce(const float *partial, int n_split, int T, int n, const float *bias, const float *resid, float *y) {
+    const int t = blockIdx.x;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        float v = bias ? bias[i] : 0.f;
+        if (resid) v += resid[(size_t)t * n + i];
+        for (int z = 0; z < n_split; ++z) v += partial[((size_t)z * T + t) * n + i];
+        y[(size_t)t * n + i] = v;
+    }
+}
+
 __global__ void k_bt_advance(int *pos, Batch bt) {
     const int i = threadIdx.x;
     if (blockIdx.x == 0 && i < bt.n && bt.adv[i]) pos[bt.slot[i]] += bt.adv[i];

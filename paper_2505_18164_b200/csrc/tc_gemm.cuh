@@ -4,7 +4,8 @@
 //     X = hi + lo to ~16 mantissa bits, accumulation in fp32.
 // The weight tile (128 rows) is the M operand of tcgen05.mma, the positions are the N operand, the
 // fp32 accumulator D[128 x n_tile] lives in tensor memory.  One block = one 128-row tile x one tile of
-// positions; operands arrive by TMA (128-byte swizzle, no multicast) through a 4-stage mbarrier ring.
+// positions; operands arrive by TMA (128-byte swizzle, no multicast) through an mbarrier ring of 4 to 9 stages
+// (as many as fit in 192 KB for the tile of positions).
 // Warp 0 lane 0 issues TMA, warp 1 lane 0 issues MMAs (and warp 1 owns the TMEM allocation), warps 2..5
 // read the accumulator back (tcgen05.ld, one TMEM lane = one weight row per thread) and store Y.
 // Every wait is bounded in wall time; on a timeout an error word is set, the block skips the remaining
@@ -19,13 +20,18 @@ namespace mdi {
 
 constexpr int TG_BM = 128;      // weight rows per block (MMA M)
 constexpr int TG_BK = 64;       // reduction elements per stage: 128 bytes, one swizzle atom
-constexpr int TG_STAGES = 4;
+constexpr int TG_MAX_STAGES = 10;
 constexpr int TG_MAX_NT = 128;  // positions per block (MMA N), a multiple of 16
 constexpr int TG_THREADS = 192;
-constexpr int TG_W_BYTES = TG_BM * TG_BK * 2;          // 16 KB
-constexpr int TG_X_BYTES = TG_MAX_NT * TG_BK * 2;      // 16 KB (hi) + 16 KB (lo)
-constexpr int TG_STAGE_BYTES = TG_W_BYTES + 2 * TG_X_BYTES;
-constexpr size_t TG_SMEM = (size_t)TG_STAGES * TG_STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int TG_W_BYTES = TG_BM * TG_BK * 2;          // 16 KB per stage
+constexpr int TG_RING_BYTES = 196608;                  // operand ring: as many stages as fit (4 at 128 positions, 9 at 16)
+constexpr size_t TG_SMEM = (size_t)TG_RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+// bytes of one stage: a 128 x 64 weight tile and two n_tile x 64 input tiles (hi, lo); every part 1024-byte aligned
+__host__ __device__ inline int tg_stage_bytes(int n_tile) { return TG_W_BYTES + 2 * n_tile * TG_BK * 2; }
+__host__ __device__ inline int tg_stages(int n_tile) {
+    const int n = TG_RING_BYTES / tg_stage_bytes(n_tile);
+    return n < TG_MAX_STAGES ? n : TG_MAX_STAGES;
+}
 constexpr unsigned long long TG_WAIT_NS = 2000000000ull;
 
 enum TgAct { TG_NONE = 0, TG_GELU_TANH = 1, TG_GELU_ERF = 2 };
@@ -38,6 +44,7 @@ struct TgArgs {
     float *y;                 // [T][ldy]
     int ldy;
     int *err;                 // set to 1 when a wait gave up
+    float *partial;           // split-K (gridDim.z > 1): raw partial sums [z][T][ldy]; bias/resid/act/y are then unused
 };
 
 __device__ __forceinline__ uint32_t tg_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -102,19 +109,21 @@ __device__ __forceinline__ float tg_apply(float v, int act) {
     return v;
 }
 
-// grid (ceil(n_rows / 128), ceil(T / n_tile))
+// grid (ceil(n_rows / 128), ceil(T / n_tile), K splits)
 __global__ void __launch_bounds__(TG_THREADS, 1)
 k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_xhi,
           const __grid_constant__ CUtensorMap tm_xlo, const TgArgs a) {
     extern __shared__ unsigned char tg_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)tg_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)TG_STAGES * TG_STAGE_BYTES);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)TG_RING_BYTES);
     // bars[0..S): full, bars[S..2S): empty, bars[2S]: accumulator ready; then the TMEM base address
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * TG_STAGES + 1);
+    const int TG_STAGES = tg_stages(a.n_tile), TG_STAGE_BYTES = tg_stage_bytes(a.n_tile), TG_X_BYTES = a.n_tile * TG_BK * 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * TG_MAX_STAGES + 1);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m0 = blockIdx.x * TG_BM, t0 = blockIdx.y * a.n_tile;
-    const int n_kb = (a.K + TG_BK - 1) / TG_BK;
-    const uint32_t full0 = tg_smem_u32(bars), empty0 = tg_smem_u32(bars + TG_STAGES), accbar = tg_smem_u32(bars + 2 * TG_STAGES);
+    const int n_kb_all = (a.K + TG_BK - 1) / TG_BK;
+    const int kb_lo = (int)((long)blockIdx.z * n_kb_all / gridDim.z), n_kb = (int)((long)(blockIdx.z + 1) * n_kb_all / gridDim.z) - kb_lo;
+    const uint32_t full0 = tg_smem_u32(bars), empty0 = tg_smem_u32(bars + TG_MAX_STAGES), accbar = tg_smem_u32(bars + 2 * TG_MAX_STAGES);
     const uint32_t tmem_cols = a.n_tile <= 32 ? 32u : a.n_tile <= 64 ? 64u : 128u;
 
     if (tid == 0) {
@@ -137,7 +146,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     if (warp == 0) {
         if (lane == 0) {
             // ---- TMA producer
-            const uint32_t stage_bytes = (uint32_t)TG_W_BYTES + 2u * (uint32_t)a.n_tile * TG_BK * 2u;
+            const uint32_t stage_bytes = (uint32_t)TG_STAGE_BYTES;
             bool ok = true;
             for (int kb = 0; kb < n_kb && ok; ++kb) {
                 const int s = kb % TG_STAGES;
@@ -146,9 +155,9 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 const uint32_t full = full0 + 8 * s;
                 const uint32_t base = tg_smem_u32(smem + (size_t)s * TG_STAGE_BYTES);
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full), "r"(stage_bytes) : "memory");
-                tg_tma_2d(base, &tm_w, kb * TG_BK, m0, full);
-                tg_tma_2d(base + TG_W_BYTES, &tm_xhi, kb * TG_BK, t0, full);
-                tg_tma_2d(base + TG_W_BYTES + TG_X_BYTES, &tm_xlo, kb * TG_BK, t0, full);
+                tg_tma_2d(base, &tm_w, (kb_lo + kb) * TG_BK, m0, full);
+                tg_tma_2d(base + TG_W_BYTES, &tm_xhi, (kb_lo + kb) * TG_BK, t0, full);
+                tg_tma_2d(base + TG_W_BYTES + TG_X_BYTES, &tm_xlo, (kb_lo + kb) * TG_BK, t0, full);
             }
         }
     } else if (warp == 1) {
@@ -192,7 +201,9 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int t = t0 + c + j;
-                        if (t < a.T) {
+                        if (t < a.T && gridDim.z > 1) {
+                            a.partial[((size_t)blockIdx.z * a.T + t) * a.ldy + row] = __uint_as_float(r[j]);
+                        } else if (t < a.T) {
                             float v = __uint_as_float(r[j]) + bias;
                             if (a.resid) v += a.resid[(size_t)t * a.ldy + row];
                             a.y[(size_t)t * a.ldy + row] = tg_apply(v, a.act);
