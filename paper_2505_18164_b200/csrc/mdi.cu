@@ -1356,7 +1356,7 @@ int mdi_sync(mdi_ctx *c) {
     CU(cudaSetDevice(c->dev));
     for (auto &P : c->part) CU(cudaStreamSynchronize(P.stream));
     CU(cudaStreamSynchronize(c->main));
-    return MDI_OK;
+    return pf_check(c);
 }
 
 int mdi_get_stats(mdi_ctx *c, mdi_stats *out) {
