@@ -441,7 +441,7 @@ int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, c
     TgArgs a{};
     a.n_rows = n_rows; a.K = K; a.T = T; a.n_tile = n_tile; a.bias = bias; a.resid = resid; a.act = act; a.y = y; a.ldy = n_rows;
     a.err = c->tg_err; a.partial = P.pf_part;
-    k_tc_gemm<<<dim3(grid_x, (T + n_tile - 1) / n_tile, splits), TG_THREADS, TG_SMEM, st>>>(*mw, *mhi, *mlo, a);
+    k_tc_gemm<<<dim3(grid_x, (T + n_tile - 1) / n_tile, splits), TG_THREADS, tg_smem_bytes(n_tile), st>>>(*mw, *mhi, *mlo, a);
     count_launch(c);
     if (splits > 1) {
         k_pf_reduce<<<T, 256, 0, st>>>(P.pf_part, splits, T, n_rows, bias, resid, y);

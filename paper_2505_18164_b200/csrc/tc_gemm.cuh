@@ -24,12 +24,16 @@ constexpr int TG_MAX_STAGES = 10;
 constexpr int TG_MAX_NT = 128;  // positions per block (MMA N), a multiple of 16
 constexpr int TG_THREADS = 192;
 constexpr int TG_W_BYTES = TG_BM * TG_BK * 2;          // 16 KB per stage
-constexpr int TG_RING_BYTES = 196608;                  // operand ring: as many stages as fit (4 at 128 positions, 9 at 16)
+constexpr int TG_RING_BYTES = 196608;                  // operand ring for tiles of 64 or 128 positions (4 stages at 128)
+constexpr int TG_RING_BYTES_SMALL = 98304;             // for tiles of 16 or 32 positions (4 stages): two blocks fit on one SM,
+                                                       // so GEMMs launched on different streams share SMs and overlap
 constexpr size_t TG_SMEM = (size_t)TG_RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+__host__ __device__ inline int tg_ring_bytes(int n_tile) { return n_tile <= 32 ? TG_RING_BYTES_SMALL : TG_RING_BYTES; }
+__host__ __device__ inline size_t tg_smem_bytes(int n_tile) { return (size_t)tg_ring_bytes(n_tile) + 1024 + 256; }
 // bytes of one stage: a 128 x 64 weight tile and two n_tile x 64 input tiles (hi, lo); every part 1024-byte aligned
 __host__ __device__ inline int tg_stage_bytes(int n_tile) { return TG_W_BYTES + 2 * n_tile * TG_BK * 2; }
 __host__ __device__ inline int tg_stages(int n_tile) {
-    const int n = TG_RING_BYTES / tg_stage_bytes(n_tile);
+    const int n = tg_ring_bytes(n_tile) / tg_stage_bytes(n_tile);
     return n < TG_MAX_STAGES ? n : TG_MAX_STAGES;
 }
 constexpr unsigned long long TG_WAIT_NS = 2000000000ull;
@@ -110,12 +114,12 @@ __device__ __forceinline__ float tg_apply(float v, int act) {
 }
 
 // grid (ceil(n_rows / 128), ceil(T / n_tile), K splits)
-__global__ void __launch_bounds__(TG_THREADS, 1)
+__global__ void __launch_bounds__(TG_THREADS)
 k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_xhi,
           const __grid_constant__ CUtensorMap tm_xlo, const TgArgs a) {
     extern __shared__ unsigned char tg_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)tg_raw + 1023) & ~(uintptr_t)1023);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)TG_RING_BYTES);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)tg_ring_bytes(a.n_tile));
     // bars[0..S): full, bars[S..2S): empty, bars[2S]: accumulator ready; then the TMEM base address
     const int TG_STAGES = tg_stages(a.n_tile), TG_STAGE_BYTES = tg_stage_bytes(a.n_tile), TG_X_BYTES = a.n_tile * TG_BK * 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * TG_MAX_STAGES + 1);
