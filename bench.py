@@ -192,6 +192,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--rounds-per-graph", type=int, default=0)
     ap.add_argument("--scheduler", type=int, default=0, help="0 auto (persistent kernel when it fits), 1 streams, 2 persistent")
+    ap.add_argument("--tc-min-group", type=int, default=0, help="smallest group whose decode steps run on the tensor cores (0 = library default)")
     ap.add_argument("--n-new", type=int, default=0, help="shorter generation (profiler captures only; not the headline)")
     ap.add_argument("--n-prompt", type=int, default=0, help="shorter prompts (profiler captures only)")
     args = ap.parse_args()
@@ -221,7 +222,7 @@ def main():
     s = w.shape
     S, P, N = w.n_samples, w.n_prompt, w.n_new
     ctx = mdi.Context(s, list(w.part_bounds), S, kv_pool_tokens=S * ((P + N + 15) // 16 * 16), rounds_per_graph=args.rounds_per_graph,
-                      scheduler=args.scheduler)
+                      scheduler=args.scheduler, tc_min_group=args.tc_min_group)
     weights = {}
     for name, a in I.iter_weights(s, w.weight_seed):
         ctx.load_weights(name, a)
