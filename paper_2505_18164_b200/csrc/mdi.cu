@@ -424,154 +424,141 @@ int pf_map(mdi_ctx *c, const void *base, uint64_t rows, uint64_t cols, uint32_t 
     return MDI_OK;
 }
 
+// A split-K GEMM leaves partial sums behind; they are added up (with bias and residual) by the next norm kernel.
+struct PfPending {
+    int splits = 0;
+    const float *bias = nullptr, *resid = nullptr;
+};
+
 // y[t][r] = act(W[r][:] . x[t][:] + bias[r] + resid[t][r]) for T positions whose inputs sit in P.pf_hi / P.pf_lo.
+// y may be null when only the bf16 planes out_hi / out_lo are wanted.  When the matrix has few 128-row tiles the
+// reduction is split over several blocks: then nothing is written but P.pf_part, and *pending says what is left
+// to add (pending must be non-null for matrices with d_model rows).
 int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, const float *bias, const float *resid, int act,
-            float *y, cudaStream_t st) {
+            float *y, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, PfPending *pending, cudaStream_t st) {
     const int n_tile = T <= 16 ? 16 : T <= 32 ? 32 : T <= 64 ? 64 : 128;
     const CUtensorMap *mw, *mhi, *mlo;
     int rc;
     if ((rc = pf_map(c, W, (uint64_t)n_rows, (uint64_t)K, TG_BM, &mw)) != MDI_OK) return rc;
     if ((rc = pf_map(c, P.pf_hi, PF_CHUNK, (uint64_t)K, (uint32_t)n_tile, &mhi)) != MDI_OK) return rc;
     if ((rc = pf_map(c, P.pf_lo, PF_CHUNK, (uint64_t)K, (uint32_t)n_tile, &mlo)) != MDI_OK) return rc;
-    // matrices with few 128-row tiles (d_model outputs) would leave most SMs idle: split the reduction over
-    // several blocks and add the partial sums up in a fixed order afterwards
     const int grid_x = (n_rows + TG_BM - 1) / TG_BM, n_kb = (K + TG_BK - 1) / TG_BK;
     int splits = 1;
-    if (n_rows == c->s.d_model && grid_x < 32) splits = std::max(1, std::min(std::min(PF_SPLIT_MAX, c->n_sm / grid_x), n_kb / 8));
+    if (pending && grid_x < 32) splits = std::max(1, std::min(std::min(PF_SPLIT_MAX, c->n_sm / grid_x), n_kb / 8));
     TgArgs a{};
     a.n_rows = n_rows; a.K = K; a.T = T; a.n_tile = n_tile; a.bias = bias; a.resid = resid; a.act = act; a.y = y; a.ldy = n_rows;
-    a.err = c->tg_err; a.partial = P.pf_part;
+    a.err = c->tg_err; a.partial = P.pf_part; a.out_hi = out_hi; a.out_lo = out_lo;
     k_tc_gemm<<<dim3(grid_x, (T + n_tile - 1) / n_tile, splits), TG_THREADS, tg_smem_bytes(n_tile), st>>>(*mw, *mhi, *mlo, a);
     count_launch(c);
-    if (splits > 1) {
-        k_pf_reduce<<<T, 256, 0, st>>>(P.pf_part, splits, T, n_rows, bias, resid, y);
-        count_launch(c);
+    if (pending) {
+        pending->splits = splits > 1 ? splits : 0;
+        pending->bias = bias;
+        pending->resid = resid;
     }
     return MDI_OK;
 }
 
-template <typename KT> void pf_attn_hd(int hd, dim3 g, cudaStream_t st, const float *q, float *o, const KvView &kv, int ll, int n_head,
-                                       const int *pos, int slot, float scale) {
+template <typename KT> void pf_attn_hd(int hd, dim3 g, cudaStream_t st, const float *q, __nv_bfloat16 *ohi, __nv_bfloat16 *olo,
+                                       const KvView &kv, int ll, int n_head, const int *pos, int slot, float scale) {
     switch (hd) {
-        case 16: k_pf_attn<KT, 16><<<g, ATT_THREADS, 0, st>>>(q, o, kv, ll, n_head, pos, slot, scale); break;
-        case 32: k_pf_attn<KT, 32><<<g, ATT_THREADS, 0, st>>>(q, o, kv, ll, n_head, pos, slot, scale); break;
-        case 64: k_pf_attn<KT, 64><<<g, ATT_THREADS, 0, st>>>(q, o, kv, ll, n_head, pos, slot, scale); break;
-        default: k_pf_attn<KT, 128><<<g, ATT_THREADS, 0, st>>>(q, o, kv, ll, n_head, pos, slot, scale); break;
+        case 16: k_pf_attn<KT, 16><<<g, ATT_THREADS, 0, st>>>(q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        case 32: k_pf_attn<KT, 32><<<g, ATT_THREADS, 0, st>>>(q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        case 64: k_pf_attn<KT, 64><<<g, ATT_THREADS, 0, st>>>(q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        default: k_pf_attn<KT, 128><<<g, ATT_THREADS, 0, st>>>(q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
     }
 }
 
-// T (<= PF_CHUNK) new positions of one slot through partition p.  x_in: [T][d] (ignored for p == 0, which embeds
-// tok_dev[0..T)); x_out: [T][d].  Cache rows pos .. pos+T-1 are written and pos advances by T at the end.
-int pf_partition_chunk(mdi_ctx *c, int p, int slot, const int *tok_dev, int T, const float *x_in, float *x_out, cudaStream_t st) {
+// The blocks of partition p on T rows with the linear layers on the tensor cores.  Two uses:
+//  - first visit (bt == null): T (<= PF_CHUNK) consecutive new positions of `slot`; partition 0 embeds tok_dev[0..T);
+//  - a group's decode step (bt != null): T = bt->n items of different slots, one new position each.
+// x_in: [T][d] (ignored for partition 0 of a first visit); x_out: [T][d].  Cache rows are appended and the
+// positions advanced at the end.  Per block: norm+split, QKV GEMM, rotary+append, attention (writes bf16 planes),
+// output-projection GEMM, norm+split (adds up split-K partials), MLP up GEMM (writes bf16 planes), MLP down GEMM.
+int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, int T, const float *x_in, float *x_out, cudaStream_t st) {
     Partition &P = c->part[p];
     const mdi_model_shape &s = c->s;
     const int d = s.d_model, F = s.d_ff, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim;
-    const int norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS;
+    const int norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS, rope = s.arch == MDI_ARCH_LLAMA;
     const KvView kv = kv_view(c, P);
     const float scale = 1.0f / std::sqrt((float)s.head_dim);
     __nv_bfloat16 *hi = (__nv_bfloat16 *)P.pf_hi, *lo = (__nv_bfloat16 *)P.pf_lo;
     int rc;
-    if (p == 0) {
+    if (!bt && p == 0) {
         k_pf_embed<__nv_bfloat16><<<T, 256, 0, st>>>((const __nv_bfloat16 *)c->wte, (const __nv_bfloat16 *)c->wpe, d, s.vocab, tok_dev,
                                                     P.pos_dev, slot, P.pf_xa);
         count_launch(c);
         x_in = P.pf_xa;
     }
+    PfPending pend; // partial sums of the previous block's MLP-down GEMM, not yet added into x_out
     for (int l = P.lo; l < P.hi; ++l) {
         const LayerW &L = c->layer[l];
+        const int ll = l - P.lo;
         const float *xin_l = l == P.lo ? x_in : x_out;
-        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(xin_l, d, norm, L.ln1g, L.ln1b, s.norm_eps, hi, lo);
+        // norm 1 (first completing the residual stream if the previous GEMM was split)
+        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(pend.splits ? pend.resid : xin_l, d, norm, L.ln1g, L.ln1b, s.norm_eps, hi, lo, P.pf_part,
+                                                  pend.splits, T, pend.bias, x_out);
         count_launch(c);
-        if ((rc = pf_gemm(c, P, L.wqkv, qw + 2 * kw, d, T, L.bqkv, nullptr, TG_NONE, P.pf_qkv, st)) != MDI_OK) return rc;
-        if (c->kv_f32)
-            k_pf_rope_append<float><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, s.arch == MDI_ARCH_LLAMA, c->rope_cos, c->rope_sin, kv,
-                                                       l - P.lo, P.pos_dev, slot, P.pf_q);
-        else
-            k_pf_rope_append<__nv_bfloat16><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, s.arch == MDI_ARCH_LLAMA, c->rope_cos,
-                                                               c->rope_sin, kv, l - P.lo, P.pos_dev, slot, P.pf_q);
-        count_launch(c);
-        if (c->kv_f32) pf_attn_hd<float>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, P.pf_o, kv, l - P.lo, s.n_head, P.pos_dev, slot, scale);
-        else pf_attn_hd<__nv_bfloat16>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, P.pf_o, kv, l - P.lo, s.n_head, P.pos_dev, slot, scale);
-        count_launch(c);
-        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.pf_o, qw, NORM_NONE, nullptr, nullptr, 0.f, hi, lo);
-        count_launch(c);
-        if ((rc = pf_gemm(c, P, L.wo, d, qw, T, L.bo, xin_l, TG_NONE, x_out, st)) != MDI_OK) return rc;
-        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(x_out, d, norm, L.ln2g, L.ln2b, s.norm_eps, hi, lo);
+        pend = PfPending();
+        if ((rc = pf_gemm(c, P, L.wqkv, qw + 2 * kw, d, T, L.bqkv, nullptr, TG_NONE, P.pf_qkv, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
+        if (bt) {
+            if (c->kv_f32) k_bt_rope_append<float><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
+            else k_bt_rope_append<__nv_bfloat16><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
+            count_launch(c);
+            AttnArgs a{};
+            a.q = P.qbuf; a.o = P.obuf; a.part = P.part; a.ticket = P.attn_ticket; a.kv = kv; a.layer_local = ll; a.n_head = s.n_head;
+            a.n_split = c->n_split; a.pos = P.pos_dev; a.scale = scale; a.o_hi = hi; a.o_lo = lo;
+            const dim3 g(s.n_head, c->n_split, T);
+            if (c->kv_f32) attn_hd<float>(s.head_dim, a, *bt, g, st); else attn_hd<__nv_bfloat16>(s.head_dim, a, *bt, g, st);
+            count_launch(c);
+        } else {
+            if (c->kv_f32) k_pf_rope_append<float><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
+            else k_pf_rope_append<__nv_bfloat16><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
+            count_launch(c);
+            if (c->kv_f32) pf_attn_hd<float>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
+            else pf_attn_hd<__nv_bfloat16>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
+            count_launch(c);
+        }
+        // output projection + residual -> x_out (or partial sums, completed by the next kernel)
+        PfPending po;
+        if ((rc = pf_gemm(c, P, L.wo, d, qw, T, L.bo, xin_l, TG_NONE, x_out, nullptr, nullptr, &po, st)) != MDI_OK) return rc;
+        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(po.splits ? po.resid : x_out, d, norm, L.ln2g, L.ln2b, s.norm_eps, hi, lo, P.pf_part, po.splits, T,
+                                                  po.bias, x_out);
         count_launch(c);
         if (s.act == MDI_ACT_SWIGLU) {
-            if ((rc = pf_gemm(c, P, L.wgate, F, d, T, nullptr, nullptr, TG_NONE, P.pf_h, st)) != MDI_OK) return rc;
-            if ((rc = pf_gemm(c, P, L.wup, F, d, T, nullptr, nullptr, TG_NONE, P.pf_u, st)) != MDI_OK) return rc;
+            if ((rc = pf_gemm(c, P, L.wgate, F, d, T, nullptr, nullptr, TG_NONE, P.pf_h, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
+            if ((rc = pf_gemm(c, P, L.wup, F, d, T, nullptr, nullptr, TG_NONE, P.pf_u, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
             k_pf_swiglu_split<<<T, 256, 0, st>>>(P.pf_h, P.pf_u, F, hi, lo);
             count_launch(c);
-            if ((rc = pf_gemm(c, P, L.wdown, d, F, T, nullptr, x_out, TG_NONE, x_out, st)) != MDI_OK) return rc;
+            if ((rc = pf_gemm(c, P, L.wdown, d, F, T, nullptr, x_out, TG_NONE, x_out, nullptr, nullptr, &pend, st)) != MDI_OK) return rc;
         } else {
-            if ((rc = pf_gemm(c, P, L.w1, F, d, T, L.b1, nullptr, s.act == MDI_ACT_GELU_ERF ? TG_GELU_ERF : TG_GELU_TANH, P.pf_h, st)) != MDI_OK)
+            // the GEMM cannot write the planes it is still reading as its input: they go to the other half of the buffers
+            if ((rc = pf_gemm(c, P, L.w1, F, d, T, L.b1, nullptr, s.act == MDI_ACT_GELU_ERF ? TG_GELU_ERF : TG_GELU_TANH, P.pf_h, nullptr, nullptr,
+                              nullptr, st)) != MDI_OK)
                 return rc;
-            k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo);
+            k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo, nullptr, 0, T, nullptr, nullptr);
             count_launch(c);
-            if ((rc = pf_gemm(c, P, L.w2, d, F, T, L.b2, x_out, TG_NONE, x_out, st)) != MDI_OK) return rc;
+            if ((rc = pf_gemm(c, P, L.w2, d, F, T, L.b2, x_out, TG_NONE, x_out, nullptr, nullptr, &pend, st)) != MDI_OK) return rc;
         }
     }
-    k_pf_advance<<<1, 32, 0, st>>>(P.pos_dev, slot, T);
+    if (pend.splits) { // complete the residual stream after the last block
+        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(pend.resid, d, NORM_NONE, nullptr, nullptr, 0.f, nullptr, nullptr, P.pf_part, pend.splits, T,
+                                                  pend.bias, x_out);
+        count_launch(c);
+    }
+    if (bt) k_bt_advance<<<1, 32, 0, st>>>(P.pos_dev, *bt);
+    else k_pf_advance<<<1, 32, 0, st>>>(P.pos_dev, slot, T);
     count_launch(c);
-    ++c->st.stage_steps;
     return MDI_OK;
 }
 
-// A group's decode step (5..8 items of different slots, one new position each) with the linear layers on the
-// tensor cores: the weights of the partition are streamed once by TMA for the whole group.
+int pf_partition_chunk(mdi_ctx *c, int p, int slot, const int *tok_dev, int T, const float *x_in, float *x_out, cudaStream_t st) {
+    const int rc = tc_layers(c, p, nullptr, slot, tok_dev, T, x_in, x_out, st);
+    if (rc == MDI_OK) ++c->st.stage_steps;
+    return rc;
+}
+
 int tc_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in, float *x_out, cudaStream_t st) {
-    Partition &P = c->part[p];
-    const mdi_model_shape &s = c->s;
-    const int d = s.d_model, F = s.d_ff, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim, T = bt.n;
-    const int norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS;
-    const KvView kv = kv_view(c, P);
-    __nv_bfloat16 *hi = (__nv_bfloat16 *)P.pf_hi, *lo = (__nv_bfloat16 *)P.pf_lo;
-    int rc;
-    for (int l = P.lo; l < P.hi; ++l) {
-        const LayerW &L = c->layer[l];
-        const float *xin_l = l == P.lo ? x_in : x_out;
-        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(xin_l, d, norm, L.ln1g, L.ln1b, s.norm_eps, hi, lo);
-        count_launch(c);
-        if ((rc = pf_gemm(c, P, L.wqkv, qw + 2 * kw, d, T, L.bqkv, nullptr, TG_NONE, P.pf_qkv, st)) != MDI_OK) return rc;
-        if (c->kv_f32)
-            k_bt_rope_append<float><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, s.arch == MDI_ARCH_LLAMA, c->rope_cos, c->rope_sin, kv,
-                                                       l - P.lo, P.pos_dev, bt, P.qbuf);
-        else
-            k_bt_rope_append<__nv_bfloat16><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, s.arch == MDI_ARCH_LLAMA, c->rope_cos,
-                                                               c->rope_sin, kv, l - P.lo, P.pos_dev, bt, P.qbuf);
-        count_launch(c);
-        {
-            AttnArgs a{};
-            a.q = P.qbuf; a.o = P.obuf; a.part = P.part; a.ticket = P.attn_ticket; a.kv = kv;
-            a.layer_local = l - P.lo; a.n_head = s.n_head; a.n_split = c->n_split; a.pos = P.pos_dev;
-            a.scale = 1.0f / std::sqrt((float)s.head_dim);
-            dim3 g(s.n_head, c->n_split, bt.n);
-            if (c->kv_f32) attn_hd<float>(s.head_dim, a, bt, g, st); else attn_hd<__nv_bfloat16>(s.head_dim, a, bt, g, st);
-            count_launch(c);
-        }
-        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.obuf, qw, NORM_NONE, nullptr, nullptr, 0.f, hi, lo);
-        count_launch(c);
-        if ((rc = pf_gemm(c, P, L.wo, d, qw, T, L.bo, xin_l, TG_NONE, x_out, st)) != MDI_OK) return rc;
-        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(x_out, d, norm, L.ln2g, L.ln2b, s.norm_eps, hi, lo);
-        count_launch(c);
-        if (s.act == MDI_ACT_SWIGLU) {
-            if ((rc = pf_gemm(c, P, L.wgate, F, d, T, nullptr, nullptr, TG_NONE, P.pf_h, st)) != MDI_OK) return rc;
-            if ((rc = pf_gemm(c, P, L.wup, F, d, T, nullptr, nullptr, TG_NONE, P.pf_u, st)) != MDI_OK) return rc;
-            k_pf_swiglu_split<<<T, 256, 0, st>>>(P.pf_h, P.pf_u, F, hi, lo);
-            count_launch(c);
-            if ((rc = pf_gemm(c, P, L.wdown, d, F, T, nullptr, x_out, TG_NONE, x_out, st)) != MDI_OK) return rc;
-        } else {
-            if ((rc = pf_gemm(c, P, L.w1, F, d, T, L.b1, nullptr, s.act == MDI_ACT_GELU_ERF ? TG_GELU_ERF : TG_GELU_TANH, P.pf_h, st)) != MDI_OK)
-                return rc;
-            k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo);
-            count_launch(c);
-            if ((rc = pf_gemm(c, P, L.w2, d, F, T, L.b2, x_out, TG_NONE, x_out, st)) != MDI_OK) return rc;
-        }
-    }
-    k_bt_advance<<<1, 32, 0, st>>>(P.pos_dev, bt);
-    count_launch(c);
-    return MDI_OK;
+    return tc_layers(c, p, &bt, 0, nullptr, bt.n, x_in, x_out, st);
 }
 
 // Did a tensor-core first visit give up on one of its bounded waits?  (Synchronises the partition streams.)

@@ -28,12 +28,26 @@ __global__ void k_pf_embed(const WT *wte, const WT *wpe, int d, int vocab, const
     }
 }
 
-// Row-wise LayerNorm / RMSNorm (or plain copy when gamma is null) followed by the hi/lo split.  grid (T)
+// Row t of the input is x[t][:] (+ bias + the split-K partial sums of the GEMM that produced it, added in a
+// fixed order; the completed row is then stored to x_store, which becomes the residual stream).  Followed by
+// LayerNorm / RMSNorm (skipped when gamma is null) and the hi/lo split (skipped when hi is null).  grid (T)
 __global__ void __launch_bounds__(PF_THREADS) k_pf_norm_split(const float *x, int n, int norm, const float *gamma, const float *beta,
-                                                               float eps, __nv_bfloat16 *hi, __nv_bfloat16 *lo) {
+                                                               float eps, __nv_bfloat16 *hi, __nv_bfloat16 *lo, const float *partial,
+                                                               int n_split, int T, const float *bias, float *x_store) {
     __shared__ float red[2 * PF_THREADS / 32];
     const int t = blockIdx.x, tid = threadIdx.x;
     const float *row = x + (size_t)t * n;
+    if (n_split > 0) {
+        float *dst = x_store + (size_t)t * n;
+        for (int i = tid; i < n; i += PF_THREADS) {
+            float v = row[i] + (bias ? bias[i] : 0.f);
+            for (int z = 0; z < n_split; ++z) v += partial[((size_t)z * T + t) * n + i];
+            dst[i] = v;
+        }
+        row = dst;
+        __syncthreads();
+    }
+    if (!hi) return;
     float mean = 0.f, rstd = 1.f;
     if (gamma) {
         const float pilot = norm == NORM_LAYER ? row[0] : 0.f;
@@ -89,8 +103,8 @@ __global__ void k_pf_rope_append(const float *qkv, int q_rows, int kv_rows, int 
 // Causal attention of the T new positions over the slot's cache (rows 0 .. pos0 + t for position t).
 // grid (n_head, T); same row-sharing scheme as k_attn_decode, no sequence split.
 template <typename KT, int HD>
-__global__ void __launch_bounds__(ATT_THREADS) k_pf_attn(const float *q, float *o, KvView kv, int layer_local, int n_head,
-                                                          const int *pos, int slot, float scale) {
+__global__ void __launch_bounds__(ATT_THREADS) k_pf_attn(const float *q, __nv_bfloat16 *o_hi, __nv_bfloat16 *o_lo, KvView kv,
+                                                          int layer_local, int n_head, const int *pos, int slot, float scale) {
     constexpr int EPL = 16 / sizeof(KT), LPR = HD / EPL, RPW = 32 / LPR, NG = ATT_WARPS * RPW;
     __shared__ float sm_m[NG], sm_l[NG];
     __shared__ float sm_o[NG][HD];
@@ -142,7 +156,7 @@ __global__ void __launch_bounds__(ATT_THREADS) k_pf_attn(const float *q, float *
             L += sm_l[g2] * w;
             O += sm_o[g2][tid] * w;
         }
-        o[((size_t)t * n_head + h) * HD + tid] = O / L;
+        pf_split_store(o_hi, o_lo, ((size_t)t * n_head + h) * HD + tid, O / L);
     }
 }
 
@@ -165,17 +179,6 @@ __global__ void k_bt_rope_append(const float *qkv, int q_rows, int kv_rows, int 
             const int rk = r - q_rows, which = rk >= kv_rows, rl = rk - which * kv_rows;
             kv_store<KT>(kv_addr<KT>(kv, slot, layer_local, which, rl / hd, p, rl % hd), y);
         }
-    }
-}
-
-// y[t][i] = sum_z partial[z][t][i] + bias[i] + resid[t][i]  (fixed summation order).  grid (T)
-__global__ void k_pf_reduce(const float *partial, int n_split, int T, int n, const float *bias, const float *resid, float *y) {
-    const int t = blockIdx.x;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        float v = bias ? bias[i] : 0.f;
-        if (resid) v += resid[(size_t)t * n + i];
-        for (int z = 0; z < n_split; ++z) v += partial[((size_t)z * T + t) * n + i];
-        y[(size_t)t * n + i] = v;
     }
 }
 

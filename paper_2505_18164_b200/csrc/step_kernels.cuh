@@ -378,6 +378,7 @@ struct AttnArgs {
     int layer_local, n_head, n_split;
     const int *pos;
     float scale;
+    __nv_bfloat16 *o_hi, *o_lo; // optional: the merged output also as two bf16 planes (input of a tensor-core GEMM)
 };
 
 // grid (n_head, n_split, n_items).  A block scans its share of the cached rows of one head of one
@@ -478,7 +479,13 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_decode(const AttnArgs a, c
                 L += __ldcg(pb + (size_t)s2 * (HD + 2) + 1) * w;
                 O += __ldcg(pb + (size_t)s2 * (HD + 2) + 2 + tid) * w;
             }
-            a.o[(size_t)b * a.n_head * HD + h * HD + tid] = O / L;
+            const float ov = O / L;
+            a.o[(size_t)b * a.n_head * HD + h * HD + tid] = ov;
+            if (a.o_hi) {
+                const __nv_bfloat16 hv = __float2bfloat16_rn(ov);
+                a.o_hi[(size_t)b * a.n_head * HD + h * HD + tid] = hv;
+                a.o_lo[(size_t)b * a.n_head * HD + h * HD + tid] = __float2bfloat16_rn(ov - __bfloat162float(hv));
+            }
         }
         if (tid == 0) a.ticket[b * a.n_head + h] = 0u;
     }

@@ -49,6 +49,7 @@ struct TgArgs {
     int ldy;
     int *err;                 // set to 1 when a wait gave up
     float *partial;           // split-K (gridDim.z > 1): raw partial sums [z][T][ldy]; bias/resid/act/y are then unused
+    __nv_bfloat16 *out_hi, *out_lo; // optional: the result also (or, with y null, only) as two bf16 planes [T][ldy]
 };
 
 __device__ __forceinline__ uint32_t tg_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -210,7 +211,13 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                         } else if (t < a.T) {
                             float v = __uint_as_float(r[j]) + bias;
                             if (a.resid) v += a.resid[(size_t)t * a.ldy + row];
-                            a.y[(size_t)t * a.ldy + row] = tg_apply(v, a.act);
+                            v = tg_apply(v, a.act);
+                            if (a.y) a.y[(size_t)t * a.ldy + row] = v;
+                            if (a.out_hi) {
+                                const __nv_bfloat16 h = __float2bfloat16_rn(v);
+                                a.out_hi[(size_t)t * a.ldy + row] = h;
+                                a.out_lo[(size_t)t * a.ldy + row] = __float2bfloat16_rn(v - __bfloat162float(h));
+                            }
                         }
                     }
                 }
