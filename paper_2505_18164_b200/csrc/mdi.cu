@@ -109,7 +109,7 @@ struct mdi_ctx {
     bool capturing = false;
     int64_t cap_launches = 0, cap_steps = 0;
     // tensor-core first visit
-    bool pf_tc = false;
+    bool pf_tc = false, pdl = true;
     int tc_min_group = 5; // groups with at least this many samples run their linear layers on the tensor cores
     int *tg_err = nullptr;
     std::map<std::tuple<const void *, uint64_t, uint64_t, uint32_t>, CUtensorMap> tmaps;
@@ -159,6 +159,21 @@ template <typename T> int dalloc(mdi_ctx *c, T **p, size_t n, int64_t *account =
 
 inline void count_launch(mdi_ctx *c) {
     if (c->capturing) ++c->cap_launches; else ++c->st.kernel_launches;
+}
+
+// Launch with the programmatic-serialization attribute when g_pdl is set (the kernels of the tensor-core chain
+// call griddepcontrol.wait before touching their predecessor's results), else as a plain launch.
+bool g_pdl = false;
+template <typename... KArgs, typename... Args>
+void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = g_pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 // ---- kernel dispatch ------------------------------------------------------------------------------
@@ -248,10 +263,10 @@ int linear(mdi_ctx *c, int mode, LinArgs a, const Batch &bt, cudaStream_t st) {
 
 template <typename KT> void attn_hd(int hd, const AttnArgs &a, const Batch &bt, dim3 grid, cudaStream_t st) {
     switch (hd) {
-        case 16: k_attn_decode<KT, 16><<<grid, ATT_THREADS, 0, st>>>(a, bt); break;
-        case 32: k_attn_decode<KT, 32><<<grid, ATT_THREADS, 0, st>>>(a, bt); break;
-        case 64: k_attn_decode<KT, 64><<<grid, ATT_THREADS, 0, st>>>(a, bt); break;
-        default: k_attn_decode<KT, 128><<<grid, ATT_THREADS, 0, st>>>(a, bt); break;
+        case 16: launch_k(k_attn_decode<KT, 16>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
+        case 32: launch_k(k_attn_decode<KT, 32>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
+        case 64: launch_k(k_attn_decode<KT, 64>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
+        default: launch_k(k_attn_decode<KT, 128>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
     }
 }
 
@@ -380,6 +395,7 @@ constexpr int PF_SPLIT_MAX = 8; // K splits of the GEMMs with few row tiles (out
 int pf_setup(mdi_ctx *c) {
     const mdi_model_shape &s = c->s;
     c->pf_tc = s.weight_dtype == MDI_DTYPE_BF16 && c->o.prefill_mode != 1;
+    c->pdl = getenv("MDI_NO_PDL") == nullptr;
     // Which decode steps use the tensor-core linear layers (stream scheduler): by default groups of 5 or more
     // samples, and every group when one block's matrices are 48 MB or more (then a step moves enough bytes per
     // kernel for launches not to matter, and TMA-fed GEMM tiles stream faster than the CUDA-core tiles).
@@ -448,7 +464,7 @@ int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, c
     TgArgs a{};
     a.n_rows = n_rows; a.K = K; a.T = T; a.n_tile = n_tile; a.bias = bias; a.resid = resid; a.act = act; a.y = y; a.ldy = n_rows;
     a.err = c->tg_err; a.partial = P.pf_part; a.out_hi = out_hi; a.out_lo = out_lo;
-    k_tc_gemm<<<dim3(grid_x, (T + n_tile - 1) / n_tile, splits), TG_THREADS, tg_smem_bytes(n_tile), st>>>(*mw, *mhi, *mlo, a);
+    launch_k(k_tc_gemm, dim3(grid_x, (T + n_tile - 1) / n_tile, splits), dim3(TG_THREADS), tg_smem_bytes(n_tile), st, *mw, *mhi, *mlo, a);
     count_launch(c);
     if (pending) {
         pending->splits = splits > 1 ? splits : 0;
@@ -461,10 +477,10 @@ int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, c
 template <typename KT> void pf_attn_hd(int hd, dim3 g, cudaStream_t st, const float *q, __nv_bfloat16 *ohi, __nv_bfloat16 *olo,
                                        const KvView &kv, int ll, int n_head, const int *pos, int slot, float scale) {
     switch (hd) {
-        case 16: k_pf_attn<KT, 16><<<g, ATT_THREADS, 0, st>>>(q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
-        case 32: k_pf_attn<KT, 32><<<g, ATT_THREADS, 0, st>>>(q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
-        case 64: k_pf_attn<KT, 64><<<g, ATT_THREADS, 0, st>>>(q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
-        default: k_pf_attn<KT, 128><<<g, ATT_THREADS, 0, st>>>(q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        case 16: launch_k(k_pf_attn<KT, 16>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        case 32: launch_k(k_pf_attn<KT, 32>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        case 64: launch_k(k_pf_attn<KT, 64>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        default: launch_k(k_pf_attn<KT, 128>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
     }
 }
 
@@ -483,8 +499,9 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
     const float scale = 1.0f / std::sqrt((float)s.head_dim);
     __nv_bfloat16 *hi = (__nv_bfloat16 *)P.pf_hi, *lo = (__nv_bfloat16 *)P.pf_lo;
     int rc;
+    struct PdlScope { PdlScope(bool on) { g_pdl = on; } ~PdlScope() { g_pdl = false; } } pdl_scope(c->pdl);
     if (!bt && p == 0) {
-        k_pf_embed<__nv_bfloat16><<<T, 256, 0, st>>>((const __nv_bfloat16 *)c->wte, (const __nv_bfloat16 *)c->wpe, d, s.vocab, tok_dev,
+        launch_k(k_pf_embed<__nv_bfloat16>, dim3(T), dim3(256), 0, st, (const __nv_bfloat16 *)c->wte, (const __nv_bfloat16 *)c->wpe, d, s.vocab, tok_dev,
                                                     P.pos_dev, slot, P.pf_xa);
         count_launch(c);
         x_in = P.pf_xa;
@@ -495,14 +512,14 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
         const int ll = l - P.lo;
         const float *xin_l = l == P.lo ? x_in : x_out;
         // norm 1 (first completing the residual stream if the previous GEMM was split)
-        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(pend.splits ? pend.resid : xin_l, d, norm, L.ln1g, L.ln1b, s.norm_eps, hi, lo, P.pf_part,
+        launch_k(k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, pend.splits ? pend.resid : xin_l, d, norm, L.ln1g, L.ln1b, s.norm_eps, hi, lo, P.pf_part,
                                                   pend.splits, T, pend.bias, x_out);
         count_launch(c);
         pend = PfPending();
         if ((rc = pf_gemm(c, P, L.wqkv, qw + 2 * kw, d, T, L.bqkv, nullptr, TG_NONE, P.pf_qkv, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
         if (bt) {
-            if (c->kv_f32) k_bt_rope_append<float><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
-            else k_bt_rope_append<__nv_bfloat16><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
+            if (c->kv_f32) launch_k(k_bt_rope_append<float>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
+            else launch_k(k_bt_rope_append<__nv_bfloat16>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
             count_launch(c);
             AttnArgs a{};
             a.q = P.qbuf; a.o = P.obuf; a.part = P.part; a.ticket = P.attn_ticket; a.kv = kv; a.layer_local = ll; a.n_head = s.n_head;
@@ -511,8 +528,8 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
             if (c->kv_f32) attn_hd<float>(s.head_dim, a, *bt, g, st); else attn_hd<__nv_bfloat16>(s.head_dim, a, *bt, g, st);
             count_launch(c);
         } else {
-            if (c->kv_f32) k_pf_rope_append<float><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
-            else k_pf_rope_append<__nv_bfloat16><<<T, 256, 0, st>>>(P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
+            if (c->kv_f32) launch_k(k_pf_rope_append<float>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
+            else launch_k(k_pf_rope_append<__nv_bfloat16>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
             count_launch(c);
             if (c->kv_f32) pf_attn_hd<float>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
             else pf_attn_hd<__nv_bfloat16>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
@@ -521,13 +538,13 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
         // output projection + residual -> x_out (or partial sums, completed by the next kernel)
         PfPending po;
         if ((rc = pf_gemm(c, P, L.wo, d, qw, T, L.bo, xin_l, TG_NONE, x_out, nullptr, nullptr, &po, st)) != MDI_OK) return rc;
-        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(po.splits ? po.resid : x_out, d, norm, L.ln2g, L.ln2b, s.norm_eps, hi, lo, P.pf_part, po.splits, T,
+        launch_k(k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, po.splits ? po.resid : x_out, d, norm, L.ln2g, L.ln2b, s.norm_eps, hi, lo, P.pf_part, po.splits, T,
                                                   po.bias, x_out);
         count_launch(c);
         if (s.act == MDI_ACT_SWIGLU) {
             if ((rc = pf_gemm(c, P, L.wgate, F, d, T, nullptr, nullptr, TG_NONE, P.pf_h, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
             if ((rc = pf_gemm(c, P, L.wup, F, d, T, nullptr, nullptr, TG_NONE, P.pf_u, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
-            k_pf_swiglu_split<<<T, 256, 0, st>>>(P.pf_h, P.pf_u, F, hi, lo);
+            launch_k(k_pf_swiglu_split, dim3(T), dim3(256), 0, st, P.pf_h, P.pf_u, F, hi, lo);
             count_launch(c);
             if ((rc = pf_gemm(c, P, L.wdown, d, F, T, nullptr, x_out, TG_NONE, x_out, nullptr, nullptr, &pend, st)) != MDI_OK) return rc;
         } else {
@@ -535,18 +552,18 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
             if ((rc = pf_gemm(c, P, L.w1, F, d, T, L.b1, nullptr, s.act == MDI_ACT_GELU_ERF ? TG_GELU_ERF : TG_GELU_TANH, P.pf_h, nullptr, nullptr,
                               nullptr, st)) != MDI_OK)
                 return rc;
-            k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo, nullptr, 0, T, nullptr, nullptr);
+            launch_k(k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo, nullptr, 0, T, nullptr, nullptr);
             count_launch(c);
             if ((rc = pf_gemm(c, P, L.w2, d, F, T, L.b2, x_out, TG_NONE, x_out, nullptr, nullptr, &pend, st)) != MDI_OK) return rc;
         }
     }
     if (pend.splits) { // complete the residual stream after the last block
-        k_pf_norm_split<<<T, PF_THREADS, 0, st>>>(pend.resid, d, NORM_NONE, nullptr, nullptr, 0.f, nullptr, nullptr, P.pf_part, pend.splits, T,
+        launch_k(k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, pend.resid, d, NORM_NONE, nullptr, nullptr, 0.f, nullptr, nullptr, P.pf_part, pend.splits, T,
                                                   pend.bias, x_out);
         count_launch(c);
     }
-    if (bt) k_bt_advance<<<1, 32, 0, st>>>(P.pos_dev, *bt);
-    else k_pf_advance<<<1, 32, 0, st>>>(P.pos_dev, slot, T);
+    if (bt) launch_k(k_bt_advance, dim3(1), dim3(32), 0, st, P.pos_dev, *bt);
+    else launch_k(k_pf_advance, dim3(1), dim3(32), 0, st, P.pos_dev, slot, T);
     count_launch(c);
     return MDI_OK;
 }

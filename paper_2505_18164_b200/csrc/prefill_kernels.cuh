@@ -18,6 +18,8 @@ __device__ __forceinline__ void pf_split_store(__nv_bfloat16 *hi, __nv_bfloat16 
 // x[t][:] = wte[tok[t]][:] (+ wpe[pos0 + t][:]);  grid (T)
 template <typename WT>
 __global__ void k_pf_embed(const WT *wte, const WT *wpe, int d, int vocab, const int *tok, const int *pos, int slot, float *x) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = blockIdx.x;
     const int id = min(max(tok[t], 0), vocab - 1);
     const int p = pos[slot] + t;
@@ -34,6 +36,8 @@ __global__ void k_pf_embed(const WT *wte, const WT *wpe, int d, int vocab, const
 __global__ void __launch_bounds__(PF_THREADS) k_pf_norm_split(const float *x, int n, int norm, const float *gamma, const float *beta,
                                                                float eps, __nv_bfloat16 *hi, __nv_bfloat16 *lo, const float *partial,
                                                                int n_split, int T, const float *bias, float *x_store) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ float red[2 * PF_THREADS / 32];
     const int t = blockIdx.x, tid = threadIdx.x;
     const float *row = x + (size_t)t * n;
@@ -72,6 +76,8 @@ __global__ void __launch_bounds__(PF_THREADS) k_pf_norm_split(const float *x, in
 
 // h = SiLU(g) * u, split.  grid (T)
 __global__ void k_pf_swiglu_split(const float *g, const float *u, int n, __nv_bfloat16 *hi, __nv_bfloat16 *lo) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = blockIdx.x;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
         const size_t k = (size_t)t * n + i;
@@ -83,6 +89,8 @@ __global__ void k_pf_swiglu_split(const float *g, const float *u, int n, __nv_bf
 template <typename KT>
 __global__ void k_pf_rope_append(const float *qkv, int q_rows, int kv_rows, int hd, int rope, const float *rope_cos,
                                  const float *rope_sin, KvView kv, int layer_local, const int *pos, int slot, float *q_out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = blockIdx.x, p = pos[slot] + t, half = hd >> 1, rows = q_rows + 2 * kv_rows;
     const float *src = qkv + (size_t)t * rows;
     for (int r = threadIdx.x; r < rows; r += blockDim.x) {
@@ -108,6 +116,8 @@ __global__ void __launch_bounds__(ATT_THREADS) k_pf_attn(const float *q, __nv_bf
     constexpr int EPL = 16 / sizeof(KT), LPR = HD / EPL, RPW = 32 / LPR, NG = ATT_WARPS * RPW;
     __shared__ float sm_m[NG], sm_l[NG];
     __shared__ float sm_o[NG][HD];
+    pdl_launch_dependents();
+    pdl_wait();
     const int h = blockIdx.x, t = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, grp = lane / LPR;
     const int n_keys = pos[slot] + t + 1;
@@ -165,6 +175,8 @@ __global__ void __launch_bounds__(ATT_THREADS) k_pf_attn(const float *q, __nv_bf
 template <typename KT>
 __global__ void k_bt_rope_append(const float *qkv, int q_rows, int kv_rows, int hd, int rope, const float *rope_cos,
                                  const float *rope_sin, KvView kv, int layer_local, const int *pos, Batch bt, float *q_out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = blockIdx.x, slot = bt.slot[t], p = pos[slot] + bt.off[t], half = hd >> 1, rows = q_rows + 2 * kv_rows;
     const float *src = qkv + (size_t)t * rows;
     for (int r = threadIdx.x; r < rows; r += blockDim.x) {
@@ -183,11 +195,15 @@ __global__ void k_bt_rope_append(const float *qkv, int q_rows, int kv_rows, int 
 }
 
 __global__ void k_bt_advance(int *pos, Batch bt) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int i = threadIdx.x;
     if (blockIdx.x == 0 && i < bt.n && bt.adv[i]) pos[bt.slot[i]] += bt.adv[i];
 }
 
 __global__ void k_pf_advance(int *pos, int slot, int by) {
+    pdl_launch_dependents();
+    pdl_wait();
     if (threadIdx.x == 0 && blockIdx.x == 0) pos[slot] += by;
 }
 

@@ -19,6 +19,12 @@ constexpr int LIN_WARPS = LIN_THREADS / 32;
 constexpr int ATT_THREADS = 128;
 constexpr int ATT_WARPS = ATT_THREADS / 32;
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may start
+// while its predecessor in the stream is still running; it must not touch the predecessor's results before
+// pdl_wait() (which returns once the predecessor has completed and flushed).  Without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 struct Batch {
     int n;
     int slot[MAXB]; // slot of the item
@@ -395,6 +401,8 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_decode(const AttnArgs a, c
     __shared__ float sm_o[NG][HD];
     __shared__ bool is_last;
 
+    pdl_launch_dependents();
+    pdl_wait();
     const int h = blockIdx.x, sp = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, grp = lane / LPR;

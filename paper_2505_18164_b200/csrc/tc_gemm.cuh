@@ -147,13 +147,28 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         if (lane == 0) {
             // ---- TMA producer
             const uint32_t stage_bytes = (uint32_t)TG_STAGE_BYTES;
             bool ok = true;
-            for (int kb = 0; kb < n_kb && ok; ++kb) {
+            // The weights depend on nothing: the first ring of weight tiles is requested before waiting for the
+            // preceding kernel (programmatic dependent launch); the inputs it produced are requested after.
+            const int pre = n_kb < TG_STAGES ? n_kb : TG_STAGES;
+            for (int kb = 0; kb < pre; ++kb) {
+                const uint32_t full = full0 + 8 * kb, base = tg_smem_u32(smem + (size_t)kb * TG_STAGE_BYTES);
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full), "r"(stage_bytes) : "memory");
+                tg_tma_2d(base, &tm_w, (kb_lo + kb) * TG_BK, m0, full);
+            }
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            for (int kb = 0; kb < pre; ++kb) {
+                const uint32_t full = full0 + 8 * kb, base = tg_smem_u32(smem + (size_t)kb * TG_STAGE_BYTES);
+                tg_tma_2d(base + TG_W_BYTES, &tm_xhi, (kb_lo + kb) * TG_BK, t0, full);
+                tg_tma_2d(base + TG_W_BYTES + TG_X_BYTES, &tm_xlo, (kb_lo + kb) * TG_BK, t0, full);
+            }
+            for (int kb = pre; kb < n_kb && ok; ++kb) {
                 const int s = kb % TG_STAGES;
                 if (kb >= TG_STAGES) ok = tg_wait(empty0 + 8 * s, ((kb / TG_STAGES) & 1) ^ 1, a.err);
                 if (!ok) break;
@@ -188,6 +203,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         }
     } else {
         // ---- epilogue: warps 2..5; a warp may only touch the TMEM lanes 32 * (warp % 4) .. + 31
+        asm volatile("griddepcontrol.wait;" ::: "memory"); // bias / residual / partial buffers belong to earlier kernels
         const bool ok = tg_wait(accbar, 0, a.err) && *(volatile int *)a.err == 0;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int lane_base = (warp & 3) * 32;
