@@ -34,9 +34,9 @@ sys.path.insert(0, ROOT)
 from paper_2505_18164_b200 import inputs as I  # noqa: E402
 
 # DRAM traffic of the persistent decode kernel relative to its algorithmic bytes, from the ncu capture
-# summarised in profiles/persistent_decode_gpt2_small.md (17.15 GB moved for 17.17 GB algorithmic; traffic
+# summarised in profiles/persistent_decode_gpt2_small.md (17.149 GB moved for 17.171 GB algorithmic; traffic
 # grows with the number of passes like the algorithmic bytes do).  None for other workloads / schedulers.
-PK_TRAFFIC_RATIO = {"gpt2_small": 17.15 / 17.17}
+PK_TRAFFIC_RATIO = {"gpt2_small": 17.149 / 17.171}
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
