@@ -126,13 +126,14 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def cpu_baseline(w: I.Workload, weights, n_new_sample: int = 256):
+def cpu_baseline(w: I.Workload, weights, n_new_sample: int = 512):
     """The CPU checker, as it stands, on a bounded sample of the workload: all samples, full prompts,
     the first n_new_sample of the new tokens, scheduled by its own recurrent-pipeline simulation."""
     from oracle import mdi_oracle as O
     orc = O.Oracle(w.shape, weights)
     prompts = I.make_prompts(w.shape.vocab, w.n_samples, w.n_prompt, w.prompt_seed)
     t0 = time.perf_counter()
+    n_new_sample = min(n_new_sample, w.n_new)
     toks, _, _ = orc.generate_pipeline([[int(t) for t in p] for p in prompts], n_new_sample, list(w.part_bounds),
                                        head_on_starter=False)
     dt = time.perf_counter() - t0

@@ -1283,11 +1283,19 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
         if ((rc = pk_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
     } else if (t_total) {
         const int R = c->rounds_per_graph;
-        const long W = R > 0 ? (long)R * K : 0;
         const long t_steady = K > 1 ? K : 0; // first tick, multiple of K, from which every partition is in steady state
-        if (W > 0 && t_steady + 2 * W <= total) {
-            if ((rc = enqueue_ticks(c, n_samples, G, 0, t_steady, total)) != MDI_OK) return rc;
-            t = t_steady;
+        // Steady-state windows are replayed from CUDA graphs: first windows of R rounds, then windows of one round
+        // for what is left, so that at most a round (plus fill and drain) is launched kernel by kernel.
+        bool started = false;
+        for (int pass = 0; pass < 2 && R > 0; ++pass) {
+            const long W = pass == 0 ? (long)R * K : (long)K;
+            if (pass == 1 && R == 1) break;
+            if ((started ? t : t_steady) + (pass == 0 ? 2 * W : W) > total) continue;
+            if (!started) {
+                if ((rc = enqueue_ticks(c, n_samples, G, 0, t_steady, total)) != MDI_OK) return rc;
+                t = t_steady;
+                started = true;
+            }
             auto key = std::make_pair(n_samples, (int)W);
             GraphEntry &ge = c->graphs[key];
             if (!ge.exec) {
