@@ -189,7 +189,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="mdi", choices=["mdi", "reference"])
-    ap.add_argument("--workload", default="gpt2_small", choices=I.WORKLOAD_ORDER)
+    ap.add_argument("--workload", default="gpt2_small", choices=list(I.ALL_WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--rounds-per-graph", type=int, default=0)
     ap.add_argument("--scheduler", type=int, default=0, help="0 auto (persistent kernel when it fits), 1 streams, 2 persistent")
@@ -197,7 +197,7 @@ def main():
     ap.add_argument("--n-new", type=int, default=0, help="shorter generation (profiler captures only; not the headline)")
     ap.add_argument("--n-prompt", type=int, default=0, help="shorter prompts (profiler captures only)")
     args = ap.parse_args()
-    w = I.WORKLOADS[args.workload]
+    w = I.ALL_WORKLOADS[args.workload]
     if args.n_new or args.n_prompt:
         w = I.scaled(w, n_new=args.n_new or w.n_new, n_prompt=args.n_prompt or w.n_prompt)
     from paper_2505_18164_b200 import build

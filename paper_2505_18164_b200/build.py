@@ -38,7 +38,7 @@ def build_mdi(force: bool = False, verbose: bool = False) -> str:
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
         cmd = [nvcc] + flags + (["-Xptxas", "-v"] if verbose else []) + \
-              ["-I", os.path.join(_ROOT, "include"), "-o", LIB_MDI] + cu + ["-lcuda"]
+              ["-I", os.path.join(_ROOT, "include"), "-o", LIB_MDI] + cu
         subprocess.check_call(cmd)
     return LIB_MDI
 

@@ -103,6 +103,27 @@ WORKLOADS: Dict[str, Workload] = {
 }
 WORKLOAD_ORDER = ["tiny_gpt_fp32", "gpt2_small", "gpt2_medium", "gpt2_xl", "llama_7b"]
 
+# The paper's own two models as synthetic shapes (Section IV-A): what it states - blocks, embedding width, heads,
+# vocabulary, context, blocks per node, three samples, fp32 (its boards had no 16-bit arithmetic), a
+# one-token prompt and 800 generated tokens - is kept; what it does not state is chosen here: the MLP width
+# (5120 gives the quoted 304 M parameters; 5632 is the width of the public 1.1 B model), the number of
+# key/value heads (16 = plain multi-head attention for the small model, 4 for the large one), untied output layer.
+PAPER_SHAPES: Dict[str, Workload] = {
+    "nanollama_3nodes": Workload(
+        "nanollama_3nodes",
+        ModelShape(ARCH_LLAMA, 12, 1024, 16, 64, 16, 5120, 32000, 2048, DT_F32, 0, 0, ACT_SWIGLU),
+        (0, 2, 7, 12), 3, 1, 800),
+    "nanollama_2nodes": Workload(
+        "nanollama_2nodes",
+        ModelShape(ARCH_LLAMA, 12, 1024, 16, 64, 16, 5120, 32000, 2048, DT_F32, 0, 0, ACT_SWIGLU),
+        (0, 5, 12), 3, 1, 800),
+    "tinyllama_3nodes": Workload(
+        "tinyllama_3nodes",
+        ModelShape(ARCH_LLAMA, 22, 2048, 32, 64, 4, 5632, 32000, 2048, DT_F32, 0, 0, ACT_SWIGLU),
+        (0, 6, 14, 22), 3, 1, 800),
+}
+ALL_WORKLOADS: Dict[str, Workload] = {**WORKLOADS, **PAPER_SHAPES}
+
 
 def scaled(w: Workload, **kw) -> Workload:
     """A copy of a workload with some fields replaced (shape fields go to the shape)."""

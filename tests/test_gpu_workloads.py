@@ -21,7 +21,7 @@ pytestmark = pytest.mark.gpu
 
 def _run(name, n_prompt=None, n_new=None, check=None, chunk=8, scheduler=0):
     from paper_2505_18164_b200 import mdi
-    w = I.WORKLOADS[name]
+    w = I.ALL_WORKLOADS[name]
     w = I.scaled(w, n_prompt=n_prompt or w.n_prompt, n_new=n_new or w.n_new)
     s, S, P, N = w.shape, w.n_samples, w.n_prompt, w.n_new
     check = list(range(S)) if check is None else check
@@ -82,3 +82,9 @@ def test_gpt2_xl_shape_uneven_groups():
 
 def test_llama_7b_shape_groups_of_eight():
     _run("llama_7b", n_prompt=8, n_new=6, check=[0, 63], chunk=3)
+
+
+@pytest.mark.parametrize("name", ["nanollama_3nodes", "nanollama_2nodes", "tinyllama_3nodes"])
+def test_paper_model_shapes(name):
+    """The paper's own models as synthetic fp32 shapes: unequal partitions, one-token prompts (Section IV-A)."""
+    _run(name, n_new=10, check=[0, 2], chunk=5)

@@ -56,6 +56,10 @@ def test_workload_tables():
         assert all(b > a for a, b in zip(w.part_bounds[:-1], w.part_bounds[1:]))
         assert w.n_prompt + w.n_new <= s.n_ctx + 1
         assert s.n_head * s.head_dim == s.d_model
+    # the paper's small model: 304 million parameters (Section IV-A)
+    nano = I.param_bytes(I.PAPER_SHAPES["nanollama_3nodes"].shape) / 4
+    assert abs(nano - 304e6) < 3e6
+    assert abs(I.param_bytes(I.PAPER_SHAPES["tinyllama_3nodes"].shape) / 4 - 1.1e9) < 0.02e9
     # sizes quoted for the shapes: whole-model parameter bytes
     mb = {n: I.param_bytes(I.WORKLOADS[n].shape) / 1e6 for n in I.WORKLOAD_ORDER}
     assert abs(mb["gpt2_small"] - 248.9) < 1.0     # 247.3 MB of matrices + wpe
