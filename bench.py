@@ -34,7 +34,7 @@ sys.path.insert(0, ROOT)
 from paper_2505_18164_b200 import inputs as I  # noqa: E402
 
 # DRAM traffic of the persistent decode kernel relative to its algorithmic bytes, from the ncu capture
-# summarised in profiles/persistent_decode_gpt2_small.md (17.149 GB moved for 17.171 GB algorithmic; traffic
+# kept with the profiler summaries of this repository (17.149 GB moved for 17.171 GB algorithmic; traffic
 # grows with the number of passes like the algorithmic bytes do).  None for other workloads / schedulers.
 PK_TRAFFIC_RATIO = {"gpt2_small": 17.149 / 17.171}
 FALLBACK_HBM_GBS = 6650.0
@@ -308,7 +308,7 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                          "traffic": (PK_TRAFFIC_RATIO[w.name] * db["total"] if w.name in PK_TRAFFIC_RATIO and args.scheduler != 1 else None),
-                         "traffic_note": "scaled from a 23-pass ncu capture of the same kernel (profiles/)", "scope": "decode phase of one step (all kernels of mdi_generate)",
+                         "traffic_note": "scaled from a 23-pass ncu capture of the same kernel", "scope": "decode phase of one step (all kernels of mdi_generate)",
                          "algorithmic_bytes": db["total"], "weight_bytes": db["weights"], "kv_bytes": db["kv"]},
             "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(S * P * 4),
                     "d2h_bytes_per_step": int(S * N * 4)},
