@@ -78,6 +78,11 @@ typedef struct {
     int tc_min_group;  /* decode steps of groups with at least this many samples run their linear layers as tensor-core
                           GEMMs (bf16 weights, prefill_mode 0; such calls use the stream scheduler).  0 (default): 5,
                           or 1 when the matrices of one block hold 48 MB or more */
+    int wait_limit_ms; /* limit of every wait inside the persistent kernel (input edge, team barrier, weight tile); when
+                          one runs out mdi_generate returns MDI_ERR_TIMEOUT, every sample is reset and the context stays
+                          usable.  0 (default): 2000 ms */
+    int debug_withhold_handoff; /* failure-detection check: p > 0 makes partition p-1 withhold its output handoff during
+                          the first persistent mdi_generate after creation, so that the next partition's wait runs out */
     int scheduler;     /* how mdi_generate runs the recurrent pipeline.  0: the persistent kernel (one launch,
                           one team of thread blocks per partition, flag handoff between teams) when the shape
                           fits it (groups of at most 4 samples), else the stream scheduler; 1: always the
@@ -150,7 +155,8 @@ int mdi_step(mdi_ctx *ctx, int partition, int slot, const void *act_in_dev, void
  * samples than partitions); a group's samples share one pass over the partition's weights.  A token produced by the last partition is fed to partition 0 one tick
  * later; the last token of the call is produced but not fed (it is fed first by a later call).
  * out_tokens: [n_samples][n_new_tokens] int32, host (or device for the _dev form).
- * Blocks until the tokens are there.  Errors: ARG, STATE, CONTEXT, OOM. */
+ * Blocks until the tokens are there.  Errors: ARG, STATE, CONTEXT, OOM, TIMEOUT (a bounded wait of the
+ * persistent kernel ran out: all samples are then reset, prefill them again). */
 int mdi_generate(mdi_ctx *ctx, int n_samples, int n_new_tokens, int32_t *out_tokens_host);
 int mdi_generate_dev(mdi_ctx *ctx, int n_samples, int n_new_tokens, int32_t *out_tokens_dev);
 

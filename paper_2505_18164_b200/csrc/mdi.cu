@@ -115,6 +115,7 @@ struct mdi_ctx {
     std::map<std::tuple<const void *, uint64_t, uint64_t, uint32_t>, CUtensorMap> tmaps;
     // persistent decode kernel
     bool pk_ok = false, pk_prof_on = false, pk_tables_stale = true;
+    int withhold_once = -1; // partition whose output flags the next persistent launch withholds (time-out test hook)
     int pk_slots = 0, pk_xs_floats = 0, pk_nb = 1, n_sm = 0, scheduler = 0;
     size_t pk_smem = 0;
     std::vector<PkTeam> pk_teams_host;
@@ -812,6 +813,9 @@ int pk_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     P.logits = c->logits; P.head_pv = c->head_pv; P.head_pi = c->head_pi; P.cur_tok = c->cur_tok; P.tok_log = c->tok_log;
     P.gen_count = c->gen_count; P.teacher = c->teacher; P.n_teacher = c->n_teacher; P.log_stride = s.n_ctx; P.err = c->pk_err;
     P.prof = c->pk_prof_on ? c->pk_prof : nullptr;
+    P.wait_ns = c->o.wait_limit_ms > 0 ? (unsigned long long)c->o.wait_limit_ms * 1000000ull : PK_WAIT_NS;
+    P.withhold_partition = c->withhold_once;
+    c->withhold_once = -1;
     int grid = 0;
     for (auto &T : c->pk_teams_host) grid += T.n_cta;
     const int nb = (n_samples + G - 1) / G;
@@ -913,6 +917,8 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     c->n_split = c->o.attn_splits > 0 ? c->o.attn_splits : std::max(1, std::min(16, s.n_ctx / 128));
     c->rounds_per_graph = c->o.rounds_per_graph != 0 ? c->o.rounds_per_graph : 16;
     if (c->o.prefill_mode < 0 || c->o.prefill_mode > 1) return bail(fail(c, MDI_ERR_ARG, "prefill_mode must be 0 or 1"));
+    if (c->o.debug_withhold_handoff < 0 || c->o.debug_withhold_handoff > K) return bail(fail(c, MDI_ERR_ARG, "debug_withhold_handoff must name a partition (1-based) or be 0"));
+    c->withhold_once = c->o.debug_withhold_handoff - 1;
     c->scheduler = c->o.scheduler;
     if (c->scheduler < 0 || c->scheduler > 2) return bail(fail(c, MDI_ERR_ARG, "scheduler must be 0, 1 or 2"));
     const int G = std::min(n_samples, K);
@@ -1339,7 +1345,12 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
     if (t_total && use_pk) {
         int kerr = 0;
         CU(cudaMemcpy(&kerr, c->pk_err, sizeof(int), cudaMemcpyDeviceToHost));
-        if (kerr) return fail(c, MDI_ERR_TIMEOUT, "persistent decode kernel gave up waiting (code %d: 1 edge flag, 2 team barrier, 3 weight tile, 4 ring slot)", kerr);
+        if (kerr) {
+            // the pipeline stopped half-way: positions, caches and counters no longer agree, so every sample is
+            // forgotten (like mdi_reset_sample); the context itself stays usable
+            for (int smp = 0; smp < c->S; ++smp) mdi_reset_sample(c, smp);
+            return fail(c, MDI_ERR_TIMEOUT, "persistent decode kernel gave up waiting (code %d: 1 edge flag, 2 team barrier, 3 weight tile, 4 ring slot); all samples were reset", kerr);
+        }
     }
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, c->ev_t0, c->ev_t1) == cudaSuccess) c->st.last_generate_ms = ms;

@@ -33,7 +33,7 @@ constexpr int PK_SLOT_BYTES = 32768;
 constexpr int PK_MAX_SLOTS = 6;
 constexpr int PK_MAXNB = 4;
 constexpr int PK_SMEM_PHASES = 48; // phase descriptors of a team kept in shared memory (more: read from global memory)
-constexpr unsigned long long PK_WAIT_NS = 2000000000ull; // 2 s
+constexpr unsigned long long PK_WAIT_NS = 2000000000ull; // default limit of a wait: 2 s
 
 enum PkKind { PK_QKV = 0, PK_ATTN = 1, PK_OUT = 2, PK_FC1 = 3, PK_GATEUP = 4, PK_FC2 = 5, PK_HEAD = 6 };
 enum PkProf { PF_FLAG = 0, PF_PROLOGUE = 1, PF_TILES = 2, PF_BARRIER = 3, PF_ATTN = 4, PF_HEADFIN = 5, PF_PROD_WAIT = 6,
@@ -71,6 +71,8 @@ struct PkParams {
     const int *teacher, *n_teacher;
     int log_stride;
     int *err;
+    unsigned long long wait_ns; // limit of every wait
+    int withhold_partition;     // >= 0: that partition never raises its output flags (checks the time-out path)
     unsigned long long *prof; // optional [grid][PK_PROF_N] nanoseconds per category (thread 0 and the producer of each block)
 };
 
@@ -122,7 +124,7 @@ __device__ __forceinline__ bool pk_probe(int kind, const void *p, uint32_t a) {
     if (kind == PKW_MBAR) return mbar_try_wait((uint32_t)(uintptr_t)p, a);
     return *reinterpret_cast<const volatile int *>(p) >= (int)a;
 }
-__device__ __noinline__ bool pk_wait_slow(int kind, const void *p, uint32_t a, int *err, int code) {
+__device__ __noinline__ bool pk_wait_slow(int kind, const void *p, uint32_t a, int *err, int code, unsigned long long limit_ns) {
     unsigned long long t0 = 0;
     for (unsigned it = 0;; ++it) {
         if (pk_probe(kind, p, a)) return false;
@@ -130,23 +132,23 @@ __device__ __noinline__ bool pk_wait_slow(int kind, const void *p, uint32_t a, i
             if (*(volatile int *)err) return true;
             const unsigned long long now = pk_now();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > PK_WAIT_NS) break;
+            else if (now - t0 > limit_ns) break;
         }
     }
     atomicCAS(err, 0, code);
     return true;
 }
-__device__ __forceinline__ void wait_ge(const unsigned *p, unsigned target, int *err, int code, bool &dead) {
+__device__ __forceinline__ void wait_ge(const unsigned *p, unsigned target, int *err, int code, bool &dead, unsigned long long lim) {
     if (dead || pk_probe(PKW_GLOBAL_GE, p, target)) return;
-    dead = pk_wait_slow(PKW_GLOBAL_GE, p, target, err, code);
+    dead = pk_wait_slow(PKW_GLOBAL_GE, p, target, err, code, lim);
 }
-__device__ __forceinline__ void wait_mbar(uint32_t bar, uint32_t parity, int *err, int code, bool &dead) {
+__device__ __forceinline__ void wait_mbar(uint32_t bar, uint32_t parity, int *err, int code, bool &dead, unsigned long long lim) {
     if (dead || pk_probe(PKW_MBAR, (const void *)(uintptr_t)bar, parity)) return;
-    dead = pk_wait_slow(PKW_MBAR, (const void *)(uintptr_t)bar, parity, err, code);
+    dead = pk_wait_slow(PKW_MBAR, (const void *)(uintptr_t)bar, parity, err, code, lim);
 }
-__device__ __forceinline__ void wait_smem_ge(const volatile int *p, int target, int *err, int code, bool &dead) {
+__device__ __forceinline__ void wait_smem_ge(const volatile int *p, int target, int *err, int code, bool &dead, unsigned long long lim) {
     if (dead || *p >= target) return;
-    dead = pk_wait_slow(PKW_SMEM_GE, (const void *)p, (uint32_t)target, err, code);
+    dead = pk_wait_slow(PKW_SMEM_GE, (const void *)p, (uint32_t)target, err, code, lim);
 }
 __device__ __noinline__ void pk_lap(unsigned long long *pf, unsigned long long *t, int cat) {
     const unsigned long long n = pk_now();
@@ -297,7 +299,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                         const int slot = (int)(seq % NS);
                         const uint32_t par = (uint32_t)((seq / NS) & 1);
                         lap(PF_PROD_TOTAL);
-                        if (lane == 0 && seq >= NS) wait_mbar(empty_base + 8 * slot, par ^ 1, P.err, PKE_EMPTY, dead);
+                        if (lane == 0 && seq >= NS) wait_mbar(empty_base + 8 * slot, par ^ 1, P.err, PKE_EMPTY, dead, P.wait_ns);
                         dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;
                         lap(PF_PROD_WAIT);
                         if (dead) break;
@@ -345,7 +347,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
             ++bar_epoch;
             if (T.n_cta > 1) {
                 red_release_add(T.bar, 1u);
-                wait_ge(T.bar, bar_epoch * (unsigned)T.n_cta, P.err, PKE_BARRIER, dead);
+                wait_ge(T.bar, bar_epoch * (unsigned)T.n_cta, P.err, PKE_BARRIER, dead, P.wait_ns);
             }
             if (dead) *s_dead = 1;
         }
@@ -368,8 +370,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
         }
         // ---- input edge
         if (tid == 0) {
-            if (!T.is_first) wait_ge(T.flag_in + j, r + 1, P.err, PKE_FLAG, dead);
-            else if (r > 0) wait_ge(T.flag_in + j, r, P.err, PKE_FLAG, dead);
+            if (!T.is_first) wait_ge(T.flag_in + j, r + 1, P.err, PKE_FLAG, dead, P.wait_ns);
+            else if (r > 0) wait_ge(T.flag_in + j, r, P.err, PKE_FLAG, dead, P.wait_ns);
             if (dead) *s_dead = 1;
         }
         consumer_bar();
@@ -650,8 +652,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                         // a parity test is only meaningful once every earlier tile of this slot has been consumed
                         // (warps run ahead of one another); then wait for this tile's bytes to land
                         lap(PF_TILES);
-                        wait_smem_ge(s_cons + slot, lap_no, P.err, PKE_FULL, dead);
-                        wait_mbar(full_base + 8 * slot, (uint32_t)(lap_no & 1), P.err, PKE_FULL, dead);
+                        wait_smem_ge(s_cons + slot, lap_no, P.err, PKE_FULL, dead, P.wait_ns);
+                        wait_mbar(full_base + 8 * slot, (uint32_t)(lap_no & 1), P.err, PKE_FULL, dead, P.wait_ns);
                         lap(PF_TWAIT);
                         const unsigned char *tb = ring_mem + (size_t)slot * PK_SLOT_BYTES;
                         for (int k0 = lane * VEC; k0 < kc_len; k0 += 32 * VEC * KSB) {
@@ -829,7 +831,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
         // ---- output edge
         if (cta == 0) {
             consumer_bar();
-            if (tid == 0) st_release(T.flag_out + j, r + 1);
+            if (tid == 0 && P.withhold_partition != p) st_release(T.flag_out + j, r + 1);
         }
     }
     // positions advance by the passes of this launch

@@ -40,7 +40,8 @@ class ModelShape(ctypes.Structure):
 
 class Options(ctypes.Structure):
     _fields_ = [("page_tokens", ctypes.c_int), ("kv_pool_tokens", ctypes.c_int), ("attn_splits", ctypes.c_int),
-                ("rounds_per_graph", ctypes.c_int), ("kv_cache_bf16", ctypes.c_int), ("prefill_mode", ctypes.c_int), ("tc_min_group", ctypes.c_int), ("scheduler", ctypes.c_int)]
+                ("rounds_per_graph", ctypes.c_int), ("kv_cache_bf16", ctypes.c_int), ("prefill_mode", ctypes.c_int), ("tc_min_group", ctypes.c_int), ("wait_limit_ms", ctypes.c_int), ("debug_withhold_handoff", ctypes.c_int),
+                ("scheduler", ctypes.c_int)]
 
 
 class Stats(ctypes.Structure):
@@ -112,14 +113,16 @@ class Context:
 
     def __init__(self, shape, part_bounds: Sequence[int], n_samples: int, page_tokens: int = 0,
                  kv_pool_tokens: int = 0, attn_splits: int = 0, rounds_per_graph: int = 0, scheduler: int = 0,
-                 kv_cache_bf16: int = 0, prefill_mode: int = 0, tc_min_group: int = 0):
+                 kv_cache_bf16: int = 0, prefill_mode: int = 0, tc_min_group: int = 0,
+                 wait_limit_ms: int = 0, debug_withhold_handoff: int = 0):
         self._h = None
         self.shape = shape
         self.K = len(part_bounds) - 1
         self.n_samples = n_samples
         cs = ModelShape(**{n: getattr(shape, n) for n, _ in ModelShape._fields_})
         bounds = (ctypes.c_int * len(part_bounds))(*part_bounds)
-        opts = Options(page_tokens, kv_pool_tokens, attn_splits, rounds_per_graph, kv_cache_bf16, prefill_mode, tc_min_group, scheduler)
+        opts = Options(page_tokens, kv_pool_tokens, attn_splits, rounds_per_graph, kv_cache_bf16, prefill_mode, tc_min_group,
+                       wait_limit_ms, debug_withhold_handoff, scheduler)
         h = ctypes.c_void_p()
         rc = lib().mdi_create(ctypes.byref(cs), bounds, self.K, n_samples, ctypes.byref(opts), ctypes.byref(h))
         if rc != MDI_OK:

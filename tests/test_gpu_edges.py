@@ -98,3 +98,35 @@ def test_generate_dev_and_prefill_dev_match_host_forms():
             res.append(ctx.generate(3, 12))
         ctx.close()
     assert np.array_equal(res[0], res[1])
+
+
+def test_a_withheld_handoff_times_out_and_the_context_survives():
+    """Failure detection without faulting anything: partition 0 is told to withhold its output handoff once, the
+    waits are given 50 ms, the call must come back with MDI_ERR_TIMEOUT (not hang), the samples are reset, and
+    the same context then generates correctly."""
+    import time
+    from paper_2505_18164_b200 import mdi
+    shape = tiny_shape("gpt", I.DT_F32, L=3, d=64, H=4, V=97, C=48)
+    orc, w = make_oracle(shape, seed=9, std=0.06)
+    ctx = mdi.Context(shape, [0, 1, 2, 3], 3, scheduler=2, wait_limit_ms=50, debug_withhold_handoff=1)
+    ctx.load_all(w)
+    prompts = I.make_prompts(97, 3, 5, seed=12)
+    for s in range(3):
+        ctx.prefill(s, prompts[s])
+    t0 = time.time()
+    with pytest.raises(mdi.MdiError) as e:
+        ctx.generate(3, 8)
+    assert e.value.code == mdi.ERR_TIMEOUT and "gave up waiting" in str(e.value)
+    assert time.time() - t0 < 20.0
+    assert ctx.stats().kv_pages_in_use[0] == 0                      # every sample was reset
+    with pytest.raises(mdi.MdiError) as e:
+        ctx.generate(3, 2)
+    assert e.value.code == mdi.ERR_STATE                            # nothing is prefilled any more
+    toks, _, margins = oracle_reference(orc, prompts, 8)
+    for s in range(3):
+        ctx.prefill(s, prompts[s])
+    out = ctx.generate(3, 8)                                        # the hook was one-shot: this run is normal
+    for s in range(3):
+        n = _safe_prefix(toks[s], margins[s], 1e-4)
+        assert list(out[s, :n]) == toks[s][:n]
+    ctx.close()
