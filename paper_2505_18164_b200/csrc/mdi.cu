@@ -796,6 +796,22 @@ int pk_fill_phases(mdi_ctx *c) {
     return MDI_OK;
 }
 
+// The kernel counts the weight tiles a block has consumed in 32 bits: an upper bound for one launch.
+bool pk_tile_count_fits(const mdi_ctx *c, int n_pass, int G) {
+    double worst = 0;
+    for (int p = 0; p < c->K; ++p) {
+        double per_step = 0;
+        for (int i = 0; i < c->pk_phase_count[p]; ++i) {
+            const PkPhase &q = c->pk_phases_host[c->pk_phase_begin[p] + i];
+            if (q.kind == PK_ATTN) continue;
+            const double chunks = std::ceil((double)q.in_dim * c->esize / (PK_SLOT_BYTES / PK_SEGS));
+            per_step += (std::floor((double)q.n_blocks / c->pk_teams_host[p].n_cta) + 1) * chunks;
+        }
+        worst = std::max(worst, per_step);
+    }
+    return worst * (double)n_pass * G < 2.0e9;
+}
+
 // One cooperative launch that runs n_pass passes of the recurrent pipeline for samples 0..n_samples-1.
 int pk_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     const mdi_model_shape &s = c->s;
@@ -813,6 +829,8 @@ int pk_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     P.logits = c->logits; P.head_pv = c->head_pv; P.head_pi = c->head_pi; P.cur_tok = c->cur_tok; P.tok_log = c->tok_log;
     P.gen_count = c->gen_count; P.teacher = c->teacher; P.n_teacher = c->n_teacher; P.log_stride = s.n_ctx; P.err = c->pk_err;
     P.prof = c->pk_prof_on ? c->pk_prof : nullptr;
+    P.hd_shift = 0;
+    while ((1 << P.hd_shift) < s.head_dim) ++P.hd_shift;
     P.wait_ns = c->o.wait_limit_ms > 0 ? (unsigned long long)c->o.wait_limit_ms * 1000000ull : PK_WAIT_NS;
     P.withhold_partition = c->withhold_once;
     c->withhold_once = -1;
@@ -1283,7 +1301,7 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
     const long t_total = total ? total + K - 1 : 0;
     long t = 0;
     const bool use_pk = c->pk_ok && c->scheduler != 1 && (n_samples + G - 1) / G <= PK_MAXNB &&
-                        !(c->pf_tc && (n_samples + G - 1) / G >= c->tc_min_group);
+                        !(c->pf_tc && (n_samples + G - 1) / G >= c->tc_min_group) && pk_tile_count_fits(c, n_pass, G);
     if (c->scheduler == 2 && !use_pk) return fail(c, MDI_ERR_SHAPE, "persistent scheduler unavailable for this call");
     if (t_total && use_pk) {
         if ((rc = pk_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;

@@ -71,6 +71,7 @@ struct PkParams {
     const int *teacher, *n_teacher;
     int log_stride;
     int *err;
+    int hd_shift;               // log2(head_dim)
     unsigned long long wait_ns; // limit of every wait
     int withhold_partition;     // >= 0: that partition never raises its output flags (checks the time-out path)
     unsigned long long *prof; // optional [grid][PK_PROF_N] nanoseconds per category (thread 0 and the producer of each block)
@@ -180,8 +181,9 @@ __device__ __forceinline__ int pk_seg_row(const PkPhase &ph, int rope, int hd, i
     second = false;
     if (ph.kind == PK_GATEUP) { second = i >= 8; return blk * 8 + (i & 7); }
     if (ph.kind == PK_QKV && rope) {
-        const int u = blk * 8 + (i & 7), half = hd >> 1;
-        return (u / half) * hd + (u % half) + (i >= 8 ? half : 0);
+        // head_dim is a power of two: u / half and u % half as shift and mask
+        const int u = blk * 8 + (i & 7), half = hd >> 1, hs = 31 - __clz(half);
+        return ((u >> hs) << (hs + 1)) + (u & (half - 1)) + (i >= 8 ? half : 0);
     }
     return blk * PK_SEGS + i;
 }
@@ -284,22 +286,25 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
         // =========================== producer ===========================
         // All 32 lanes walk the schedule; lane 0 waits for the ring slot and posts the byte count, then either
         // lane 0 copies the whole tile at once (rows contiguous in memory) or lanes 0..15 copy one segment each.
-        long seq = 0;
+        unsigned seq = 0;   // tiles issued so far (fits 32 bits: checked on the host)
+        int pslot = 0;
+        uint32_t ppar = 0;
         for (long v = 0; v < total_slots && !dead; ++v) {
             if ((int)(v % K) >= G) continue;
             for (int pi = 0; pi < T.n_phases && !dead; ++pi) {
                 const PkPhase ph = phases[pi];
                 if (ph.kind == PK_ATTN) continue;
                 const bool whole = ph.in_dim <= KC && ph.kind != PK_GATEUP && !(ph.kind == PK_QKV && P.rope);
-                const int b0 = (int)((long)cta * ph.n_blocks / T.n_cta), b1 = (int)((long)(cta + 1) * ph.n_blocks / T.n_cta);
+                const int b0 = (int)((unsigned)cta * (unsigned)ph.n_blocks / (unsigned)T.n_cta), b1 = (int)((unsigned)(cta + 1) * (unsigned)ph.n_blocks / (unsigned)T.n_cta);
                 for (int blk = b0; blk < b1 && !dead; ++blk)
                     for (int kc0 = 0; kc0 < ph.in_dim; kc0 += KC, ++seq) {
                         const int kc_len = min(KC, ph.in_dim - kc0);
                         const uint32_t seg_bytes = (uint32_t)kc_len * ES;
-                        const int slot = (int)(seq % NS);
-                        const uint32_t par = (uint32_t)((seq / NS) & 1);
+                        const int slot = pslot;
+                        const uint32_t par = ppar;
+                        if (++pslot == NS) { pslot = 0; ppar ^= 1u; }
                         lap(PF_PROD_TOTAL);
-                        if (lane == 0 && seq >= NS) wait_mbar(empty_base + 8 * slot, par ^ 1, P.err, PKE_EMPTY, dead, P.wait_ns);
+                        if (lane == 0 && seq >= (unsigned)NS) wait_mbar(empty_base + 8 * slot, par ^ 1, P.err, PKE_EMPTY, dead, P.wait_ns);
                         dead = __shfl_sync(0xffffffffu, (int)dead, 0) != 0;
                         lap(PF_PROD_WAIT);
                         if (dead) break;
@@ -332,7 +337,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
         if (dead && lane == 0) {
             // copies already issued target this block's shared memory: give them bounded time to land
             const unsigned long long t0 = pk_now();
-            for (long q = seq > NS ? seq - NS : 0; q < seq; ++q)
+            for (unsigned q = seq > (unsigned)NS ? seq - NS : 0; q < seq; ++q)
                 while (!mbar_try_wait(full_base + 8 * (int)(q % NS), (uint32_t)((q / NS) & 1)) && pk_now() - t0 < 100000000ull) {}
         }
         return;
@@ -340,7 +345,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
 
     // =========================== consumers ===========================
     unsigned bar_epoch = 0;
-    long tile_seq = 0; // tiles this block has consumed so far (same in every consumer warp)
+    unsigned tile_seq = 0; // tiles this block has consumed so far (same in every consumer warp; fits 32 bits)
     auto team_barrier = [&]() {
         consumer_bar();
         if (tid == 0) {
@@ -389,7 +394,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                 // ---------------- attention over the cache: items (item, head, split) dealt to the team's blocks
                 constexpr int EPL = 16 / (int)sizeof(KT);
                 const int LPR = hd / EPL, RPW = 32 / LPR, NG = PK_CWARPS * RPW;
-                const int sub = lane % LPR, grp = lane / LPR;
+                const int sub = lane & (LPR - 1), grp = lane >> (31 - __clz(LPR));
                 const int n_items = nb * P.n_head * T.n_split;
                 for (int it = cta; it < n_items; it += T.n_cta) {
                     const int sp = it % T.n_split, h = (it / T.n_split) % P.n_head, b = it / (T.n_split * P.n_head);
@@ -525,7 +530,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                     }
                 } else if (ph.kind == PK_OUT) {
                     for (int i = tid; i < Kd; i += PK_CTHREADS) {
-                        const int h = i / hd;
+                        const int h = i >> P.hd_shift;
                         xs[b * Kpad + xs_perm<ES>(i)] =
                             live ? pk_merge_splits(T.part + ((size_t)b * P.n_head + h) * T.n_split * (hd + 2), T.n_split, hd, i - h * hd) : 0.f;
                     }
@@ -596,7 +601,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
             //  ROWS = 16: a warp owns whole tiles (row blocks b0+w, b0+w+8, ...), so up to 8 tiles are in work
             //            at once (the long output-layer phase).
             // Either way the totals end up one row per even lane: lane 2i finishes the warp's i-th row.
-            const int b0 = (int)((long)cta * ph.n_blocks / T.n_cta), b1 = (int)((long)(cta + 1) * ph.n_blocks / T.n_cta);
+            const int b0 = (int)((unsigned)cta * (unsigned)ph.n_blocks / (unsigned)T.n_cta), b1 = (int)((unsigned)(cta + 1) * (unsigned)ph.n_blocks / (unsigned)T.n_cta);
             const int n_chunks = (Kd + KC - 1) / KC;
             float best_v[NB];
             int best_i[NB];
@@ -633,7 +638,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                         for (int b = 0; b < NB; ++b) {
                             if (b < nb && (ph.kind == PK_OUT || ph.kind == PK_FC2)) xr[b] = __ldcg(xres + (size_t)b * d + row);
                             if (b < nb && ph.kind == PK_QKV && P.rope && row < qw + kw) {
-                                const int i = (row % hd) & ((hd >> 1) - 1);
+                                const int i = row & ((hd >> 1) - 1);
                                 rc[b] = P.rope_cos[(size_t)pos[b] * (hd >> 1) + i];
                                 rs[b] = P.rope_sin[(size_t)pos[b] * (hd >> 1) + i];
                             }
@@ -644,10 +649,10 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                     for (int r2 = 0; r2 < ROWS; ++r2)
 #pragma unroll
                         for (int b = 0; b < NB; ++b) acc[r2][b][0] = acc[r2][b][1] = 0.f;
-                    const long seq0 = tile_seq + (long)(blk - b0) * n_chunks;
+                    const unsigned seq0 = tile_seq + (unsigned)(blk - b0) * (unsigned)n_chunks;
                     for (int c = 0; c < n_chunks; ++c) {
-                        const long seq = seq0 + c;
-                        const int slot = (int)(seq % NS), lap_no = (int)(seq / NS);
+                        const unsigned seq = seq0 + (unsigned)c;
+                        const int lap_no = (int)(seq / (unsigned)NS), slot = (int)(seq - (unsigned)lap_no * (unsigned)NS);
                         const int kc0 = c * KC, kc_len = min(KC, Kd - kc0);
                         // a parity test is only meaningful once every earlier tile of this slot has been consumed
                         // (warps run ahead of one another); then wait for this tile's bytes to land
@@ -745,7 +750,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                                 else {
                                     const int rk = row - qw, which = rk >= kw, rl = rk - which * kw;
                                     KT *dst = reinterpret_cast<KT *>(T.kv.pool) + page_off[b] +
-                                              ((size_t)(which * T.kv.n_kv_head + rl / hd) * T.kv.page_tokens + (pos[b] & (T.kv.page_tokens - 1))) * hd + rl % hd;
+                                              ((size_t)(which * T.kv.n_kv_head + (rl >> P.hd_shift)) * T.kv.page_tokens + (pos[b] & (T.kv.page_tokens - 1))) * hd + (rl & (hd - 1));
                                     kv_store<KT>(dst, y);
                                 }
                             } else if (ph.kind == PK_FC1) {
@@ -765,7 +770,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
             };
             if (b1 - b0 >= 6) run_tiles(std::integral_constant<int, 16>{});
             else run_tiles(std::integral_constant<int, 2>{});
-            tile_seq += (long)(b1 - b0) * n_chunks;
+            tile_seq += (unsigned)(b1 - b0) * (unsigned)n_chunks;
             lap(PF_TILES);
 
             if (ph.kind == PK_HEAD) {
