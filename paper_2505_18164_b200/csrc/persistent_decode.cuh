@@ -85,8 +85,8 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+__device__ __forceinline__ void mbar_arrive(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(full_base + 8 * s, 1);
-            mbar_init(empty_base + 8 * s, 1);
+            mbar_init(empty_base + 8 * s, PK_CWARPS); // one arrival per consumer warp (a warp that owns a tile brings all 8)
         }
         *s_dead = 0;
         for (int s = 0; s < PK_MAX_SLOTS; ++s) s_cons[s] = 0;
@@ -700,8 +700,12 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                                 }
                             }
                         }
-                        if constexpr (SHARED) consumer_bar(); else __syncwarp();
-                        if (lane == 0 && (!SHARED || warp == 0)) { s_cons[slot] = lap_no + 1; mbar_arrive(empty_base + 8 * slot); }
+                        __syncwarp();
+                        if (lane == 0) {
+                            // s_cons: "tile lap_no of this slot has landed" (any consumer that saw it may say so)
+                            if (!SHARED || warp == 0) s_cons[slot] = lap_no + 1;
+                            mbar_arrive(empty_base + 8 * slot, SHARED ? 1u : (uint32_t)PK_CWARPS);
+                        }
                         lap(PF_TCOMP);
                     }
                     // reduce across lanes: lane 2i (and 2i+1) ends with the total of the warp's i-th row
