@@ -160,6 +160,17 @@ int mdi_step(mdi_ctx *ctx, int partition, int slot, const void *act_in_dev, void
 int mdi_generate(mdi_ctx *ctx, int n_samples, int n_new_tokens, int32_t *out_tokens_host);
 int mdi_generate_dev(mdi_ctx *ctx, int n_samples, int n_new_tokens, int32_t *out_tokens_dev);
 
+/* Token choice.  The paper samples the next token from the probability mass function given by the logits
+ * (Section III-B); the default here is the greedy argmax.  temperature > 0 switches to sampling: the top_k
+ * (1..64) most likely tokens are kept (larger logit first, lower id first on ties), p_j = exp((l_j - l_0) /
+ * temperature) in fp64, and token j is chosen when the running sum in that order first exceeds u * sum(p),
+ * where u in [0,1) is a counter-based uniform of (seed, sample, index of the output-layer evaluation counted
+ * from the prefill): u = (h >> 11) / 2^53, h = mix(mix(seed ^ (sample << 32)) + index), mix = the splitmix64
+ * output function.  The same (seed, sample, index) always gives the same u, so a run can be reproduced.
+ * temperature <= 0 returns to greedy.  Sampling calls run on the stream scheduler.  mdi_step keeps the argmax.
+ * Errors: ARG (top_k out of range). */
+int mdi_set_sampling(mdi_ctx *ctx, float temperature, int top_k, uint64_t seed);
+
 /* Logits (fp32[vocab]) of the sample's most recent output-layer evaluation, copied to host. */
 int mdi_get_logits(mdi_ctx *ctx, int sample, float *out_host);
 

@@ -24,6 +24,7 @@ the starter, the last of which is not fed back.
 from __future__ import annotations
 
 import ctypes
+import math
 import os
 import subprocess
 from collections import deque
@@ -158,6 +159,42 @@ def argmax(x) -> int:
     return lib().orc_argmax(_p(x), x.size)
 
 
+# ---- sampling from the pmf (Section III-B: "a probability mass function that is then sampled") ----------
+
+_M64 = (1 << 64) - 1
+
+
+def splitmix64_mix(z: int) -> int:
+    """Output function of the splitmix64 generator (Steele, Lea, Flood 2014), on a 64-bit state z."""
+    z = (z + 0x9E3779B97F4A7C15) & _M64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return z ^ (z >> 31)
+
+
+def sample_uniform(seed: int, sample: int, index: int) -> float:
+    """Counter-based uniform in [0, 1) for (seed, sample, index of the output-layer evaluation)."""
+    h = splitmix64_mix((splitmix64_mix((seed ^ (sample << 32)) & _M64) + index) & _M64)
+    return (h >> 11) / 9007199254740992.0
+
+
+def sample_top_k(logits, top_k: int, temperature: float, u: float) -> int:
+    """Keep the top_k largest logits (larger first, lower index first on ties), p_j = exp((l_j - l_0) / T) in
+    fp64, and return the first token whose running sum exceeds u * sum(p)."""
+    lg = np.asarray(logits, np.float32)
+    order = sorted(range(lg.size), key=lambda i: (-float(lg[i]), i))[:top_k]
+    p = [math.exp((float(lg[i]) - float(lg[order[0]])) / float(temperature)) for i in order]
+    z = 0.0
+    for v in p:
+        z += v
+    target, c = u * z, 0.0
+    for i, v in zip(order, p):
+        c += v
+        if c > target:
+            return i
+    return order[-1]
+
+
 # ---- model ----------------------------------------------------------------------------------
 
 class Cache:
@@ -235,11 +272,13 @@ class Oracle:
         return seq[len(prompt):], np.stack(logits)
 
     def generate_sequential(self, prompt: Sequence[int], n_new: int, bounds: Sequence[int] = None,
-                            forced: Sequence[int] = None):
+                            forced: Sequence[int] = None, sampler=None):
         """One sample, cached greedy decoding through the chunks given by ``bounds``.
 
         ``forced``: tokens fed back in place of the argmax (the argmax is still
         returned), so that a second implementation can be compared step by step.
+        ``sampler``: None for greedy, or (temperature, top_k, seed, sample index): the i-th token is then drawn
+        with sample_top_k and the uniform sample_uniform(seed, sample index, i).
         Returns (tokens [n_new], logits [n_new][V])."""
         L = self.shape.n_layer
         bounds = list(bounds) if bounds is not None else [0, L]
@@ -254,7 +293,11 @@ class Oracle:
             pos += len(feed)
             lg = self.head(X[-1])
             logits.append(lg)
-            toks.append(argmax(lg))
+            if sampler is None:
+                toks.append(argmax(lg))
+            else:
+                temperature, top_k, seed, smp = sampler
+                toks.append(sample_top_k(lg, top_k, temperature, sample_uniform(seed, smp, i)))
             feed = [toks[-1] if forced is None else int(forced[i])]
         return toks, np.stack(logits)
 

@@ -115,6 +115,9 @@ struct mdi_ctx {
     std::map<std::tuple<const void *, uint64_t, uint64_t, uint32_t>, CUtensorMap> tmaps;
     // persistent decode kernel
     bool pk_ok = false, pk_prof_on = false, pk_tables_stale = true;
+    float temperature = 0.f; // > 0: sample from the pmf (top_k most likely tokens) instead of taking the argmax
+    int top_k = 0;
+    unsigned long long sample_seed = 0;
     int withhold_once = -1; // partition whose output flags the next persistent launch withholds (time-out test hook)
     int pk_slots = 0, pk_xs_floats = 0, pk_nb = 1, n_sm = 0, scheduler = 0;
     size_t pk_smem = 0;
@@ -303,6 +306,7 @@ int enqueue_head(mdi_ctx *c, const Batch &hb, const float *x_rows, const HeadReq
     if (head.update_state) {
         a.cur_tok = c->cur_tok; a.tok_log = c->tok_log; a.gen_count = c->gen_count;
         a.teacher = c->teacher; a.n_teacher = c->n_teacher;
+        a.temperature = c->temperature; a.top_k = c->top_k; a.sample_seed = c->sample_seed;
     }
     return linear(c, LIN_HEAD, a, hb, st);
 }
@@ -1300,7 +1304,7 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
     const long total = (long)n_pass * K;        // phase slots per partition
     const long t_total = total ? total + K - 1 : 0;
     long t = 0;
-    const bool use_pk = c->pk_ok && c->scheduler != 1 && (n_samples + G - 1) / G <= PK_MAXNB &&
+    const bool use_pk = c->pk_ok && c->scheduler != 1 && c->temperature <= 0.f && (n_samples + G - 1) / G <= PK_MAXNB &&
                         !(c->pf_tc && (n_samples + G - 1) / G >= c->tc_min_group) && pk_tile_count_fits(c, n_pass, G);
     if (c->scheduler == 2 && !use_pk) return fail(c, MDI_ERR_SHAPE, "persistent scheduler unavailable for this call");
     if (t_total && use_pk) {
@@ -1382,6 +1386,18 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
 
 int mdi_generate(mdi_ctx *c, int n_samples, int n_new, int32_t *out_host) { return generate_impl(c, n_samples, n_new, out_host, false); }
 int mdi_generate_dev(mdi_ctx *c, int n_samples, int n_new, int32_t *out_dev) { return generate_impl(c, n_samples, n_new, out_dev, true); }
+
+int mdi_set_sampling(mdi_ctx *c, float temperature, int top_k, uint64_t seed) {
+    if (!c) return MDI_ERR_ARG;
+    if (temperature > 0.f && (top_k < 1 || top_k > 64)) return fail(c, MDI_ERR_ARG, "top_k must be between 1 and 64 when sampling");
+    if (!(temperature == temperature)) return fail(c, MDI_ERR_ARG, "temperature is not a number");
+    CU(cudaSetDevice(c->dev));
+    CU(cudaDeviceSynchronize());
+    c->temperature = temperature > 0.f ? temperature : 0.f;
+    c->top_k = top_k;
+    c->sample_seed = seed;
+    return MDI_OK;
+}
 
 int mdi_get_logits(mdi_ctx *c, int sample, float *out_host) {
     if (!c || !out_host) return fail(c, MDI_ERR_ARG, "null argument");

@@ -80,6 +80,10 @@ struct LinArgs {
     const int *teacher; // optional [n_slots][log_stride]
     const int *n_teacher;
     int log_stride;
+    // sampling from the pmf instead of the argmax (temperature > 0): top_k most likely tokens, counter-based uniform
+    float temperature;
+    int top_k;
+    unsigned long long sample_seed;
 };
 
 // ---- 16-byte weight vectors ------------------------------------------------------------------
@@ -161,6 +165,67 @@ __global__ void k_embed(const WT *wte, const WT *wpe, int d, int vocab, const in
     }
 }
 
+// ---- sampling ---------------------------------------------------------------------------------
+// Counter-based uniform in [0,1) for (seed, sample, step): two rounds of the splitmix64 output function.
+__device__ __forceinline__ unsigned long long sm64(unsigned long long z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+__device__ __forceinline__ double sample_uniform(unsigned long long seed, int sample, int step) {
+    const unsigned long long h = sm64(sm64(seed ^ ((unsigned long long)(unsigned)sample << 32)) + (unsigned long long)(unsigned)step);
+    return (double)(h >> 11) * (1.0 / 9007199254740992.0);
+}
+
+// Whole block (LIN_THREADS threads): the top_k (<= 64) largest of lg[0..n) in the order "larger value first,
+// lower index first on ties", then one draw from softmax(values / temperature) restricted to them, with the
+// cumulative sum taken in that order in fp64.  Returns the chosen index (valid in every thread).
+__device__ int block_sample_top_k(const float *lg, int n, int top_k, float temperature, double u, float *sv /*[64]*/, int *si /*[64]*/,
+                                  float *wv /*[LIN_WARPS]*/, int *wi /*[LIN_WARPS]*/, int *result) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float pv = INFINITY;
+    int pi = -1;
+    for (int r = 0; r < top_k; ++r) {
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int i = tid; i < n; i += LIN_THREADS) {
+            const float v = __ldcg(lg + i);
+            const bool after_prev = v < pv || (v == pv && i > pi);
+            if (after_prev && (v > bv || (v == bv && i < bi))) { bv = v; bi = i; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float v = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int ix = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (v > bv || (v == bv && ix < bi)) { bv = v; bi = ix; }
+        }
+        if (lane == 0) { wv[warp] = bv; wi[warp] = bi; }
+        __syncthreads();
+        bv = wv[0];
+        bi = wi[0];
+#pragma unroll
+        for (int w = 1; w < LIN_WARPS; ++w)
+            if (wv[w] > bv || (wv[w] == bv && wi[w] < bi)) { bv = wv[w]; bi = wi[w]; }
+        if (tid == 0) { sv[r] = bv; si[r] = bi; }
+        pv = bv;
+        pi = bi;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        const int k = top_k < n ? top_k : n;
+        double z = 0.0, p[64];
+        for (int j = 0; j < k; ++j) { p[j] = exp(((double)sv[j] - (double)sv[0]) / (double)temperature); z += p[j]; }
+        const double target = u * z;
+        double c = 0.0;
+        int pick = si[k - 1];
+        for (int j = 0; j < k; ++j) { c += p[j]; if (c > target) { pick = si[j]; break; } }
+        *result = pick;
+    }
+    __syncthreads();
+    return *result;
+}
+
 // ---- weight-streaming linear layer ------------------------------------------------------------
 // Each warp owns one unit of two weight rows and streams them once with 16-byte loads; the NB
 // input vectors sit in shared memory as fp32 (normalised in the prologue where asked).
@@ -171,6 +236,9 @@ __global__ void __launch_bounds__(LIN_THREADS) k_linear(const LinArgs a, const B
     __shared__ float hv[LIN_WARPS][NB];
     __shared__ int hi_[LIN_WARPS][NB];
     __shared__ bool is_last;
+    __shared__ float smp_v[64];
+    __shared__ int smp_i[64], smp_w[LIN_WARPS], smp_res;
+    __shared__ float smp_wv[LIN_WARPS];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int K = a.in_dim;
 
@@ -340,7 +408,28 @@ __global__ void __launch_bounds__(LIN_THREADS) k_linear(const LinArgs a, const B
         __syncthreads();
         if (tid == 0) is_last = atomicAdd(a.ticket, 1u) == gridDim.x - 1;
         __syncthreads();
-        if (is_last) {
+        if (is_last && a.temperature > 0.f && a.gen_count) {
+            // draw from the pmf instead of taking the argmax: one item at a time, the whole block on each
+            __threadfence();
+            for (int i = 0; i < bt.n; ++i) {
+                const int slot = bt.slot[i];
+                const int g = a.gen_count[slot];
+                const float *lg = a.logits + (size_t)(a.logits_by_item ? i : slot) * a.n_rows;
+                const int tok = block_sample_top_k(lg, a.n_rows, a.top_k, a.temperature, sample_uniform(a.sample_seed, slot, g), smp_v, smp_i,
+                                                   smp_wv, smp_w, &smp_res);
+                __syncthreads();
+                if (tid == 0) {
+                    if (a.tok_out) a.tok_out[i] = tok;
+                    if (g < a.log_stride) a.tok_log[(size_t)slot * a.log_stride + g] = tok;
+                    int feed = tok;
+                    if (a.teacher && g < a.n_teacher[slot]) feed = a.teacher[(size_t)slot * a.log_stride + g];
+                    a.cur_tok[slot] = feed;
+                    a.gen_count[slot] = g + 1;
+                }
+                __syncthreads();
+            }
+            if (tid == 0) *a.ticket = 0u;
+        } else if (is_last) {
             __threadfence();
             for (int i = warp; i < bt.n; i += LIN_WARPS) {
                 float bv = -INFINITY;

@@ -21,7 +21,7 @@ _ERR_NAMES = {ERR_ARG: "MDI_ERR_ARG", ERR_SHAPE: "MDI_ERR_SHAPE", ERR_OOM: "MDI_
               ERR_STATE: "MDI_ERR_STATE", ERR_TIMEOUT: "MDI_ERR_TIMEOUT", ERR_CUDA: "MDI_ERR_CUDA"}
 
 EXPORTS = ["mdi_create", "mdi_destroy", "mdi_load_weights", "mdi_prefill", "mdi_prefill_dev", "mdi_step",
-           "mdi_generate", "mdi_generate_dev", "mdi_get_logits", "mdi_set_teacher_tokens", "mdi_reset_sample",
+           "mdi_generate", "mdi_generate_dev", "mdi_get_logits", "mdi_set_sampling", "mdi_set_teacher_tokens", "mdi_reset_sample",
            "mdi_get_stats", "mdi_get_partition_times", "mdi_memory_bytes", "mdi_sync", "mdi_last_error", "mdi_greedy_argmax_static"]
 
 
@@ -75,6 +75,7 @@ def lib():
         L.mdi_generate.argtypes = [vp, ci, ci, vp]
         L.mdi_generate_dev.argtypes = [vp, ci, ci, vp]
         L.mdi_get_logits.argtypes = [vp, ci, vp]
+        L.mdi_set_sampling.argtypes = [vp, ctypes.c_float, ci, ctypes.c_uint64]
         L.mdi_set_teacher_tokens.argtypes = [vp, ci, vp, ci]
         L.mdi_reset_sample.argtypes = [vp, ci]
         L.mdi_get_stats.argtypes = [vp, ctypes.POINTER(Stats)]
@@ -178,6 +179,9 @@ class Context:
         out = np.empty(self.shape.vocab, np.float32)
         self._check(lib().mdi_get_logits(self._h, sample, out.ctypes.data))
         return out
+
+    def set_sampling(self, temperature: float, top_k: int, seed: int):
+        self._check(lib().mdi_set_sampling(self._h, temperature, top_k, seed))
 
     def set_teacher_tokens(self, sample: int, tokens: Sequence[int]):
         t = np.ascontiguousarray(tokens, np.int32)

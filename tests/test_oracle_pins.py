@@ -345,3 +345,57 @@ def test_forced_tokens_only_change_what_is_fed_back():
     # equals recomputing from the forced history
     full = orc.full_logits([1, 2, 3] + forced[:4])
     assert np.abs(full[2:] - l3).max() <= 1e-5
+
+
+# ---------------- sampling ----------------------------------------------------------------------
+
+def test_splitmix64_known_answers():
+    """First outputs of splitmix64 seeded with 1234567, as published with the reference implementation."""
+    x, got = 1234567, []
+    for _ in range(5):
+        got.append(O.splitmix64_mix(x))
+        x = (x + 0x9E3779B97F4A7C15) & ((1 << 64) - 1)
+    assert got == [6457827717110365317, 3203168211198807973, 9817491932198370423, 4593380528125082431, 16408922859458223821]
+
+
+def test_sample_uniform_is_a_pure_function_and_roughly_uniform():
+    u = [O.sample_uniform(7, s, i) for s in range(4) for i in range(2000)]
+    assert all(0.0 <= v < 1.0 for v in u)
+    assert O.sample_uniform(7, 2, 5) == O.sample_uniform(7, 2, 5) != O.sample_uniform(7, 5, 2)
+    a = np.array(u)
+    assert abs(a.mean() - 0.5) < 0.01 and abs(a.var() - 1 / 12) < 0.005
+    hist, _ = np.histogram(a, bins=10, range=(0, 1))
+    assert hist.min() > 0.85 * a.size / 10 and hist.max() < 1.15 * a.size / 10
+
+
+def test_sample_top_k_special_cases_and_frequencies():
+    lg = np.array([0.1, 2.0, -1.0, 2.0, 0.5, 1.5], np.float32)
+    for u in (0.0, 0.3, 0.999):
+        assert O.sample_top_k(lg, 1, 0.7, u) == 1                       # top-1 is the argmax, lowest index on ties
+    assert O.sample_top_k(lg, 3, 1.0, 0.0) == 1                         # u = 0 -> the most likely token
+    assert O.sample_top_k(lg, 3, 1.0, 1.0 - 1e-12) == 5                 # u -> 1 -> the last kept token (order 1, 3, 5)
+    assert O.sample_top_k(lg, 2, 1.0, 0.49) == 1 and O.sample_top_k(lg, 2, 1.0, 0.51) == 3   # equal logits: halves
+    # empirical frequencies over a grid of u equal softmax(l / T) restricted to the kept tokens
+    T, k = 0.8, 4
+    order = [1, 3, 5, 4]
+    p = np.exp((lg[order].astype(np.float64) - 2.0) / T)
+    p /= p.sum()
+    n = 20000
+    counts = {i: 0 for i in order}
+    for j in range(n):
+        counts[O.sample_top_k(lg, k, T, (j + 0.5) / n)] += 1
+    for i, pi in zip(order, p):
+        assert abs(counts[i] / n - pi) < 2e-4
+    # very low temperature concentrates on the argmax
+    assert all(O.sample_top_k(lg, 6, 1e-3, u) in (1, 3) for u in np.linspace(0, 0.999, 50))
+
+
+def test_sampled_generation_reduces_to_greedy_with_top_1():
+    shape = tiny_shape("gpt", I.DT_F32)
+    orc, _ = make_oracle(shape, std=0.2)
+    g, _ = orc.generate_sequential([1, 2, 3], 6)
+    s1, _ = orc.generate_sequential([1, 2, 3], 6, sampler=(0.9, 1, 11, 0))
+    assert s1 == g
+    s2, _ = orc.generate_sequential([1, 2, 3], 6, sampler=(1.5, 8, 11, 0))
+    s3, _ = orc.generate_sequential([1, 2, 3], 6, sampler=(1.5, 8, 11, 0))
+    assert s2 == s3                                                      # reproducible from (seed, sample, index)
