@@ -34,9 +34,9 @@ sys.path.insert(0, ROOT)
 from paper_2505_18164_b200 import inputs as I  # noqa: E402
 
 # DRAM traffic of the persistent decode kernel relative to its algorithmic bytes, from the ncu capture
-# kept with the profiler summaries of this repository (17.149 GB moved for 17.171 GB algorithmic; traffic
+# kept with the profiler summaries of this repository (17.143 GB moved for 17.171 GB algorithmic; traffic
 # grows with the number of passes like the algorithmic bytes do).  None for other workloads / schedulers.
-PK_TRAFFIC_RATIO = {"gpt2_small": 17.149 / 17.171}
+PK_TRAFFIC_RATIO = {"gpt2_small": 17.143 / 17.171}
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
