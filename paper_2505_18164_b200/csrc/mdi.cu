@@ -15,6 +15,7 @@
 #include <tuple>
 #include <vector>
 
+#include "fused_decode.cuh"
 #include "persistent_decode.cuh"
 #include "prefill_kernels.cuh"
 #include "step_kernels.cuh"
@@ -129,6 +130,28 @@ struct mdi_ctx {
     unsigned *pk_sync = nullptr; // [K][64]: word 0 team barrier, words 32.. output-edge flags
     int *pk_err = nullptr;
     unsigned long long *pk_prof = nullptr; // [n_sm][PK_PROF_N]
+    // fused-phase persistent kernel (GPT block, bf16 weights): plan made at creation, weight stream built at first use
+    bool fz_ok = false, fz_stale = true, fz_prof_on = false;
+    int fz_slots = 0, fz_nb = 1, fz_xb_stride = 0, fz_hb_stride = 0, fz_ob_stride = 0, fz_part_floats = 0, fz_grid = 0;
+    int last_kernel = 0; // which persistent kernel the last generate call used: 1 phase-per-matrix, 2 fused-phase
+    size_t fz_smem = 0;
+    std::vector<FzTeam> fz_teams_host;
+    std::vector<FzWork> fz_works_host;
+    std::vector<FzBlock> fz_blocks_host;
+    std::vector<int> fz_units_host, fz_phase_begin, fz_phase_count;
+    std::vector<std::vector<int>> fz_unit_lists; // hidden units of (block, phase B), indexed like fz_works_host
+    FzTeam *fz_teams = nullptr;
+    FzPhase *fz_phases = nullptr;
+    FzWork *fz_works = nullptr;
+    FzBlock *fz_blocks = nullptr;
+    FzSeg *fz_segs = nullptr;
+    int *fz_units = nullptr, *fz_err = nullptr;
+    int fz_kv_pps = 1;
+    uint4 *fz_stream = nullptr;
+    long long *fz_acc = nullptr;
+    unsigned *fz_sync = nullptr;
+    unsigned long long *fz_prof = nullptr;
+    int64_t fz_stream_bytes = 0;
     mdi_stats st{};
     std::string err;
 };
@@ -651,7 +674,7 @@ int pk_setup(mdi_ctx *c) {
     cudaDeviceProp prop;
     CU(cudaGetDeviceProperties(&prop, c->dev));
     c->n_sm = prop.multiProcessorCount;
-    if (c->scheduler == 1) return MDI_OK;
+    if (c->scheduler == 1 || c->scheduler == 3) return MDI_OK;
     const bool want = c->scheduler == 2;
     if (c->gmax > PK_MAXNB) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: at most %d samples per group", PK_MAXNB) : MDI_OK;
     if (K > 32 || K > c->n_sm) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: too many partitions") : MDI_OK;
@@ -850,6 +873,375 @@ int pk_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     return MDI_OK;
 }
 
+
+// ---- fused-phase persistent kernel: plan, weight stream and launch -------------------------------------
+const void *fz_func(int nb) {
+    return nb == 1 ? (const void *)k_fused_decode<1> : nb == 2 ? (const void *)k_fused_decode<2> : (const void *)k_fused_decode<4>;
+}
+
+// Plan of the fused-phase kernel: team sizes, which block serves which head of which layer, which hidden
+// units of the MLP, which rows of the output layer, so that every block streams about the same number of
+// bytes per step.  Independent of the weights' addresses.  Leaves fz_ok false when the shape does not fit
+// (not the GPT block, weights not bf16, cache not fp32, grouped-query attention, more than 4 samples per
+// group, a team smaller than the number of heads).
+int fz_setup(mdi_ctx *c) {
+    const mdi_model_shape &s = c->s;
+    const int K = c->K, d = s.d_model, hd = s.head_dim, H = s.n_head;
+    const bool want = c->scheduler == 3;
+    auto no = [&](const char *why) { return want ? fail(c, MDI_ERR_SHAPE, "fused-phase scheduler: %s", why) : MDI_OK; };
+    if (c->scheduler == 1 || c->scheduler == 2) return MDI_OK;
+    if (getenv("MDI_NO_FUSED") && !want) return MDI_OK;
+    if (s.arch != MDI_ARCH_GPT || s.weight_dtype != MDI_DTYPE_BF16 || !c->kv_f32) return no("needs the GPT block, bf16 weights and an fp32 cache");
+    if (s.n_kv_head != H || H * hd != d) return no("needs n_kv_head = n_head and n_head * head_dim = d_model");
+    if (d % 16 || s.d_ff % 16 || hd % 16) return no("widths must be multiples of 16");
+    if (d > FZ_U * PK_CTHREADS) return no("d_model above 1024");
+    if (c->gmax > FZ_MAXNB) return no("at most 4 samples per group");
+    if (K > 32) return no("too many partitions");
+    cudaDeviceProp prop;
+    CU(cudaGetDeviceProperties(&prop, c->dev));
+    const int n_sm = prop.multiProcessorCount;
+    c->fz_nb = c->gmax <= 1 ? 1 : c->gmax <= 2 ? 2 : 4;
+    const int NB = c->fz_nb;
+    // team sizes in proportion to the bytes a step streams
+    std::vector<double> bytes(K, 0.0);
+    const double layer_bytes = 2.0 * (4.0 * d * d + 2.0 * (double)s.d_ff * d);
+    for (int p = 0; p < K; ++p) {
+        bytes[p] = layer_bytes * (c->part[p].hi - c->part[p].lo);
+        if (p == K - 1) bytes[p] += 2.0 * (double)s.vocab * d;
+    }
+    std::vector<int> n_cta(K, 0);
+    {
+        const char *env = getenv("MDI_FZ_TEAM_CTAS");
+        bool from_env = false;
+        if (env) {
+            std::vector<int> v;
+            const char *q = env;
+            while (*q) { v.push_back(atoi(q)); while (*q && *q != ',') ++q; if (*q == ',') ++q; }
+            int tot = 0;
+            for (int x : v) tot += x;
+            if ((int)v.size() == K && tot <= n_sm && *std::min_element(v.begin(), v.end()) >= 1) { n_cta = v; from_env = true; }
+        }
+        if (!from_env) {
+            double tot = 0;
+            for (double b : bytes) tot += b;
+            int used = 0, big = 0;
+            for (int p = 0; p < K; ++p) if (bytes[p] > bytes[big]) big = p;
+            for (int p = 0; p < K; ++p) {
+                if (p == big) continue;
+                n_cta[p] = std::max(1, (int)std::floor(n_sm * bytes[p] / tot));
+                used += n_cta[p];
+            }
+            n_cta[big] = n_sm - used;
+        }
+    }
+    for (int p = 0; p < K; ++p) if (n_cta[p] < H) return no("a team has fewer blocks than the model has heads");
+
+    // per team: phases; per block: work items
+    c->fz_teams_host.assign(K, FzTeam{});
+    c->fz_phase_begin.assign(K, 0);
+    c->fz_phase_count.assign(K, 0);
+    c->fz_works_host.clear();
+    c->fz_unit_lists.clear();
+    c->fz_blocks_host.clear();
+    int n_phases_total = 0, first = 0, m_max = 1;
+    const double a_bytes = 2.0 * (4.0 * hd * d) + (double)NB * (s.n_ctx / 4) * hd * 8.0; // weights of one head + a guess of its cache rows
+    const double u_bytes = 2.0 * 2.0 * 16.0 * d, t_bytes = 2.0 * 16.0 * d;
+    for (int p = 0; p < K; ++p) {
+        const int n = n_cta[p], Lp = c->part[p].hi - c->part[p].lo, np = 2 * Lp + (p == K - 1 ? 1 : 0);
+        c->fz_phase_begin[p] = n_phases_total;
+        c->fz_phase_count[p] = np;
+        n_phases_total += np;
+        std::vector<double> cum(n, 0.0);
+        std::vector<std::vector<FzWork>> wk(n, std::vector<FzWork>(np, FzWork{-1, 0, 0, 0, 0, 0, 0}));
+        std::vector<std::vector<std::vector<int>>> ul(n, std::vector<std::vector<int>>(np));
+        auto least = [&](const std::vector<char> *skip) {
+            int best = -1;
+            for (int b = 0; b < n; ++b)
+                if (!(skip && (*skip)[b]) && (best < 0 || cum[b] < cum[best])) best = b;
+            return best;
+        };
+        for (int l = 0; l < Lp; ++l) {
+            std::vector<char> used(n, 0);
+            for (int h = 0; h < H; ++h) {
+                const int b = least(&used);
+                used[b] = 1;
+                wk[b][2 * l].unit = h;
+                wk[b][2 * l].n_tiles = 3 * hd / 16;
+                cum[b] += a_bytes;
+            }
+            for (int u = 0; u < s.d_ff / 16; ++u) {
+                const int b = least(nullptr);
+                ul[b][2 * l + 1].push_back(u);
+                cum[b] += u_bytes;
+            }
+            for (int b = 0; b < n; ++b) {
+                wk[b][2 * l + 1].n_tiles = (int)ul[b][2 * l + 1].size();
+                m_max = std::max(m_max, wk[b][2 * l + 1].n_tiles);
+            }
+        }
+        if (p == K - 1) {
+            const int NT = (s.vocab + 15) / 16;
+            double tot = (double)NT * t_bytes;
+            for (double x : cum) tot += x;
+            const double target = tot / n;
+            std::vector<int> give(n, 0);
+            int left = NT;
+            for (int b = 0; b < n; ++b) {
+                give[b] = std::max(0, std::min(left, (int)std::floor((target - cum[b]) / t_bytes)));
+                left -= give[b];
+                cum[b] += give[b] * t_bytes;
+            }
+            while (left > 0) { const int b = least(nullptr); ++give[b]; cum[b] += t_bytes; --left; }
+            int t0 = 0;
+            for (int b = 0; b < n; ++b) { wk[b][np - 1].n_tiles = give[b]; wk[b][np - 1].tile0 = t0; t0 += give[b]; }
+        }
+        for (int b = 0; b < n; ++b) {
+            FzBlock fb{};
+            fb.work_begin = (int)c->fz_works_host.size();
+            c->fz_blocks_host.push_back(fb);
+            for (int i = 0; i < np; ++i) { c->fz_works_host.push_back(wk[b][i]); c->fz_unit_lists.push_back(ul[b][i]); }
+        }
+        FzTeam &T = c->fz_teams_host[p];
+        T.first_cta = first; T.n_cta = n; first += n;
+        T.phase_begin = c->fz_phase_begin[p]; T.n_phases = np;
+        T.is_first = p == 0; T.is_last = p == K - 1;
+    }
+    c->fz_grid = first;
+    for (int p = 0; p < K; ++p) {
+        if (c->fz_phase_count[p] > FZ_MAX_PHASES) return no("too many blocks of the model in one partition");
+        // a block serves at most one head per layer, so it has at most Lp + 1 segments
+        if (c->part[p].hi - c->part[p].lo + 1 > FZ_MAX_SEGS) return no("too many blocks of the model in one partition");
+    }
+    for (size_t b = 0; b < c->fz_blocks_host.size(); ++b) {
+        size_t nu = 0;
+        const size_t w0 = c->fz_blocks_host[b].work_begin, w1 = b + 1 < c->fz_blocks_host.size() ? c->fz_blocks_host[b + 1].work_begin : c->fz_unit_lists.size();
+        for (size_t i = w0; i < w1; ++i) nu += c->fz_unit_lists[i].size();
+        if (nu > FZ_MAX_UNITS) return no("too many hidden units per thread block");
+    }
+    // cache rows through the ring: whole pages of one head, as many as fit a slot
+    {
+        const size_t page_kv_bytes = (size_t)2 * c->page_tokens * hd * 4;
+        if (page_kv_bytes > (size_t)FZ_SLOT_BYTES) return no("one head's rows of a cache page exceed a ring slot");
+        c->fz_kv_pps = std::min<int>(32, (int)(FZ_SLOT_BYTES / page_kv_bytes));
+    }
+    // shared memory
+    m_max = (m_max + 3) & ~3;
+    const int max_tiles = std::max(3 * hd / 16, m_max);
+    c->fz_xb_stride = d + 8; c->fz_hb_stride = 16 * m_max + 8; c->fz_ob_stride = hd + 8;
+    c->fz_part_floats = max_tiles * PK_CWARPS * 16 * NB;
+    const size_t fixed = fz_smem_layout(NB, 0, d, hd, c->fz_part_floats, c->pages_per_seq, c->fz_xb_stride, c->fz_hb_stride, c->fz_ob_stride).total;
+    const size_t budget = (size_t)prop.sharedMemPerBlockOptin;
+    if (fixed + 3 * (size_t)FZ_SLOT_BYTES > budget) return no("activations do not fit in shared memory");
+    c->fz_slots = (int)std::min<size_t>(FZ_MAX_SLOTS, (budget - fixed) / FZ_SLOT_BYTES);
+    c->fz_smem = fz_smem_layout(NB, c->fz_slots, d, hd, c->fz_part_floats, c->pages_per_seq, c->fz_xb_stride, c->fz_hb_stride, c->fz_ob_stride).total;
+    for (int nb : {1, 2, 4}) CU(cudaFuncSetAttribute(fz_func(nb), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->fz_smem));
+    int rc;
+    if ((rc = dalloc(c, &c->fz_sync, (size_t)K * 64)) != MDI_OK) return rc;
+    if ((rc = dalloc(c, &c->fz_err, 1)) != MDI_OK) return rc;
+    if ((rc = dalloc(c, &c->fz_acc, (size_t)K * 3 * FZ_MAXNB * d)) != MDI_OK) return rc;
+    c->fz_prof_on = getenv("MDI_PK_PROFILE") != nullptr;
+    if (c->fz_prof_on && (rc = dalloc(c, &c->fz_prof, (size_t)c->fz_grid * PK_PROF_N)) != MDI_OK) return rc;
+    c->fz_ok = true;
+    return MDI_OK;
+}
+
+// The weights in the order the plan consumes them: one descriptor per fragment block, gathered on the device.
+// Runs before the first fused launch and again after weights were replaced.
+int fz_build(mdi_ctx *c) {
+    if (!c->fz_stale) return MDI_OK;
+    const mdi_model_shape &s = c->s;
+    const int K = c->K, d = s.d_model, hd = s.head_dim, H = s.n_head, qw = H * hd, ks = d / 16;
+    void *old[] = {c->fz_teams, c->fz_phases, c->fz_works, c->fz_blocks, c->fz_segs, c->fz_units, c->fz_stream};
+    for (void *q : old) if (q) cudaFree(q);
+    c->fz_teams = nullptr; c->fz_phases = nullptr; c->fz_works = nullptr; c->fz_blocks = nullptr; c->fz_segs = nullptr; c->fz_units = nullptr; c->fz_stream = nullptr;
+    std::vector<FzPhase> phases;
+    std::vector<FzFbDesc> desc;
+    std::vector<FzSeg> segs;
+    c->fz_units_host.clear();
+    const void *head_w = s.tied_lm_head ? c->wte : c->lm_head;
+    auto rounds = [&](const void *W, int ld, int n_t, int n_k, auto &&row_of, auto &&col_of, int row_limit) {
+        for (int r0 = 0; r0 < n_t; r0 += PK_CWARPS) {
+            const int n_r = std::min(PK_CWARPS, n_t - r0);
+            for (int k = 0; k < n_k; ++k)
+                for (int w = 0; w < n_r; ++w) {
+                    const int row0 = row_of(r0 + w);
+                    desc.push_back(FzFbDesc{W, ld, row0, col_of(k), std::max(0, std::min(16, row_limit - row0))});
+                }
+        }
+    };
+    for (int p = 0; p < K; ++p) {
+        Partition &P = c->part[p];
+        FzTeam &T = c->fz_teams_host[p];
+        const int Lp = P.hi - P.lo, np = T.n_phases;
+        for (int l = 0; l < Lp; ++l) {
+            const LayerW &L = c->layer[P.lo + l];
+            FzPhase a{}; a.kind = FZ_A; a.layer_local = l; a.gamma = L.ln1g; a.beta = L.ln1b;
+            a.bias_in = l > 0 ? c->layer[P.lo + l - 1].b2 : nullptr; a.bias_rows = L.bqkv;
+            phases.push_back(a);
+            FzPhase b{}; b.kind = FZ_B; b.layer_local = l; b.gamma = L.ln2g; b.beta = L.ln2b; b.bias_in = L.bo; b.bias_rows = L.b1;
+            phases.push_back(b);
+        }
+        if (p == K - 1) {
+            FzPhase h{}; h.kind = FZ_HEAD; h.gamma = c->lnfg; h.beta = c->lnfb; h.bias_in = c->layer[P.hi - 1].b2;
+            phases.push_back(h);
+        }
+        T.kv = kv_view(c, P);
+        T.ring_in = p > 0 ? c->part[p - 1].ring : nullptr;
+        T.ring_out = p < K - 1 ? P.ring : nullptr;
+        T.bias_final = c->layer[P.hi - 1].b2;
+        T.pos = P.pos_dev;
+        T.bar = c->fz_sync + (size_t)p * 64;
+        T.flag_out = c->fz_sync + (size_t)p * 64 + 32;
+        T.flag_in = c->fz_sync + (size_t)((p + K - 1) % K) * 64 + 32;
+        T.acc = c->fz_acc + (size_t)p * 3 * FZ_MAXNB * d;
+        for (int b = 0; b < T.n_cta; ++b) {
+            FzBlock &FB = c->fz_blocks_host[T.first_cta + b];
+            const size_t fb_begin = desc.size();
+            FB.seg_begin = (int)segs.size();
+            FB.unit_begin = (int)c->fz_units_host.size();
+            size_t seg_fb0 = fb_begin; // first fragment block of the open segment
+            int slots_before = 0;
+            auto close_segment = [&](int kv_layer, int kv_head) {
+                FzSeg sg{};
+                sg.fb_begin = (int)(seg_fb0 - fb_begin); sg.n_fb = (int)(desc.size() - seg_fb0); sg.slots_before = slots_before;
+                sg.kv_layer = kv_layer; sg.kv_head = kv_head;
+                segs.push_back(sg);
+                slots_before += (sg.n_fb + FZ_SLOT_FB - 1) / FZ_SLOT_FB;
+                seg_fb0 = desc.size();
+            };
+            for (int i = 0; i < np; ++i) {
+                FzWork &wk = c->fz_works_host[FB.work_begin + i];
+                const std::vector<int> &ul = c->fz_unit_lists[FB.work_begin + i];
+                const bool is_head = p == K - 1 && i == np - 1;
+                const LayerW &L = c->layer[P.lo + std::min(i / 2, Lp - 1)];
+                wk.seg0 = wk.seg1 = (int)segs.size() - FB.seg_begin;
+                wk.fb0 = wk.fb1 = (int)(desc.size() - seg_fb0);
+                if (is_head) {
+                    const int t0 = wk.tile0;
+                    rounds(head_w, d, wk.n_tiles, ks, [&](int t) { return (t0 + t) * 16; }, [&](int k) { return 16 * k; }, s.vocab);
+                } else if (i % 2 == 0) {
+                    if (wk.unit < 0) continue;
+                    const int h = wk.unit, tph = hd / 16;
+                    for (int t = 0; t < wk.n_tiles; ++t)
+                        for (int k = 0; k < ks; ++k)
+                            desc.push_back(FzFbDesc{L.wqkv, d, (t / tph) * qw + h * hd + (t % tph) * 16, 16 * k, 16});
+                    close_segment(i / 2, h); // this head's cache rows follow in the ring
+                    wk.seg1 = (int)segs.size() - FB.seg_begin;
+                    wk.fb1 = 0;
+                    rounds(L.wo, qw, d / 16, hd / 16, [&](int t) { return t * 16; }, [&](int k) { return h * hd + 16 * k; }, d);
+                } else {
+                    wk.tile0 = (int)c->fz_units_host.size() - FB.unit_begin;
+                    for (int u : ul) c->fz_units_host.push_back(u);
+                    if (ul.empty()) continue;
+                    for (int u : ul)
+                        for (int k = 0; k < ks; ++k) desc.push_back(FzFbDesc{L.w1, d, u * 16, 16 * k, 16});
+                    wk.fb1 = (int)(desc.size() - seg_fb0);
+                    rounds(L.w2, s.d_ff, d / 16, (int)ul.size(), [&](int t) { return t * 16; }, [&](int k) { return ul[k] * 16; }, d);
+                }
+            }
+            close_segment(-1, -1);
+            FB.n_seg = (int)segs.size() - FB.seg_begin;
+            FB.n_units = (int)c->fz_units_host.size() - FB.unit_begin;
+            FB.n_fb = (int)(desc.size() - fb_begin);
+            FB.stream = reinterpret_cast<const uint4 *>(fb_begin); // fragment-block index for now; the address follows
+        }
+    }
+    const size_t n_fb = desc.size();
+    c->fz_stream_bytes = (int64_t)n_fb * FZ_FB_BYTES;
+    CU(cudaMalloc((void **)&c->fz_stream, std::max<size_t>(n_fb, 1) * FZ_FB_BYTES));
+    for (auto &FB : c->fz_blocks_host) FB.stream = c->fz_stream + reinterpret_cast<size_t>(FB.stream) * (FZ_FB_BYTES / 16);
+    {
+        FzFbDesc *ddesc = nullptr;
+        CU(cudaMalloc((void **)&ddesc, std::max<size_t>(n_fb, 1) * sizeof(FzFbDesc)));
+        cudaError_t e = cudaMemcpy(ddesc, desc.data(), n_fb * sizeof(FzFbDesc), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess && n_fb) {
+            k_fz_repack<<<(unsigned)((n_fb + 7) / 8), 256, 0, c->main>>>(ddesc, c->fz_stream, (long)n_fb);
+            ++c->st.kernel_launches;
+            e = cudaStreamSynchronize(c->main);
+        }
+        cudaFree(ddesc);
+        CU(e);
+    }
+    auto up = [&](auto **dst, const auto &v) -> cudaError_t {
+        using E = typename std::remove_reference<decltype(v[0])>::type;
+        cudaError_t e = cudaMalloc((void **)dst, std::max<size_t>(v.size(), 1) * sizeof(E));
+        if (e != cudaSuccess) return e;
+        return cudaMemcpy(*dst, v.data(), v.size() * sizeof(E), cudaMemcpyHostToDevice);
+    };
+    CU(up(&c->fz_teams, c->fz_teams_host));
+    CU(up(&c->fz_phases, phases));
+    CU(up(&c->fz_works, c->fz_works_host));
+    CU(up(&c->fz_blocks, c->fz_blocks_host));
+    CU(up(&c->fz_segs, segs));
+    CU(up(&c->fz_units, c->fz_units_host));
+    c->fz_stale = false;
+    return MDI_OK;
+}
+
+// The kernel counts ring slots in 32 bits per launch.
+bool fz_slot_count_fits(const mdi_ctx *c, int n_pass, int G) {
+    double worst = 0;
+    // static slots of a step plus, per head unit and sample, the slots of a full context of cache rows
+    const double kv = (double)FZ_MAXNB * (c->pages_per_seq / (double)c->fz_kv_pps + 1.0);
+    for (const auto &FB : c->fz_blocks_host) worst = std::max(worst, std::ceil((double)FB.n_fb / FZ_SLOT_FB) + FB.n_seg * (1.0 + kv));
+    return worst * (double)n_pass * G < 2.0e9;
+}
+
+int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
+    const mdi_model_shape &s = c->s;
+    int rc = fz_build(c);
+    if (rc != MDI_OK) return rc;
+    CU(cudaMemsetAsync(c->fz_sync, 0, (size_t)c->K * 64 * sizeof(unsigned), c->main));
+    CU(cudaMemsetAsync(c->fz_err, 0, sizeof(int), c->main));
+    CU(cudaMemsetAsync(c->fz_acc, 0, (size_t)c->K * 3 * FZ_MAXNB * s.d_model * sizeof(long long), c->main));
+    if (c->fz_prof_on) CU(cudaMemsetAsync(c->fz_prof, 0, (size_t)c->fz_grid * PK_PROF_N * 8, c->main));
+    FzParams P{};
+    P.d = s.d_model; P.n_head = s.n_head; P.head_dim = s.head_dim; P.d_ff = s.d_ff; P.vocab = s.vocab; P.act = s.act == MDI_ACT_GELU_ERF;
+    P.K = c->K; P.G = G; P.n_samples = n_samples; P.gmax = c->gmax; P.n_pass = n_pass; P.n_slots_ring = c->fz_slots;
+    P.xb_stride = c->fz_xb_stride; P.hb_stride = c->fz_hb_stride; P.ob_stride = c->fz_ob_stride; P.part_floats = c->fz_part_floats;
+    P.pages_per_seq = c->pages_per_seq; P.kv_pps = c->fz_kv_pps; P.segs = c->fz_segs;
+    P.eps = s.norm_eps; P.scale = 1.0f / std::sqrt((float)s.head_dim);
+    P.teams = c->fz_teams; P.phases = c->fz_phases; P.works = c->fz_works; P.blocks = c->fz_blocks; P.units = c->fz_units;
+    P.wte = c->wte; P.wpe = c->wpe; P.logits = c->logits; P.head_pv = c->head_pv; P.head_pi = c->head_pi;
+    P.cur_tok = c->cur_tok; P.tok_log = c->tok_log; P.gen_count = c->gen_count; P.teacher = c->teacher; P.n_teacher = c->n_teacher;
+    P.log_stride = s.n_ctx; P.err = c->fz_err;
+    P.wait_ns = c->o.wait_limit_ms > 0 ? (unsigned long long)c->o.wait_limit_ms * 1000000ull : PK_WAIT_NS;
+    P.withhold_partition = c->withhold_once;
+    c->withhold_once = -1;
+    P.prof = c->fz_prof_on ? c->fz_prof : nullptr;
+    // MDI_FZ_TRACE=<schedule slot>: with in-kernel timing on, thread 0 of every block also records a time stamp at every
+    // phase boundary of that slot; the stamps are written as text to MDI_FZ_TRACE_FILE after the call (a tuning aid)
+    unsigned long long *trace = nullptr;
+    if (c->fz_prof_on && getenv("MDI_FZ_TRACE") && getenv("MDI_FZ_TRACE_FILE")) {
+        CU(cudaMalloc((void **)&trace, (size_t)c->fz_grid * FZ_TRACE_N * 8));
+        CU(cudaMemsetAsync(trace, 0, (size_t)c->fz_grid * FZ_TRACE_N * 8, c->main));
+        P.trace = trace;
+        P.trace_step = atoi(getenv("MDI_FZ_TRACE"));
+    }
+    // the template parameter fixes the accumulator stride, so it is the context's group size, not this call's
+    const void *fn = fz_func(c->fz_nb);
+    void *args[] = {&P};
+    CU(cudaLaunchCooperativeKernel(fn, dim3(c->fz_grid), dim3(PK_THREADS), args, c->fz_smem, c->main));
+    ++c->st.kernel_launches;
+    c->st.stage_steps += (int64_t)c->K * n_pass * G;
+    if (trace) {
+        std::vector<unsigned long long> h((size_t)c->fz_grid * FZ_TRACE_N);
+        cudaStreamSynchronize(c->main);
+        cudaMemcpy(h.data(), trace, h.size() * 8, cudaMemcpyDeviceToHost);
+        cudaFree(trace);
+        if (FILE *f = fopen(getenv("MDI_FZ_TRACE_FILE"), "w")) {
+            for (int b = 0; b < c->fz_grid; ++b) {
+                fprintf(f, "%d", b);
+                for (int i = 0; i < FZ_TRACE_N && h[(size_t)b * FZ_TRACE_N + i]; ++i)
+                    fprintf(f, " %llu:%llu", h[(size_t)b * FZ_TRACE_N + i] & 15ull, h[(size_t)b * FZ_TRACE_N + i] >> 4);
+                fprintf(f, "\n");
+            }
+            fclose(f);
+        }
+    }
+    return MDI_OK;
+}
+
 } // namespace
 
 // Used by entry points that take no context (other files of the library): text for mdi_last_error(NULL).
@@ -881,7 +1273,8 @@ void mdi_destroy(mdi_ctx *c) {
         if (P.stream) cudaStreamDestroy(P.stream);
     }
     void *ptrs[] = {c->rope_cos, c->rope_sin, c->logits, c->head_pv, c->head_pi, c->head_ticket, c->cur_tok, c->tok_log,
-                    c->gen_count, c->teacher, c->n_teacher, c->prompt_buf, c->pk_teams, c->pk_phases, c->pk_sync, c->pk_err, c->pk_prof, c->tg_err};
+                    c->gen_count, c->teacher, c->n_teacher, c->prompt_buf, c->pk_teams, c->pk_phases, c->pk_sync, c->pk_err, c->pk_prof, c->tg_err,
+                    c->fz_teams, c->fz_phases, c->fz_works, c->fz_blocks, c->fz_segs, c->fz_units, c->fz_err, c->fz_stream, c->fz_acc, c->fz_sync, c->fz_prof};
     for (void *q : ptrs) if (q) cudaFree(q);
     cudaEvent_t evs[] = {c->ev_fork, c->ev_fork_cap, c->ev_t0, c->ev_t1, c->ev_pf0, c->ev_pf1};
     for (auto e : evs) if (e) cudaEventDestroy(e);
@@ -942,7 +1335,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     if (c->o.debug_withhold_handoff < 0 || c->o.debug_withhold_handoff > K) return bail(fail(c, MDI_ERR_ARG, "debug_withhold_handoff must name a partition (1-based) or be 0"));
     c->withhold_once = c->o.debug_withhold_handoff - 1;
     c->scheduler = c->o.scheduler;
-    if (c->scheduler < 0 || c->scheduler > 2) return bail(fail(c, MDI_ERR_ARG, "scheduler must be 0, 1 or 2"));
+    if (c->scheduler < 0 || c->scheduler > 3) return bail(fail(c, MDI_ERR_ARG, "scheduler must be 0, 1, 2 or 3"));
     const int G = std::min(n_samples, K);
     c->gmax = (n_samples + G - 1) / G;
     const long pool_tokens = c->o.kv_pool_tokens > 0 ? c->o.kv_pool_tokens : (long)n_samples * s.n_ctx;
@@ -1071,6 +1464,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     c->prefilled.assign(n_samples, 0);
     TRY(pk_setup(c));
     TRY(pf_setup(c));
+    TRY(fz_setup(c));
     CUB(cudaDeviceSynchronize());
 #undef TRY
 #undef CUB
@@ -1100,6 +1494,7 @@ int mdi_load_weights(mdi_ctx *c, const char *name, const void *host, size_t nbyt
     }
     if (!t.loaded) { t.loaded = true; ++c->n_loaded; }
     c->pk_tables_stale = true;
+    c->fz_stale = true;
     return MDI_OK;
 }
 
@@ -1304,11 +1699,19 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
     const long total = (long)n_pass * K;        // phase slots per partition
     const long t_total = total ? total + K - 1 : 0;
     long t = 0;
-    const bool use_pk = c->pk_ok && c->scheduler != 1 && c->temperature <= 0.f && (n_samples + G - 1) / G <= PK_MAXNB &&
-                        !(c->pf_tc && (n_samples + G - 1) / G >= c->tc_min_group) && pk_tile_count_fits(c, n_pass, G);
+    // fused-phase kernel where the shape fits it, else the phase-per-matrix kernel, else streams
+    const bool small_groups = c->temperature <= 0.f && (n_samples + G - 1) / G <= PK_MAXNB &&
+                              !(c->pf_tc && c->scheduler == 0 && (n_samples + G - 1) / G >= c->tc_min_group);
+    const bool use_fz = c->fz_ok && (c->scheduler == 0 || c->scheduler == 3) && small_groups && fz_slot_count_fits(c, n_pass, G);
+    const bool use_pk = !use_fz && c->pk_ok && c->scheduler != 1 && c->scheduler != 3 && small_groups && pk_tile_count_fits(c, n_pass, G);
     if (c->scheduler == 2 && !use_pk) return fail(c, MDI_ERR_SHAPE, "persistent scheduler unavailable for this call");
-    if (t_total && use_pk) {
+    if (c->scheduler == 3 && !use_fz) return fail(c, MDI_ERR_SHAPE, "fused-phase scheduler unavailable for this call");
+    if (t_total && use_fz) {
+        if ((rc = fz_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
+        c->last_kernel = 2;
+    } else if (t_total && use_pk) {
         if ((rc = pk_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
+        c->last_kernel = 1;
     } else if (t_total) {
         const int R = c->rounds_per_graph;
         const long t_steady = K > 1 ? K : 0; // first tick, multiple of K, from which every partition is in steady state
@@ -1364,9 +1767,9 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
         c->st.tokens_generated += n_pass;
     }
     CU(cudaStreamSynchronize(c->main));
-    if (t_total && use_pk) {
+    if (t_total && (use_pk || use_fz)) {
         int kerr = 0;
-        CU(cudaMemcpy(&kerr, c->pk_err, sizeof(int), cudaMemcpyDeviceToHost));
+        CU(cudaMemcpy(&kerr, use_fz ? c->fz_err : c->pk_err, sizeof(int), cudaMemcpyDeviceToHost));
         if (kerr) {
             // the pipeline stopped half-way: positions, caches and counters no longer agree, so every sample is
             // forgotten (like mdi_reset_sample); the context itself stays usable
@@ -1439,18 +1842,21 @@ int mdi_get_stats(mdi_ctx *c, mdi_stats *out) {
 int mdi_get_partition_times(mdi_ctx *c, int p, double *out_ms, int n) {
     if (!c || !out_ms) return fail(c, MDI_ERR_ARG, "null argument");
     if (p < 0 || p >= c->K || n < 1) return fail(c, MDI_ERR_ARG, "partition out of range");
-    if (!c->pk_ok || !c->pk_prof_on) return fail(c, MDI_ERR_STATE, "in-kernel timing is off (set MDI_PK_PROFILE=1 before mdi_create; persistent scheduler only)");
+    const bool fz = c->last_kernel == 2;
+    if (fz ? !(c->fz_ok && c->fz_prof_on) : !(c->pk_ok && c->pk_prof_on))
+        return fail(c, MDI_ERR_STATE, "in-kernel timing is off (set MDI_PK_PROFILE=1 before mdi_create; persistent schedulers only)");
     CU(cudaSetDevice(c->dev));
     CU(cudaDeviceSynchronize());
-    const PkTeam &T = c->pk_teams_host[p];
-    std::vector<unsigned long long> h((size_t)T.n_cta * PK_PROF_N);
-    CU(cudaMemcpy(h.data(), c->pk_prof + (size_t)T.first_cta * PK_PROF_N, h.size() * 8, cudaMemcpyDeviceToHost));
+    const int first_cta = fz ? c->fz_teams_host[p].first_cta : c->pk_teams_host[p].first_cta;
+    const int n_cta = fz ? c->fz_teams_host[p].n_cta : c->pk_teams_host[p].n_cta;
+    std::vector<unsigned long long> h((size_t)n_cta * PK_PROF_N);
+    CU(cudaMemcpy(h.data(), (fz ? c->fz_prof : c->pk_prof) + (size_t)first_cta * PK_PROF_N, h.size() * 8, cudaMemcpyDeviceToHost));
     for (int i = 0; i < n; ++i) {
         double acc = 0;
-        for (int k = 0; k < T.n_cta && i < PK_PROF_N; ++k) acc += (double)h[(size_t)k * PK_PROF_N + i];
-        out_ms[i] = acc / T.n_cta * 1e-6;
+        for (int k = 0; k < n_cta && i < PK_PROF_N; ++k) acc += (double)h[(size_t)k * PK_PROF_N + i];
+        out_ms[i] = acc / n_cta * 1e-6;
     }
-    return T.n_cta;
+    return n_cta;
 }
 
 int64_t mdi_memory_bytes(mdi_ctx *c, int p) {

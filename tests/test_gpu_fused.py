@@ -1,0 +1,90 @@
+"""The fused-phase persistent kernel (scheduler 3: two team barriers per block of the model, weights repacked
+per thread block into tensor-core fragment order) against the CPU oracle, through the C ABI.
+
+Same protocol as test_gpu_parity.py.  Shapes cover: one and several samples per group (1, 2 and 3-4 columns
+pairs of the B operand), fewer samples than partitions, head_dim 16/32/64, a vocabulary that is not a multiple
+of the 16-row tile, a hidden width that gives blocks unequal numbers of hidden units, resumed generate calls,
+and agreement with the other schedulers.
+"""
+import numpy as np
+import pytest
+
+from paper_2505_18164_b200 import inputs as I
+from helpers import make_oracle, oracle_reference, parity_tolerance, tiny_shape
+from test_gpu_parity import _ctx, _check_teacher_forced_stepwise, _check_free_running
+
+pytestmark = pytest.mark.gpu
+
+FUSED_CASES = [
+    # L, d, H, V, C, bounds, S, P, N, opts
+    (4, 64, 4, 97, 64, [0, 2, 4], 2, 9, 16, dict(page_tokens=8)),
+    (4, 64, 4, 97, 64, [0, 2, 4], 5, 9, 16, dict(page_tokens=8)),            # groups of 3 and 2
+    (3, 128, 2, 131, 96, [0, 1, 2, 3], 2, 17, 30, {}),                        # fewer samples than partitions, head_dim 64
+    (3, 128, 2, 131, 96, [0, 1, 2, 3], 3, 17, 40, dict(prefill_mode=1)),
+    (4, 64, 2, 97, 64, [0, 1, 2, 3, 4], 1, 4, 9, {}),                         # one sample, four partitions
+    (2, 256, 4, 2100, 48, [0, 1, 2], 4, 5, 8, {}),                            # 2 per group, 132 vocabulary tiles
+    (2, 256, 16, 333, 160, [0, 2], 4, 100, 50, dict(page_tokens=4)),          # one partition, 4 per group, head_dim 16, long cache
+    (5, 192, 3, 1000, 64, [0, 1, 5], 2, 3, 20, {}),                           # unequal partitions, d_ff 768 = 48 hidden units
+]
+
+
+@pytest.mark.parametrize("L,d,H,V,C,bounds,S,P,N,opts", FUSED_CASES)
+def test_fused_kernel_matches_oracle(L, d, H, V, C, bounds, S, P, N, opts):
+    shape = tiny_shape("gpt", I.DT_BF16, L=L, d=d, H=H, V=V, C=C)
+    orc, w = make_oracle(shape, seed=3, std=0.04)
+    prompts = I.make_prompts(V, S, P, seed=5)
+    toks, lgs, margins = oracle_reference(orc, prompts, N)
+    ctx = _ctx(shape, bounds, S, w, scheduler=3, **opts)
+    _check_teacher_forced_stepwise(ctx, shape, prompts, toks, lgs, margins, N)
+    _check_free_running(ctx, shape, prompts, toks, margins, N)
+    ctx.close()
+
+
+def test_fused_kernel_agrees_with_the_other_schedulers():
+    """Tokens of a long free-running call (and of a resumed one) equal those of the stream scheduler and of the
+    phase-per-matrix kernel wherever the oracle's margin is clear; final logits agree to rounding."""
+    shape = tiny_shape("gpt", I.DT_BF16, L=3, d=128, H=4, V=211, C=160)
+    orc, w = make_oracle(shape, seed=11, std=0.05)
+    prompts = I.make_prompts(211, 3, 6, seed=2)
+    toks, lgs, margins = oracle_reference(orc, prompts, 90)
+    outs, logits = [], []
+    for sched in (1, 2, 3):
+        ctx = _ctx(shape, [0, 1, 2, 3], 3, w, scheduler=sched)
+        for s in range(3):
+            ctx.set_teacher_tokens(s, toks[s])
+            ctx.prefill(s, prompts[s])
+        a = ctx.generate(3, 50)
+        b = ctx.generate(3, 40)          # resumed call: feeds the last token first
+        outs.append(np.concatenate([a, b], axis=1))
+        logits.append(np.stack([ctx.get_logits(s) for s in range(3)]))
+        ctx.close()
+    tol = parity_tolerance(shape)
+    for s in range(3):
+        ok = margins[s] > 2 * tol
+        for o in outs:
+            assert np.array_equal(o[s][ok], np.asarray(toks[s])[ok])
+    assert np.abs(logits[2] - logits[0]).max() < 1e-3 and np.abs(logits[2] - logits[1]).max() < 1e-3
+
+
+def test_fused_kernel_is_deterministic():
+    """Partial sums meet in integer accumulators, so two runs give bit-identical logits."""
+    shape = tiny_shape("gpt", I.DT_BF16, L=2, d=128, H=2, V=300, C=64)
+    _, w = make_oracle(shape, seed=4, std=0.05)
+    prompts = I.make_prompts(300, 2, 5, seed=9)
+    res = []
+    for _ in range(2):
+        ctx = _ctx(shape, [0, 1, 2], 2, w, scheduler=3)
+        for s in range(2):
+            ctx.prefill(s, prompts[s])
+        out = ctx.generate(2, 30)
+        res.append((out.copy(), ctx.get_logits(0).copy(), ctx.get_logits(1).copy()))
+        ctx.close()
+    assert np.array_equal(res[0][0], res[1][0])
+    assert np.array_equal(res[0][1], res[1][1]) and np.array_equal(res[0][2], res[1][2])
+
+
+def test_fused_scheduler_refuses_shapes_it_does_not_cover():
+    from paper_2505_18164_b200 import mdi
+    shape = tiny_shape("llama", I.DT_BF16, L=2, d=64, H=4, V=50, C=32)
+    with pytest.raises(mdi.MdiError):
+        mdi.Context(shape, [0, 1, 2], 2, scheduler=3)
