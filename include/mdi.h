@@ -63,7 +63,8 @@ typedef struct {
 
 /* Optional tuning; zero means "default". */
 typedef struct {
-    int page_tokens;   /* rows per key/value page (default 16; power of two) */
+    int page_tokens;   /* rows per key/value page (power of two; default 16, or 128 for shapes the fused-phase
+                          scheduler covers, whose bulk copies of cache rows want large pages) */
     int kv_pool_tokens;/* tokens of cache each partition's pool can hold over all samples
                           (default n_samples * n_ctx, rounded up to pages) */
     int attn_splits;   /* sequence splits of decode attention (default: chosen from n_ctx) */

@@ -18,7 +18,7 @@
 // Weights are stored a second time, per thread block, in exactly the order that block consumes them and in the
 // register layout of the tensor-core instruction (mma.sync m16n8k16, bf16 x bf16 -> fp32): a "fragment block"
 // (FB) of 512 bytes is a 16-row x 16-column tile, 16 bytes per lane.  The producer copies the block's stream
-// 32 KB at a time (cp.async.bulk + mbarrier); consumers read a lane's 16 bytes with one shared-memory load
+// 64 KB at a time (cp.async.bulk + mbarrier); consumers read a lane's 16 bytes with one shared-memory load
 // and issue one MMA per FB.  The activation is the B operand: column 2b holds the high bf16 half of sample
 // b's value, column 2b+1 the low half (x = hi + lo to ~16 mantissa bits), so up to 4 samples share a pass.
 //
@@ -28,16 +28,22 @@
 
 namespace mdi {
 
-constexpr int FZ_SLOT_FB = 64;       // fragment blocks per ring slot
+// One bulk copy costs this GPU's copy engine about 0.26 us whatever its size (measured: 8 KB copies stream 31 GB/s per
+// SM, 32 KB copies 125 GB/s, 64 KB copies 245 GB/s, however many are in flight), so slots are as large as the ring allows.
+constexpr int FZ_SLOT_SHIFT = 7;
+constexpr int FZ_SLOT_FB = 1 << FZ_SLOT_SHIFT; // fragment blocks per ring slot (64 KB)
 constexpr int FZ_FB_BYTES = 512;
 constexpr int FZ_SLOT_BYTES = FZ_SLOT_FB * FZ_FB_BYTES;
-constexpr int FZ_MAX_SLOTS = 6;
+constexpr int FZ_MAX_SLOTS = 3;
 constexpr int FZ_MAXNB = 4;
-constexpr int FZ_KREG = 8;           // k-steps of a warp whose B fragments stay in registers (split-K parts)
+constexpr int FZ_CWARPS = 8;          // consumer warps (16 were measured slower: more barrier cost, fewer registers, the same chains)
+constexpr int FZ_CTHREADS = FZ_CWARPS * 32;
+constexpr int FZ_THREADS = FZ_CTHREADS + 32; // + the producer warp
+constexpr int FZ_KREG = 8;           // k-steps per warp and tile in split-K parts (d_model <= 1024: 64 k-steps over 8 warps)
 constexpr int FZ_TRACE_N = 128;
-constexpr int FZ_MAX_PHASES = 64;    // phases of a team, segments and hidden units of a block kept in shared memory
+constexpr int FZ_MAX_PHASES = 40;    // phases of a team, segments and hidden units of a block kept in shared memory
 constexpr int FZ_MAX_SEGS = 16;
-constexpr int FZ_MAX_UNITS = 1024;
+constexpr int FZ_MAX_UNITS = 256;
 constexpr int FZ_U = 4;              // elements of a d_model vector per consumer thread (d_model <= 1024)
 
 constexpr float FZ_FIX_SCALE = 4294967296.f; // 2^32: accumulator resolution 2.3e-10
@@ -144,6 +150,18 @@ __device__ __forceinline__ void fz_split(float v, uint16_t &hi, uint16_t &lo) {
     lo = __bfloat16_as_ushort(l);
 }
 
+__device__ __forceinline__ void fz_bar() { asm volatile("bar.sync 1, %0;" ::"n"(FZ_CTHREADS) : "memory"); }
+__device__ __forceinline__ void fz_block_sum2(float &a, float &b, float *red /* [2 * FZ_CWARPS] */) { // over the consumer threads
+    a = warp_sum(a);
+    b = warp_sum(b);
+    fz_bar();
+    if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = a; red[FZ_CWARPS + (threadIdx.x >> 5)] = b; }
+    fz_bar();
+    a = b = 0.f;
+#pragma unroll
+    for (int w = 0; w < FZ_CWARPS; ++w) { a += red[w]; b += red[FZ_CWARPS + w]; }
+}
+
 // Moves a consumer warp's ring cursor to slot `target` (slots counted from the launch): for every slot on the way,
 // arrive on the empty barrier of the slot left behind and wait (bounded) for the next one to be full.  Out of line:
 // the kernel calls it from many places and its instruction footprint matters more than the call.
@@ -180,12 +198,14 @@ __host__ __device__ inline FzSmem fz_smem_layout(int NB, int NS, int d, int hd, 
     L.xres = take((size_t)4 * NB * d, 16);
     L.part = take((size_t)4 * part_floats, 16);
     L.qkv = take((size_t)4 * NB * 3 * hd, 16);
-    L.att_o = take(4 * 1024, 16);
-    L.att_m = take(4 * 64, 16);
-    L.att_l = take(4 * 64, 16);
-    L.red = take(4 * 16, 16);
-    L.hbest_v = take(4 * PK_CWARPS * FZ_MAXNB, 16);
-    L.hbest_i = take(4 * PK_CWARPS * FZ_MAXNB, 16);
+    // attention scratch lives in the split-K buffer (never in use at the same time; the host sizes `part` for both):
+    // [groups][hd] with groups * hd = 128 per warp, then up to 8 groups per warp (head_dim 16) of maxima and sums
+    L.att_o = L.part;
+    L.att_m = L.att_o + 4 * 128 * FZ_CWARPS;
+    L.att_l = L.att_m + 4 * 8 * FZ_CWARPS;
+    L.red = take(4 * 2 * FZ_CWARPS, 16);
+    L.hbest_v = take(4 * FZ_CWARPS * FZ_MAXNB, 16);
+    L.hbest_i = take(4 * FZ_CWARPS * FZ_MAXNB, 16);
     L.s_dead = take(8, 8);
     L.s_kvdone = take(8, 8);
     L.s_pilot = take(4 * FZ_MAXNB, 16);
@@ -203,7 +223,7 @@ __host__ __device__ inline FzSmem fz_smem_layout(int NB, int NS, int d, int hd, 
 }
 
 template <int NB>
-__global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P) {
+__global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P) {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int d = P.d, hd = P.head_dim, NS = P.n_slots_ring, K = P.K, G = P.G;
@@ -240,15 +260,15 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(full_base + 8 * s, 1);
-            mbar_init(empty_base + 8 * s, PK_CWARPS);
+            mbar_init(empty_base + 8 * s, FZ_CWARPS);
         }
         *s_dead = 0;
         *s_kvdone = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = tid; i < T.n_phases; i += PK_THREADS) { s_ph[i] = P.phases[T.phase_begin + i]; s_wk[i] = P.works[B.work_begin + i]; }
-    for (int i = tid; i < B.n_seg; i += PK_THREADS) s_seg[i] = P.segs[B.seg_begin + i];
-    for (int i = tid; i < B.n_units; i += PK_THREADS) s_units[i] = P.units[B.unit_begin + i];
+    for (int i = tid; i < T.n_phases; i += FZ_THREADS) { s_ph[i] = P.phases[T.phase_begin + i]; s_wk[i] = P.works[B.work_begin + i]; }
+    for (int i = tid; i < B.n_seg; i += FZ_THREADS) s_seg[i] = P.segs[B.seg_begin + i];
+    for (int i = tid; i < B.n_units; i += FZ_THREADS) s_units[i] = P.units[B.unit_begin + i];
     __syncthreads();
     bool dead = false;
     const long total_slots = (long)P.n_pass * K;
@@ -257,7 +277,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
     const uint32_t page_k_bytes = (uint32_t)pt * hd * 4u;
     // ring slots one sample's cached rows take
     auto kv_slots_of = [&](int n_old) { return (((n_old + pt - 1) >> pshift) + P.kv_pps - 1) >> pps_shift; };
-    const bool prof_on = P.prof != nullptr && lane == 0 && (warp == 0 || warp == PK_CWARPS);
+    const bool prof_on = P.prof != nullptr && lane == 0 && (warp == 0 || warp == FZ_CWARPS);
     unsigned long long pf[PK_PROF_N] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}, pf_t = prof_on ? pk_now() : 0;
     int trace_ev = -1; // >= 0 while the traced step runs (thread 0 only)
     auto lap = [&](int cat) {
@@ -267,7 +287,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
         }
     };
 
-    if (warp == PK_CWARPS) {
+    if (warp == FZ_CWARPS) {
         // =========================== producer: weight segments and cache rows, slot by slot, step after step ===========================
         unsigned seq = 0;
         int slot = 0;
@@ -310,9 +330,11 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                     if (smp >= P.n_samples) break;
                     const int n_old = __ldcg(T.pos + smp) + r, pages = (n_old + pt - 1) >> pshift;
                     const int *ptab = T.kv.page_table + ((size_t)smp * T.kv.n_layers_local + S.kv_layer) * T.kv.pages_per_seq;
+                    int pg32 = 0; // page ids of 32 consecutive pages, one per lane: one request serves many slots
                     for (int i0 = 0; i0 < pages; i0 += P.kv_pps) {
+                        if ((i0 & 31) == 0) pg32 = i0 + lane < pages ? ptab[i0 + lane] : 0;
                         const int cnt = min(P.kv_pps, pages - i0);
-                        const int pg = lane < cnt ? ptab[i0 + lane] : 0; // requested before the wait for the slot
+                        const int pg = __shfl_sync(0xffffffffu, pg32, (i0 + lane) & 31); // kv_pps divides 32: one chunk of 32 per slot
                         if (!next_slot()) break;
                         if (lane == 0) mbar_expect_tx(full_base + 8 * slot, (uint32_t)cnt * 2u * page_k_bytes);
                         __syncwarp();
@@ -353,7 +375,9 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
     unsigned step_base = 0;                  // first slot of the current step
     auto advance = [&](unsigned target) {
         if (cur.x != target) {
+            const unsigned long long w0 = prof_on ? pk_now() : 0;
             cur = fz_advance_slow(cur, target, full_base, empty_base, NS, P.err, P.wait_ns);
+            if (prof_on) pf[11] += pk_now() - w0; // time in ring waits (also counted in the phase part that waited)
             slot4 = ring4 + (size_t)(cur.y & 0xffu) * SLOT_U4;
             if ((cur.y >> 16) & 1u) dead = true;
         }
@@ -361,7 +385,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
 
     unsigned bar_epoch = 0;
     auto team_barrier = [&]() {
-        consumer_bar();
+        fz_bar();
         if (tid == 0) {
             ++bar_epoch;
             if (T.n_cta > 1) {
@@ -370,7 +394,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
             }
             if (dead) *s_dead = 1;
         }
-        consumer_bar();
+        fz_bar();
         if (*(volatile int *)s_dead) dead = true;
     };
 
@@ -378,7 +402,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
     // segment whose first slot is slot0; warp w takes k-steps [w ks / 8, (w+1) ks / 8) of every tile (at most
     // FZ_KREG); partial sums go to `part`, to be added up after a block barrier.
     auto split_k = [&](unsigned slot0, int fb0, int n_t, int ks) {
-        const int k0 = warp * ks / PK_CWARPS, k1 = (warp + 1) * ks / PK_CWARPS, nk = k1 - k0;
+        const int k0 = warp * ks / FZ_CWARPS, k1 = (warp + 1) * ks / FZ_CWARPS, nk = k1 - k0;
         uint32_t bf[FZ_KREG][2];
         const uint16_t *brow = xb + (size_t)g * P.xb_stride + 2 * q;
 #pragma unroll
@@ -390,7 +414,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
         for (int t = 0; t < n_t; ++t) {
             float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
             const int f0 = fb0 + t * ks + k0;
-            advance(slot0 + (unsigned)(f0 >> 6));
+            advance(slot0 + (unsigned)(f0 >> FZ_SLOT_SHIFT));
             if (nk > 0) {
                 const int n1 = min(nk, FZ_SLOT_FB - (f0 & (FZ_SLOT_FB - 1)));
                 const uint4 *p1 = slot4 + (f0 & (FZ_SLOT_FB - 1)) * 32 + lane;
@@ -399,7 +423,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                 for (int kk = 0; kk < FZ_KREG; ++kk)
                     if (kk < n1) a[kk] = p1[kk * 32];
                 if (n1 < nk) { // the warp's run crosses into the next slot
-                    advance(slot0 + (unsigned)(f0 >> 6) + 1u);
+                    advance(slot0 + (unsigned)(f0 >> FZ_SLOT_SHIFT) + 1u);
                     const uint4 *p2 = slot4 + lane;
 #pragma unroll
                     for (int kk = 0; kk < FZ_KREG; ++kk)
@@ -410,8 +434,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                     if (kk < nk) fz_mma((kk & 1) ? cb : ca, a[kk], bf[kk][0], bf[kk][1]);
             }
             if (q < NB) {
-                part[((t * PK_CWARPS + warp) * 16 + g) * NB + q] = (ca[0] + cb[0]) + (ca[1] + cb[1]);
-                part[((t * PK_CWARPS + warp) * 16 + g + 8) * NB + q] = (ca[2] + cb[2]) + (ca[3] + cb[3]);
+                part[((t * FZ_CWARPS + warp) * 16 + g) * NB + q] = (ca[0] + cb[0]) + (ca[1] + cb[1]);
+                part[((t * FZ_CWARPS + warp) * 16 + g + 8) * NB + q] = (ca[2] + cb[2]) + (ca[3] + cb[3]);
             }
         }
     };
@@ -421,17 +445,17 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
     auto tile_split = [&](unsigned slot0, int fb0, int n_t, int ks, const uint16_t *opnd, int stride, auto &&epi) {
         const uint16_t *brow = opnd + (size_t)g * stride + 2 * q;
         const bool bon = g < 2 * NB;
-        for (int r0 = 0; r0 < n_t; r0 += PK_CWARPS) {
-            const int n_r = min(PK_CWARPS, n_t - r0);
+        for (int r0 = 0; r0 < n_t; r0 += FZ_CWARPS) {
+            const int n_r = min(FZ_CWARPS, n_t - r0);
             const bool active = warp < n_r;
             const int base = fb0 + r0 * ks + (active ? warp : 0); // idle warps follow warp 0 through the ring
             float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
             int k = 0;
             while (k < ks) {
                 const int fb = base + k * n_r;
-                advance(slot0 + (unsigned)(fb >> 6));
+                advance(slot0 + (unsigned)(fb >> FZ_SLOT_SHIFT));
                 const int room = FZ_SLOT_FB - (fb & (FZ_SLOT_FB - 1));
-                const int k_end = min(ks, k + (n_r == PK_CWARPS ? (room + 7) >> 3 : (room + n_r - 1) / n_r)); // k-steps in this slot
+                const int k_end = min(ks, k + (n_r == FZ_CWARPS ? (room + FZ_CWARPS - 1) / FZ_CWARPS : (room + n_r - 1) / n_r)); // k-steps in this slot
                 const uint4 *ap = slot4 + (fb & (FZ_SLOT_FB - 1)) * 32 + lane;
                 const int stp = n_r * 32;
                 for (; k + 4 <= k_end; k += 4, ap += 4 * stp) {
@@ -469,7 +493,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
     auto prefetch_vectors = [&](const FzPhase &ph, bool norm) {
 #pragma unroll
         for (int u = 0; u < FZ_U; ++u) {
-            const int i = tid + u * PK_CTHREADS;
+            const int i = tid + u * FZ_CTHREADS;
             gam[u] = (norm && i < d) ? ph.gamma[i] : 0.f;
             bet[u] = (norm && i < d) ? ph.beta[i] : 0.f;
             bin[u] = (ph.bias_in && i < d) ? ph.bias_in[i] : 0.f;
@@ -482,7 +506,6 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
         if (j >= G) continue;
         const unsigned r = (unsigned)(v / K);
         trace_ev = (P.trace && tid == 0 && (long)P.trace_step == v) ? 0 : -1;
-        lap(10);
         int nb = 0;
         int slots[NB], pos[NB];
 #pragma unroll
@@ -498,7 +521,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
             else if (r > 0) wait_ge(T.flag_in + j, r, P.err, PKE_FLAG, dead, P.wait_ns);
             if (dead) *s_dead = 1;
         }
-        consumer_bar();
+        fz_bar();
         if (*(volatile int *)s_dead) dead = true;
         lap(FZP_FLAG);
         int kvs_per_unit = 0; // ring slots the cached rows of one head take in this step (all samples of the group)
@@ -514,7 +537,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                 const int tok = b < nb ? min(max(__ldcg(P.cur_tok + slots[b]), 0), P.vocab - 1) : 0;
                 const __nv_bfloat16 *te = reinterpret_cast<const __nv_bfloat16 *>(P.wte) + (size_t)tok * d;
                 const __nv_bfloat16 *pe = P.wpe ? reinterpret_cast<const __nv_bfloat16 *>(P.wpe) + (size_t)pos[b] * d : nullptr;
-                for (int i = tid; i < d; i += PK_CTHREADS) {
+                for (int i = tid; i < d; i += FZ_CTHREADS) {
                     float xv = 0.f;
                     if (b < nb) { xv = __bfloat162float(te[i]); if (pe) xv += __bfloat162float(pe[i]); }
                     xres[b * d + i] = xv;
@@ -522,14 +545,14 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                 }
             } else {
                 const float *src = T.ring_in + ((size_t)j * P.gmax + b) * d;
-                for (int i = tid; i < d; i += PK_CTHREADS) {
+                for (int i = tid; i < d; i += FZ_CTHREADS) {
                     const float xv = b < nb ? __ldcg(src + i) : 0.f;
                     xres[b * d + i] = xv;
                     if (i == 0) s_pilot[b] = xv;
                 }
             }
         }
-        consumer_bar();
+        fz_bar();
 
         for (int pi = 0; pi < T.n_phases; ++pi, ++phase_ctr) {
             const FzPhase ph = s_ph[pi];
@@ -545,7 +568,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                 for (int b = 0; b < NB; ++b)
 #pragma unroll
                     for (int u = 0; u < FZ_U; ++u) {
-                        const int i = tid + u * PK_CTHREADS;
+                        const int i = tid + u * FZ_CTHREADS;
                         av[b][u] = (i < d && b < nb) ? __ldcg(acc_r + (size_t)b * d + i) : 0ll;
                     }
             }
@@ -554,11 +577,11 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                 const int n_out = nb * 3 * hd, qw = P.n_head * hd;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int o = tid + u * PK_CTHREADS;
+                    const int o = tid + u * FZ_CTHREADS;
                     if (o < n_out) { const int rr = o % (3 * hd), which = rr / hd; brw[u] = ph.bias_rows[which * qw + wk.unit * hd + (rr - which * hd)]; }
                 }
                 // page-table entries of this head's cache rows
-                for (int i = tid; i < NB * P.pages_per_seq; i += PK_CTHREADS) {
+                for (int i = tid; i < NB * P.pages_per_seq; i += FZ_CTHREADS) {
                     const int b = i / P.pages_per_seq, pg = i - b * P.pages_per_seq;
                     s_pt[i] = (b < nb && pg <= (pos[b] >> pshift))
                                   ? T.kv.page_table[((size_t)slots[b] * T.kv.n_layers_local + ph.layer_local) * T.kv.pages_per_seq + pg] : 0;
@@ -567,7 +590,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                 const int n_out = NB * 16 * wk.n_tiles;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int o = tid + u * PK_CTHREADS;
+                    const int o = tid + u * FZ_CTHREADS;
                     if (o < n_out) { const int rr = o % (16 * wk.n_tiles); brw[u] = ph.bias_rows[s_units[wk.tile0 + (rr >> 4)] * 16 + (rr & 15)]; }
                 }
             }
@@ -577,7 +600,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                 float xv[FZ_U];
 #pragma unroll
                 for (int u = 0; u < FZ_U; ++u) {
-                    const int i = tid + u * PK_CTHREADS;
+                    const int i = tid + u * FZ_CTHREADS;
                     xv[u] = 0.f;
                     if (i < d) {
                         xv[u] = xres[b * d + i];
@@ -594,13 +617,13 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                 float s1 = 0.f, s2 = 0.f;
 #pragma unroll
                 for (int u = 0; u < FZ_U; ++u)
-                    if (tid + u * PK_CTHREADS < d) { const float cv = xv[u] - pilot; s1 += cv; s2 += cv * cv; }
-                cblock_sum2(s1, s2, red);
+                    if (tid + u * FZ_CTHREADS < d) { const float cv = xv[u] - pilot; s1 += cv; s2 += cv * cv; }
+                fz_block_sum2(s1, s2, red);
                 const float dm = s1 / (float)d, mean = pilot + dm;
                 const float rstd = rsqrtf(fmaxf(s2 / (float)d - dm * dm, 0.f) + P.eps);
 #pragma unroll
                 for (int u = 0; u < FZ_U; ++u) {
-                    const int i = tid + u * PK_CTHREADS;
+                    const int i = tid + u * FZ_CTHREADS;
                     if (i < d) {
                         const float nv = (xv[u] - mean) * rstd * gam[u] + bet[u];
                         uint16_t hi, lo;
@@ -612,8 +635,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
             }
             // accumulator of the phase after next: cleared by one block of the team (all its readers passed the last barrier)
             if ((int)(phase_ctr % (unsigned)T.n_cta) == cta)
-                for (int i = tid; i < (int)acc_stride; i += PK_CTHREADS) acc_z[i] = 0ll;
-            consumer_bar();
+                for (int i = tid; i < (int)acc_stride; i += FZ_CTHREADS) acc_z[i] = 0ll;
+            fz_bar();
             lap(FZP_PROLOGUE);
 
             const unsigned seg_slot0 = step_base + (unsigned)s_seg[wk.seg0].slots_before + (unsigned)(wk.seg0 * kvs_per_unit);
@@ -624,14 +647,14 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                 const bool is_a = ph.kind == FZ_A;
                 const int n_t = wk.n_tiles, h = wk.unit, qw = P.n_head * hd;
                 split_k(seg_slot0, wk.fb0, n_t, ks);
-                consumer_bar();
+                fz_bar();
                 lap(FZP_MMA1);
                 const int per = is_a ? 3 * hd : 16 * n_t, n_out = (is_a ? nb : NB) * per;
                 auto finish_row = [&](int o, float bias) {
                     const int b = o / per, rr = o - b * per, t = rr >> 4, row = rr & 15;
                     float s = 0.f;
 #pragma unroll
-                    for (int w = 0; w < PK_CWARPS; ++w) s += part[((t * PK_CWARPS + w) * 16 + row) * NB + b];
+                    for (int w = 0; w < FZ_CWARPS; ++w) s += part[((t * FZ_CWARPS + w) * 16 + row) * NB + b];
                     s += bias;
                     if (is_a) {
                         // q, k, v of head h; k and v are appended to the cache
@@ -654,9 +677,9 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                     }
                 };
 #pragma unroll
-                for (int u = 0; u < 4; ++u) { const int o = tid + u * PK_CTHREADS; if (o < n_out) finish_row(o, brw[u]); }
+                for (int u = 0; u < 4; ++u) { const int o = tid + u * FZ_CTHREADS; if (o < n_out) finish_row(o, brw[u]); }
 #pragma unroll 1
-                for (int o = tid + 4 * PK_CTHREADS; o < n_out; o += PK_CTHREADS) {
+                for (int o = tid + 4 * FZ_CTHREADS; o < n_out; o += FZ_CTHREADS) {
                     const int rr = o % per;
                     float bias;
                     if (is_a) { const int which = rr / hd; bias = ph.bias_rows[which * qw + h * hd + (rr - which * hd)]; }
@@ -664,7 +687,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                     finish_row(o, bias);
                 }
                 if (is_a) asm volatile("fence.proxy.async.global;" ::: "memory"); // the producer's bulk copies read these rows in later steps
-                consumer_bar();
+                fz_bar();
                 if (is_a) {
                     ++kv_units_done;
                     if (tid == 0) { __threadfence_block(); *s_kvdone = kv_units_done; }
@@ -673,7 +696,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
             }
             // ---- attention of head h over cache rows 0..pos-1 (from the ring) and the new row (shared memory)
             if (has_work && ph.kind == FZ_A) {
-                const int LPR = hd >> 2, RPW = 32 / LPR, NG = PK_CWARPS * RPW;
+                const int LPR = hd >> 2, RPW = 32 / LPR, NG = FZ_CWARPS * RPW;
                 const int sub = lane & (LPR - 1), grp = warp * RPW + lane / LPR;
                 unsigned kv_slot = seg_slot0 + (unsigned)((s_seg[wk.seg0].n_fb + FZ_SLOT_FB - 1) / FZ_SLOT_FB);
                 const int kps = P.kv_pps << pshift; // cache rows per ring slot
@@ -687,7 +710,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
 #pragma unroll
                     for (int i = 1; i < NB; ++i) if (b == i) n_old = pos[i];
                     // chunks: one per ring slot of cached rows, then one for the new row (group 0, from shared memory);
-                    // a warp folds two rows per group and iteration
+                    // a group folds four rows per iteration: four independent dot products, one rescale of the running sums
                     const int n_sl = kv_slots_of(n_old);
 #pragma unroll 1
                     for (int c = 0; c <= n_sl; ++c) {
@@ -700,15 +723,14 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                             n_here = min(kps, n_old - c * kps);
                         }
 #pragma unroll 1
-                        for (int jj0 = 0; jj0 < n_here; jj0 += 2 * NG) {
-                            float4 kk[2], vv[2];
-                            bool live[2];
+                        for (int jj0 = 0; jj0 < n_here; jj0 += 4 * NG) {
+                            float4 kk[4], vv[4];
+                            float sc[4];
 #pragma unroll
-                            for (int u = 0; u < 2; ++u) {
+                            for (int u = 0; u < 4; ++u) {
                                 const int jj = jj0 + u * NG + grp;
-                                live[u] = jj < n_here;
                                 kk[u] = vv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                if (live[u]) {
+                                if (jj < n_here) {
                                     if (!last) {
                                         const unsigned char *kp = sp + (size_t)(jj >> pshift) * 2u * page_k_bytes + (size_t)(jj & (pt - 1)) * hd * 4;
                                         kk[u] = *reinterpret_cast<const float4 *>(kp);
@@ -720,37 +742,59 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                                 }
                             }
 #pragma unroll
-                            for (int u = 0; u < 2; ++u) {
-                                float sc = q4.x * kk[u].x + q4.y * kk[u].y + q4.z * kk[u].z + q4.w * kk[u].w;
-                                for (int w = LPR >> 1; w > 0; w >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, w);
-                                if (live[u]) {
-                                    const float mn = fmaxf(m, sc), corr = __expf(m - mn), pr = __expf(sc - mn);
-                                    l = l * corr + pr;
-                                    o4.x = o4.x * corr + pr * vv[u].x; o4.y = o4.y * corr + pr * vv[u].y;
-                                    o4.z = o4.z * corr + pr * vv[u].z; o4.w = o4.w * corr + pr * vv[u].w;
-                                    m = mn;
+                            for (int u = 0; u < 4; ++u) sc[u] = q4.x * kk[u].x + q4.y * kk[u].y + q4.z * kk[u].z + q4.w * kk[u].w;
+                            for (int w = LPR >> 1; w > 0; w >>= 1) {
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) sc[u] += __shfl_xor_sync(0xffffffffu, sc[u], w);
+                            }
+                            if (jj0 + grp < n_here) { // this group's first row exists (rows past the end count as -inf)
+                                float mn = m;
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    if (jj0 + u * NG + grp >= n_here) sc[u] = -INFINITY;
+                                    mn = fmaxf(mn, sc[u]);
                                 }
+                                const float corr = __expf(m - mn);
+                                float pr[4];
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) pr[u] = __expf(sc[u] - mn);
+                                l = l * corr + ((pr[0] + pr[1]) + (pr[2] + pr[3]));
+                                o4.x = o4.x * corr + ((pr[0] * vv[0].x + pr[1] * vv[1].x) + (pr[2] * vv[2].x + pr[3] * vv[3].x));
+                                o4.y = o4.y * corr + ((pr[0] * vv[0].y + pr[1] * vv[1].y) + (pr[2] * vv[2].y + pr[3] * vv[3].y));
+                                o4.z = o4.z * corr + ((pr[0] * vv[0].z + pr[1] * vv[1].z) + (pr[2] * vv[2].z + pr[3] * vv[3].z));
+                                o4.w = o4.w * corr + ((pr[0] * vv[0].w + pr[1] * vv[1].w) + (pr[2] * vv[2].w + pr[3] * vv[3].w));
+                                m = mn;
                             }
                         }
                     }
                     if (sub == 0) { att_m[grp] = m; att_l[grp] = l; }
                     *reinterpret_cast<float4 *>(att_o + grp * hd + sub * 4) = o4;
-                    consumer_bar();
+                    fz_bar();
+                    if (warp == 0) {
+                        // weights of the groups' partial results, normalised (NG <= 64: two groups per lane)
+                        const float m0 = lane < NG ? att_m[lane] : -INFINITY, m1 = lane + 32 < NG ? att_m[lane + 32] : -INFINITY;
+                        float M = fmaxf(m0, m1);
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+                        const float w0 = m0 == -INFINITY ? 0.f : __expf(m0 - M), w1 = m1 == -INFINITY ? 0.f : __expf(m1 - M);
+                        const float Ls = warp_sum((lane < NG ? att_l[lane] * w0 : 0.f) + (lane + 32 < NG ? att_l[lane + 32] * w1 : 0.f));
+                        __syncwarp();
+                        if (lane < NG) att_m[lane] = w0 / Ls;
+                        if (lane + 32 < NG) att_m[lane + 32] = w1 / Ls;
+                    }
+                    fz_bar();
                     if (tid < hd) {
-                        float M = -INFINITY;
-                        for (int g2 = 0; g2 < NG; ++g2) M = fmaxf(M, att_m[g2]);
-                        float Ls = 0.f, O = 0.f;
-                        for (int g2 = 0; g2 < NG; ++g2) {
-                            const float w = att_m[g2] == -INFINITY ? 0.f : __expf(att_m[g2] - M);
-                            Ls += att_l[g2] * w;
-                            O += att_o[g2 * hd + tid] * w;
+                        float O0 = 0.f, O1 = 0.f;
+                        for (int g2 = 0; g2 < NG; g2 += 2) {
+                            O0 += att_o[g2 * hd + tid] * att_m[g2];
+                            O1 += att_o[(g2 + 1) * hd + tid] * att_m[g2 + 1];
                         }
                         uint16_t hi, lo;
-                        fz_split(O / Ls, hi, lo);
+                        fz_split(O0 + O1, hi, lo);
                         ob[(size_t)(2 * b) * P.ob_stride + tid] = hi;
                         ob[(size_t)(2 * b + 1) * P.ob_stride + tid] = lo;
                     }
-                    consumer_bar();
+                    fz_bar();
                 }
                 lap(FZP_ATTN);
             }
@@ -796,11 +840,11 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
                     if (vv > best_v || (vv == best_v && ii < best_i)) { best_v = vv; best_i = ii; }
                 }
                 if (lane < FZ_MAXNB) { hbest_v[warp * FZ_MAXNB + lane] = best_v; hbest_i[warp * FZ_MAXNB + lane] = best_i; }
-                consumer_bar();
+                fz_bar();
                 if (tid < NB) {
                     float bv = hbest_v[tid];
                     int bi = hbest_i[tid];
-                    for (int w = 1; w < PK_CWARPS; ++w) {
+                    for (int w = 1; w < FZ_CWARPS; ++w) {
                         const float vv = hbest_v[w * FZ_MAXNB + tid];
                         const int ii = hbest_i[w * FZ_MAXNB + tid];
                         if (vv > bv || (vv == bv && ii < bi)) { bv = vv; bi = ii; }
@@ -824,7 +868,7 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
         // ---- end of the step
         if (T.is_last) {
             if (cta == 0) {
-                for (int i = warp; i < nb; i += PK_CWARPS) {
+                for (int i = warp; i < nb; i += FZ_CWARPS) {
                     float bv = -INFINITY;
                     int bi = 0x7fffffff;
                     for (int c2 = lane; c2 < T.n_cta; c2 += 32) {
@@ -853,18 +897,18 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_fused_decode(const FzParams P
             // complete the residual stream with the last phase's sum and hand it to the next partition
             const long long *acc_f = T.acc + (size_t)((phase_ctr + 2u) % 3u) * acc_stride;
             for (int b = 0; b < nb; ++b)
-                for (int i = tid; i < d; i += PK_CTHREADS)
+                for (int i = tid; i < d; i += FZ_CTHREADS)
                     T.ring_out[((size_t)j * P.gmax + b) * d + i] =
                         xres[b * d + i] + (T.bias_final[i] + (float)((double)__ldcg(acc_f + (size_t)b * d + i) * (1.0 / 4294967296.0)));
         }
         if (cta == 0) {
-            consumer_bar();
+            fz_bar();
             if (tid == 0 && P.withhold_partition != p) st_release(T.flag_out + j, r + 1);
         }
         lap(FZP_FIN);
     }
     if (cta == 0)
-        for (int s = tid; s < P.n_samples; s += PK_CTHREADS) T.pos[s] += P.n_pass;
+        for (int s = tid; s < P.n_samples; s += FZ_CTHREADS) T.pos[s] += P.n_pass;
     if (prof_on)
         for (int i = 0; i < PK_PROF_N; ++i)
             if (i != PF_PROD_WAIT && i != PF_PROD_TOTAL) P.prof[(size_t)blockIdx.x * PK_PROF_N + i] = pf[i];

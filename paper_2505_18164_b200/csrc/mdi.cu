@@ -894,7 +894,7 @@ int fz_setup(mdi_ctx *c) {
     if (s.arch != MDI_ARCH_GPT || s.weight_dtype != MDI_DTYPE_BF16 || !c->kv_f32) return no("needs the GPT block, bf16 weights and an fp32 cache");
     if (s.n_kv_head != H || H * hd != d) return no("needs n_kv_head = n_head and n_head * head_dim = d_model");
     if (d % 16 || s.d_ff % 16 || hd % 16) return no("widths must be multiples of 16");
-    if (d > FZ_U * PK_CTHREADS) return no("d_model above 1024");
+    if (d > FZ_U * FZ_CTHREADS) return no("d_model above 1024");
     if (c->gmax > FZ_MAXNB) return no("at most 4 samples per group");
     if (K > 32) return no("too many partitions");
     cudaDeviceProp prop;
@@ -944,36 +944,27 @@ int fz_setup(mdi_ctx *c) {
     c->fz_unit_lists.clear();
     c->fz_blocks_host.clear();
     int n_phases_total = 0, first = 0, m_max = 1;
-    const double a_bytes = 2.0 * (4.0 * hd * d) + (double)NB * (s.n_ctx / 4) * hd * 8.0; // weights of one head + a guess of its cache rows
-    const double u_bytes = 2.0 * 2.0 * 16.0 * d, t_bytes = 2.0 * 16.0 * d;
     for (int p = 0; p < K; ++p) {
         const int n = n_cta[p], Lp = c->part[p].hi - c->part[p].lo, np = 2 * Lp + (p == K - 1 ? 1 : 0);
         c->fz_phase_begin[p] = n_phases_total;
         c->fz_phase_count[p] = np;
         n_phases_total += np;
-        std::vector<double> cum(n, 0.0);
+        // Phases end in a team barrier, so what counts is the slowest block of each phase: hidden units and output
+        // rows are dealt out evenly within their own phase; heads rotate over the blocks from layer to layer so
+        // that the same blocks do not wait (with full rings) through every attention phase.
         std::vector<std::vector<FzWork>> wk(n, std::vector<FzWork>(np, FzWork{-1, 0, 0, 0, 0, 0, 0}));
         std::vector<std::vector<std::vector<int>>> ul(n, std::vector<std::vector<int>>(np));
-        auto least = [&](const std::vector<char> *skip) {
-            int best = -1;
-            for (int b = 0; b < n; ++b)
-                if (!(skip && (*skip)[b]) && (best < 0 || cum[b] < cum[best])) best = b;
-            return best;
-        };
+        int next_head_block = 0;
         for (int l = 0; l < Lp; ++l) {
-            std::vector<char> used(n, 0);
             for (int h = 0; h < H; ++h) {
-                const int b = least(&used);
-                used[b] = 1;
+                const int b = next_head_block;
+                next_head_block = (next_head_block + 1) % n;
                 wk[b][2 * l].unit = h;
                 wk[b][2 * l].n_tiles = 3 * hd / 16;
-                cum[b] += a_bytes;
             }
-            for (int u = 0; u < s.d_ff / 16; ++u) {
-                const int b = least(nullptr);
-                ul[b][2 * l + 1].push_back(u);
-                cum[b] += u_bytes;
-            }
+            // blocks without a head in this layer come first: their rings had the attention phase to fill up
+            const int n_units = s.d_ff / 16;
+            for (int u = 0; u < n_units; ++u) ul[(next_head_block + u) % n][2 * l + 1].push_back(u);
             for (int b = 0; b < n; ++b) {
                 wk[b][2 * l + 1].n_tiles = (int)ul[b][2 * l + 1].size();
                 m_max = std::max(m_max, wk[b][2 * l + 1].n_tiles);
@@ -981,19 +972,11 @@ int fz_setup(mdi_ctx *c) {
         }
         if (p == K - 1) {
             const int NT = (s.vocab + 15) / 16;
-            double tot = (double)NT * t_bytes;
-            for (double x : cum) tot += x;
-            const double target = tot / n;
-            std::vector<int> give(n, 0);
-            int left = NT;
-            for (int b = 0; b < n; ++b) {
-                give[b] = std::max(0, std::min(left, (int)std::floor((target - cum[b]) / t_bytes)));
-                left -= give[b];
-                cum[b] += give[b] * t_bytes;
-            }
-            while (left > 0) { const int b = least(nullptr); ++give[b]; cum[b] += t_bytes; --left; }
             int t0 = 0;
-            for (int b = 0; b < n; ++b) { wk[b][np - 1].n_tiles = give[b]; wk[b][np - 1].tile0 = t0; t0 += give[b]; }
+            for (int b = 0; b < n; ++b) {
+                const int give = NT / n + (b < NT % n ? 1 : 0);
+                wk[b][np - 1].n_tiles = give; wk[b][np - 1].tile0 = t0; t0 += give;
+            }
         }
         for (int b = 0; b < n; ++b) {
             FzBlock fb{};
@@ -1028,10 +1011,10 @@ int fz_setup(mdi_ctx *c) {
     m_max = (m_max + 3) & ~3;
     const int max_tiles = std::max(3 * hd / 16, m_max);
     c->fz_xb_stride = d + 8; c->fz_hb_stride = 16 * m_max + 8; c->fz_ob_stride = hd + 8;
-    c->fz_part_floats = max_tiles * PK_CWARPS * 16 * NB;
+    c->fz_part_floats = std::max(max_tiles * FZ_CWARPS * 16 * NB, (128 + 16) * FZ_CWARPS); // also the attention scratch
     const size_t fixed = fz_smem_layout(NB, 0, d, hd, c->fz_part_floats, c->pages_per_seq, c->fz_xb_stride, c->fz_hb_stride, c->fz_ob_stride).total;
     const size_t budget = (size_t)prop.sharedMemPerBlockOptin;
-    if (fixed + 3 * (size_t)FZ_SLOT_BYTES > budget) return no("activations do not fit in shared memory");
+    if (fixed + 2 * (size_t)FZ_SLOT_BYTES > budget) return no("activations do not fit in shared memory");
     c->fz_slots = (int)std::min<size_t>(FZ_MAX_SLOTS, (budget - fixed) / FZ_SLOT_BYTES);
     c->fz_smem = fz_smem_layout(NB, c->fz_slots, d, hd, c->fz_part_floats, c->pages_per_seq, c->fz_xb_stride, c->fz_hb_stride, c->fz_ob_stride).total;
     for (int nb : {1, 2, 4}) CU(cudaFuncSetAttribute(fz_func(nb), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->fz_smem));
@@ -1060,8 +1043,8 @@ int fz_build(mdi_ctx *c) {
     c->fz_units_host.clear();
     const void *head_w = s.tied_lm_head ? c->wte : c->lm_head;
     auto rounds = [&](const void *W, int ld, int n_t, int n_k, auto &&row_of, auto &&col_of, int row_limit) {
-        for (int r0 = 0; r0 < n_t; r0 += PK_CWARPS) {
-            const int n_r = std::min(PK_CWARPS, n_t - r0);
+        for (int r0 = 0; r0 < n_t; r0 += FZ_CWARPS) {
+            const int n_r = std::min(FZ_CWARPS, n_t - r0);
             for (int k = 0; k < n_k; ++k)
                 for (int w = 0; w < n_r; ++w) {
                     const int row0 = row_of(r0 + w);
@@ -1221,7 +1204,7 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     // the template parameter fixes the accumulator stride, so it is the context's group size, not this call's
     const void *fn = fz_func(c->fz_nb);
     void *args[] = {&P};
-    CU(cudaLaunchCooperativeKernel(fn, dim3(c->fz_grid), dim3(PK_THREADS), args, c->fz_smem, c->main));
+    CU(cudaLaunchCooperativeKernel(fn, dim3(c->fz_grid), dim3(FZ_THREADS), args, c->fz_smem, c->main));
     ++c->st.kernel_launches;
     c->st.stage_steps += (int64_t)c->K * n_pass * G;
     if (trace) {
@@ -1320,7 +1303,13 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
 #define TRY(x) do { if ((rc = (x)) != MDI_OK) return bail(rc); } while (0)
 #define CUB(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return bail(fail(c, e_ == cudaErrorMemoryAllocation ? MDI_ERR_OOM : MDI_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_))); } while (0)
 
-    c->page_tokens = c->o.page_tokens > 0 ? c->o.page_tokens : 16;
+    // default page: 16 rows; 128 rows where the fused-phase kernel can run (GPT block, bf16 weights, fp32 cache), which
+    // copies one head's rows of a page with one bulk copy each for keys and values and wants those copies large
+    {
+        const bool fused_candidate = s.arch == MDI_ARCH_GPT && s.weight_dtype == MDI_DTYPE_BF16 && !c->o.kv_cache_bf16 &&
+                                     s.n_kv_head == s.n_head && c->o.scheduler != 1 && c->o.scheduler != 2 && s.head_dim <= 64;
+        c->page_tokens = c->o.page_tokens > 0 ? c->o.page_tokens : (fused_candidate ? 128 : 16);
+    }
     if (c->page_tokens & (c->page_tokens - 1)) return bail(fail(c, MDI_ERR_ARG, "page_tokens must be a power of two"));
     c->page_shift = 0;
     while ((1 << c->page_shift) < c->page_tokens) ++c->page_shift;
@@ -1407,7 +1396,8 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
         P.hi = part_bounds[p + 1];
         const int Lp = P.hi - P.lo;
         CUB(cudaStreamCreateWithFlags(&P.stream, cudaStreamNonBlocking));
-        const long pages_per_layer = (pool_tokens + c->page_tokens - 1) / c->page_tokens;
+        // every sample may leave one page partly filled: with pages above 16 rows that slack is added to the pool
+        const long pages_per_layer = (pool_tokens + c->page_tokens - 1) / c->page_tokens + (c->page_tokens > 16 ? n_samples : 0);
         P.n_pages = (int)(pages_per_layer * Lp);
         P.kv_bytes = (size_t)P.n_pages * c->page_elems * c->kv_esize;
         CUB(cudaMalloc(&P.kv_pool, std::max<size_t>(P.kv_bytes, 16)));
