@@ -192,7 +192,7 @@ def main():
     ap.add_argument("--workload", default="gpt2_small", choices=list(I.ALL_WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--rounds-per-graph", type=int, default=0)
-    ap.add_argument("--scheduler", type=int, default=0, help="0 auto (persistent kernel when it fits), 1 streams, 2 persistent")
+    ap.add_argument("--scheduler", type=int, default=0, help="0 auto (a persistent kernel when the shape fits), 1 streams, 2 phase-per-matrix persistent kernel, 3 fused-phase persistent kernel")
     ap.add_argument("--tc-min-group", type=int, default=0, help="smallest group whose decode steps run on the tensor cores (0 = library default)")
     ap.add_argument("--n-new", type=int, default=0, help="shorter generation (profiler captures only; not the headline)")
     ap.add_argument("--n-prompt", type=int, default=0, help="shorter prompts (profiler captures only)")

@@ -84,10 +84,17 @@ typedef struct {
                           usable.  0 (default): 2000 ms */
     int debug_withhold_handoff; /* failure-detection check: p > 0 makes partition p-1 withhold its output handoff during
                           the first persistent mdi_generate after creation, so that the next partition's wait runs out */
-    int scheduler;     /* how mdi_generate runs the recurrent pipeline.  0: the persistent kernel (one launch,
-                          one team of thread blocks per partition, flag handoff between teams) when the shape
-                          fits it (groups of at most 4 samples), else the stream scheduler; 1: always the
-                          stream scheduler (one stream per partition, event handoff); 2: persistent or fail */
+    int scheduler;     /* how mdi_generate runs the recurrent pipeline.
+                          0: a persistent kernel when the shape fits one (one cooperative launch for the whole call,
+                             one team of thread blocks per partition, flag handoff between teams), else the stream
+                             scheduler.  Two persistent kernels exist: the fused-phase kernel (GPT block, bf16 weights,
+                             fp32 cache, n_kv_head = n_head, d_model <= 1024, groups of at most 4 samples, every team
+                             at least n_head blocks: two team barriers per block of the model, weights re-stored per
+                             thread block in tensor-core fragment order) is preferred; the phase-per-matrix kernel
+                             (groups of at most 4 samples, any block type) comes next;
+                          1: always the stream scheduler (one stream per partition, event handoff);
+                          2: the phase-per-matrix persistent kernel, or fail;
+                          3: the fused-phase persistent kernel, or fail */
 } mdi_options;
 
 typedef struct {

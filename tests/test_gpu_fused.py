@@ -88,3 +88,33 @@ def test_fused_scheduler_refuses_shapes_it_does_not_cover():
     shape = tiny_shape("llama", I.DT_BF16, L=2, d=64, H=4, V=50, C=32)
     with pytest.raises(mdi.MdiError):
         mdi.Context(shape, [0, 1, 2], 2, scheduler=3)
+
+
+def test_fused_kernel_withheld_handoff_times_out_and_the_context_survives():
+    """Failure detection without faulting anything (as for the other persistent kernel): partition 0 withholds its
+    output handoff once, waits are given 50 ms, the call returns MDI_ERR_TIMEOUT, the samples are reset, and the
+    same context then generates correctly."""
+    import time
+    from paper_2505_18164_b200 import mdi
+    shape = tiny_shape("gpt", I.DT_BF16, L=3, d=64, H=4, V=97, C=48)
+    orc, w = make_oracle(shape, seed=9, std=0.06)
+    ctx = mdi.Context(shape, [0, 1, 2, 3], 3, scheduler=3, wait_limit_ms=50, debug_withhold_handoff=1)
+    ctx.load_all(w)
+    prompts = I.make_prompts(97, 3, 5, seed=12)
+    for s in range(3):
+        ctx.prefill(s, prompts[s])
+    t0 = time.time()
+    with pytest.raises(mdi.MdiError) as e:
+        ctx.generate(3, 8)
+    assert e.value.code == mdi.ERR_TIMEOUT and "gave up waiting" in str(e.value)
+    assert time.time() - t0 < 20.0
+    assert ctx.stats().kv_pages_in_use[0] == 0                      # every sample was reset
+    toks, _, margins = oracle_reference(orc, prompts, 8)
+    for s in range(3):
+        ctx.prefill(s, prompts[s])
+    out = ctx.generate(3, 8)                                        # the hook was one-shot: this run is normal
+    tol = parity_tolerance(shape)
+    for s in range(3):
+        ok = margins[s] > 2 * tol
+        assert np.array_equal(out[s][ok], np.asarray(toks[s])[ok])
+    ctx.close()
