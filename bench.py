@@ -33,10 +33,13 @@ sys.path.insert(0, ROOT)
 
 from paper_2505_18164_b200 import inputs as I  # noqa: E402
 
-# DRAM traffic of the persistent decode kernel relative to its algorithmic bytes, from the ncu capture
-# kept with the profiler summaries of this repository (17.143 GB moved for 17.171 GB algorithmic; traffic
-# grows with the number of passes like the algorithmic bytes do).  None for other workloads / schedulers.
+# DRAM traffic of the persistent decode kernels relative to their algorithmic bytes, from the ncu captures kept with
+# the profiler summaries of this repository (23-pass captures of the GPT-2-small shape: fused-phase kernel 17.756 GB
+# moved for 17.171 GB algorithmic, phase-per-matrix kernel 17.143 GB).  Weights are 99% of both and are read once per
+# group and pass, so traffic grows with the number of passes like the algorithmic bytes do; the fused kernel's excess
+# is whole 128-row cache pages, which shrinks as the pages fill.  None for other workloads / schedulers.
 PK_TRAFFIC_RATIO = {"gpt2_small": 17.143 / 17.171}
+FZ_TRAFFIC_RATIO = {"gpt2_small": 17.756 / 17.171}
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
@@ -307,7 +310,8 @@ def main():
             "prefill_ms": sum(pf_ms) / len(pf_ms), "decode_ms": gen_avg_ms,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                         "traffic": (PK_TRAFFIC_RATIO[w.name] * db["total"] if w.name in PK_TRAFFIC_RATIO and args.scheduler != 1 else None),
+                         "traffic": ((FZ_TRAFFIC_RATIO if args.scheduler in (0, 3) else PK_TRAFFIC_RATIO)[w.name] * db["total"]
+                                     if w.name in PK_TRAFFIC_RATIO and args.scheduler != 1 else None),
                          "traffic_note": "scaled from a 23-pass ncu capture of the same kernel", "scope": "decode phase of one step (all kernels of mdi_generate)",
                          "algorithmic_bytes": db["total"], "weight_bytes": db["weights"], "kv_bytes": db["kv"]},
             "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(S * P * 4),
