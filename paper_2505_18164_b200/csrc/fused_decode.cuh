@@ -60,7 +60,8 @@ struct FzPhase {                 // one per (team, phase)
 struct FzWork {                  // one per (block, phase)
     int unit;                    // A: head served by this block in this layer (-1: none)
     int n_tiles;                 // A: row tiles of q,k,v of one head; B: hidden units (16 rows each); HEAD: row tiles
-    int tile0;                   // B: offset into the block's unit list; HEAD: first row tile
+    int tile0;                   // A: first of this block's q,k,v row tiles of the head; B: offset into the block's unit list; HEAD: first row tile
+    int row_tile0, row_tiles;    // A: this block's row tiles of the head's output-projection columns
     int fb0, fb1;                // offsets of the two parts of the phase inside their segments
     int seg0, seg1;              // segment of each part
 };
@@ -90,6 +91,9 @@ struct FzParams {
     int d, n_head, head_dim, d_ff, vocab, act, K, G, n_samples, gmax, n_pass, n_slots_ring;
     int xb_stride, hb_stride, ob_stride, part_floats, pages_per_seq;
     int kv_pps;                  // cache pages (of one head) per ring slot: cached rows reach the consumers through the ring
+    int pair;                    // 1: a head is served by the two blocks of a cluster (q,k,v rows, cache rows of every page and
+                                 // output rows split in halves; exchanges through distributed shared memory); 0: by one block
+    int kv_rows;                 // rows of a cache page a block handles: page_tokens, or half of it when pair
     float eps, scale;
     const FzTeam *teams;
     const FzPhase *phases;
@@ -162,6 +166,43 @@ __device__ __forceinline__ void fz_block_sum2(float &a, float &b, float *red /* 
     for (int w = 0; w < FZ_CWARPS; ++w) { a += red[w]; b += red[FZ_CWARPS + w]; }
 }
 
+// ---- the two blocks of a cluster (pair mode): remote shared memory and a pair barrier built on mbarriers ----
+__device__ __forceinline__ uint32_t fz_cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t fz_mapa(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void fz_st_remote(uint32_t addr, float v) { asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory"); }
+__device__ __forceinline__ void fz_arrive_remote(uint32_t bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool fz_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(20000u) : "memory");
+    return ok != 0;
+}
+// Bounded wait for the peer's arrivals on this block's pair barrier; true when the wait ran out (or another did).
+__device__ __noinline__ bool fz_pair_wait(uint32_t bar, uint32_t parity, int *err, unsigned long long limit_ns) {
+    unsigned long long t0 = 0;
+    for (unsigned it = 0;; ++it) {
+        if (fz_try_wait_cluster(bar, parity)) return false;
+        if ((it & 63u) == 63u) {
+            if (*(volatile int *)err) return true;
+            const unsigned long long now = pk_now();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > limit_ns) break;
+        }
+    }
+    atomicCAS(err, 0, (int)PKE_BARRIER);
+    return true;
+}
+__device__ __forceinline__ void fz_cluster_sync_all() { // every thread of every block of the cluster
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // Moves a consumer warp's ring cursor to slot `target` (slots counted from the launch): for every slot on the way,
 // arrive on the empty barrier of the slot left behind and wait (bounded) for the next one to be full.  Out of line:
 // the kernel calls it from many places and its instruction footprint matters more than the call.
@@ -189,7 +230,7 @@ __device__ __noinline__ uint2 fz_advance_slow(uint2 cur, unsigned target, uint32
 // device call the same function, so the launch size and the carve-up cannot disagree.
 struct FzSmem {
     size_t xres, part, qkv, att_o, att_m, att_l, red, hbest_v, hbest_i, s_dead, s_kvdone, s_pilot, s_pt, s_units, xb, hb, ob,
-        bars, s_ph, s_wk, s_seg, total;
+        pairbuf, bars, s_ph, s_wk, s_seg, total;
 };
 __host__ __device__ inline FzSmem fz_smem_layout(int NB, int NS, int d, int hd, int part_floats, int pages_per_seq, int xbs, int hbs, int obs) {
     FzSmem L;
@@ -214,7 +255,8 @@ __host__ __device__ inline FzSmem fz_smem_layout(int NB, int NS, int d, int hd, 
     L.xb = take((size_t)2 * 2 * NB * xbs, 16);
     L.hb = take((size_t)2 * 2 * NB * hbs, 16);
     L.ob = take((size_t)2 * 2 * NB * obs, 16);
-    L.bars = take(2 * FZ_MAX_SLOTS * 8, 16);
+    L.pairbuf = take((size_t)4 * 2 * NB * (hd + 2), 16); // [2 blocks][NB][max, sum, o[hd]] of the halves of a head's attention
+    L.bars = take((2 * FZ_MAX_SLOTS + 1) * 8, 16);       // full[NS], empty[NS], then the pair barrier
     L.s_ph = take(sizeof(FzPhase) * FZ_MAX_PHASES, 16);
     L.s_wk = take(sizeof(FzWork) * FZ_MAX_PHASES, 16);
     L.s_seg = take(sizeof(FzSeg) * FZ_MAX_SEGS, 16);
@@ -246,6 +288,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
     uint16_t *xb = reinterpret_cast<uint16_t *>(smem + L.xb);     // [2 NB][xb_stride] norm output, hi/lo rows
     uint16_t *hb = reinterpret_cast<uint16_t *>(smem + L.hb);     // [2 NB][hb_stride] hidden units, hi/lo rows
     uint16_t *ob = reinterpret_cast<uint16_t *>(smem + L.ob);     // [2 NB][ob_stride] attention output, hi/lo rows
+    float *pairbuf = reinterpret_cast<float *>(smem + L.pairbuf);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
     FzPhase *s_ph = reinterpret_cast<FzPhase *>(smem + L.s_ph);
     FzWork *s_wk = reinterpret_cast<FzWork *>(smem + L.s_wk);
@@ -256,12 +299,14 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
     const FzTeam T = P.teams[p];
     const FzBlock B = P.blocks[blockIdx.x];
     const int cta = blockIdx.x - T.first_cta;
-    const uint32_t slot_base = smem_u32(ring_mem), full_base = smem_u32(bars), empty_base = smem_u32(bars + NS);
+    const uint32_t slot_base = smem_u32(ring_mem), full_base = smem_u32(bars), empty_base = smem_u32(bars + NS), pair_bar = smem_u32(bars + 2 * FZ_MAX_SLOTS);
+    const uint32_t rank = P.pair ? fz_cluster_rank() : 0u; // this block's half of a head
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             mbar_init(full_base + 8 * s, 1);
             mbar_init(empty_base + 8 * s, FZ_CWARPS);
         }
+        mbar_init(pair_bar, FZ_CTHREADS); // every consumer thread of the peer arrives
         *s_dead = 0;
         *s_kvdone = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -270,11 +315,13 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
     for (int i = tid; i < B.n_seg; i += FZ_THREADS) s_seg[i] = P.segs[B.seg_begin + i];
     for (int i = tid; i < B.n_units; i += FZ_THREADS) s_units[i] = P.units[B.unit_begin + i];
     __syncthreads();
+    fz_cluster_sync_all(); // the peer's barriers exist before anything arrives on them (a cluster of one block otherwise)
     bool dead = false;
     const long total_slots = (long)P.n_pass * K;
     const int n_seg = B.n_seg, n_kvu = n_seg - 1; // head units (cache visits) of this block per step
     const int pt = T.kv.page_tokens, pshift = T.kv.page_shift, pps_shift = 31 - __clz(P.kv_pps);
-    const uint32_t page_k_bytes = (uint32_t)pt * hd * 4u;
+    const int kvr = P.kv_rows, kvr_shift = 31 - __clz(P.kv_rows), kv_row0 = (int)rank * P.kv_rows;
+    const uint32_t page_k_bytes = (uint32_t)kvr * hd * 4u; // keys (or values) of this block's rows of one page of one head
     // ring slots one sample's cached rows take
     auto kv_slots_of = [&](int n_old) { return (((n_old + pt - 1) >> pshift) + P.kv_pps - 1) >> pps_shift; };
     const bool prof_on = P.prof != nullptr && lane == 0 && (warp == 0 || warp == FZ_CWARPS);
@@ -339,7 +386,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                         if (lane == 0) mbar_expect_tx(full_base + 8 * slot, (uint32_t)cnt * 2u * page_k_bytes);
                         __syncwarp();
                         if (lane < cnt) {
-                            const float *kp = reinterpret_cast<const float *>(T.kv.pool) + (size_t)pg * T.kv.page_elems + (size_t)S.kv_head * pt * hd;
+                            const float *kp = reinterpret_cast<const float *>(T.kv.pool) + (size_t)pg * T.kv.page_elems + ((size_t)S.kv_head * pt + kv_row0) * hd;
                             const uint32_t dst = slot_base + slot * FZ_SLOT_BYTES + (uint32_t)lane * 2u * page_k_bytes;
                             bulk_g2s(dst, kp, page_k_bytes, full_base + 8 * slot);
                             bulk_g2s(dst + page_k_bytes, kp + (size_t)T.kv.n_kv_head * pt * hd, page_k_bytes, full_base + 8 * slot);
@@ -361,9 +408,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
             for (unsigned q = seq > (unsigned)NS ? seq - NS : 0; q < seq; ++q)
                 while (!mbar_try_wait(full_base + 8 * (int)(q % NS), (uint32_t)((q / NS) & 1)) && pk_now() - t0 < 100000000ull) {}
         }
-        return;
-    }
-
+    } else {
     // =========================== consumers ===========================
     const int g = lane >> 2, q = lane & 3;
     const uint4 *ring4 = reinterpret_cast<const uint4 *>(ring_mem);
@@ -381,6 +426,15 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
             slot4 = ring4 + (size_t)(cur.y & 0xffu) * SLOT_U4;
             if ((cur.y >> 16) & 1u) dead = true;
         }
+    };
+
+    // pair mode: arrive on the peer's barrier (after this thread's remote stores), wait for the peer's arrivals on ours
+    const uint32_t peer_bar = P.pair ? fz_mapa(pair_bar, rank ^ 1u) : 0u;
+    uint32_t pair_parity = 0;
+    auto pair_sync = [&]() {
+        fz_arrive_remote(peer_bar);
+        if (!dead && fz_pair_wait(pair_bar, pair_parity, P.err, P.wait_ns)) dead = true;
+        pair_parity ^= 1u;
     };
 
     unsigned bar_epoch = 0;
@@ -574,11 +628,11 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
             }
             float brw[4] = {0.f, 0.f, 0.f, 0.f}; // biases of the first four rows this thread finishes after the split-K part
             if (has_work && ph.kind == FZ_A) {
-                const int n_out = nb * 3 * hd, qw = P.n_head * hd;
+                const int per_a = 16 * wk.n_tiles, n_out = nb * per_a, qw = P.n_head * hd;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int o = tid + u * FZ_CTHREADS;
-                    if (o < n_out) { const int rr = o % (3 * hd), which = rr / hd; brw[u] = ph.bias_rows[which * qw + wk.unit * hd + (rr - which * hd)]; }
+                    if (o < n_out) { const int rr = wk.tile0 * 16 + o % per_a, which = rr / hd; brw[u] = ph.bias_rows[which * qw + wk.unit * hd + (rr - which * hd)]; }
                 }
                 // page-table entries of this head's cache rows
                 for (int i = tid; i < NB * P.pages_per_seq; i += FZ_CTHREADS) {
@@ -649,7 +703,8 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                 split_k(seg_slot0, wk.fb0, n_t, ks);
                 fz_bar();
                 lap(FZP_MMA1);
-                const int per = is_a ? 3 * hd : 16 * n_t, n_out = (is_a ? nb : NB) * per;
+                const int per = 16 * n_t, n_out = (is_a ? nb : NB) * per;
+                const uint32_t peer_qkv = (is_a && P.pair) ? fz_mapa(smem_u32(qkv), rank ^ 1u) : 0u;
                 auto finish_row = [&](int o, float bias) {
                     const int b = o / per, rr = o - b * per, t = rr >> 4, row = rr & 15;
                     float s = 0.f;
@@ -657,9 +712,10 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                     for (int w = 0; w < FZ_CWARPS; ++w) s += part[((t * FZ_CWARPS + w) * 16 + row) * NB + b];
                     s += bias;
                     if (is_a) {
-                        // q, k, v of head h; k and v are appended to the cache
-                        const int which = rr / hd, e = rr - which * hd;
-                        qkv[b * 3 * hd + rr] = s;
+                        // q, k, v of head h (this block's rows of them; the peer gets a copy); k and v are appended to the cache
+                        const int rg = wk.tile0 * 16 + rr, which = rg / hd, e = rg - which * hd;
+                        qkv[b * 3 * hd + rg] = s;
+                        if (P.pair) fz_st_remote(peer_qkv + (uint32_t)(b * 3 * hd + rg) * 4u, s);
                         if (which > 0) {
                             int pb = pos[0];
 #pragma unroll
@@ -682,11 +738,12 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                 for (int o = tid + 4 * FZ_CTHREADS; o < n_out; o += FZ_CTHREADS) {
                     const int rr = o % per;
                     float bias;
-                    if (is_a) { const int which = rr / hd; bias = ph.bias_rows[which * qw + h * hd + (rr - which * hd)]; }
+                    if (is_a) { const int rg = wk.tile0 * 16 + rr, which = rg / hd; bias = ph.bias_rows[which * qw + h * hd + (rg - which * hd)]; }
                     else bias = ph.bias_rows[s_units[wk.tile0 + (rr >> 4)] * 16 + (rr & 15)];
                     finish_row(o, bias);
                 }
-                if (is_a) asm volatile("fence.proxy.async.global;" ::: "memory"); // the producer's bulk copies read these rows in later steps
+                if (is_a) asm volatile("fence.proxy.async.global;" ::: "memory"); // the producers' bulk copies read these rows in later steps
+                if (is_a && P.pair) pair_sync(); // both halves of q, k, v are in place, and the peer's cache rows are written
                 fz_bar();
                 if (is_a) {
                     ++kv_units_done;
@@ -699,7 +756,8 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                 const int LPR = hd >> 2, RPW = 32 / LPR, NG = FZ_CWARPS * RPW;
                 const int sub = lane & (LPR - 1), grp = warp * RPW + lane / LPR;
                 unsigned kv_slot = seg_slot0 + (unsigned)((s_seg[wk.seg0].n_fb + FZ_SLOT_FB - 1) / FZ_SLOT_FB);
-                const int kps = P.kv_pps << pshift; // cache rows per ring slot
+                const uint32_t peer_pairbuf = P.pair ? fz_mapa(smem_u32(pairbuf), rank ^ 1u) : 0u;
+                float *my_half = pairbuf + (size_t)rank * NB * (hd + 2);
 #pragma unroll 1
                 for (int b = 0; b < nb; ++b) {
                     const float *qv = qkv + b * 3 * hd;
@@ -709,30 +767,35 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                     int n_old = pos[0];
 #pragma unroll
                     for (int i = 1; i < NB; ++i) if (b == i) n_old = pos[i];
-                    // chunks: one per ring slot of cached rows, then one for the new row (group 0, from shared memory);
-                    // a group folds four rows per iteration: four independent dot products, one rescale of the running sums
-                    const int n_sl = kv_slots_of(n_old);
+                    // chunks: one per ring slot of cached rows (this block's rows of each page), then one for the new row
+                    // (first block of the head, group 0, from shared memory); a group folds four rows per iteration:
+                    // four independent dot products, one rescale of the running sums
+                    const int n_sl = kv_slots_of(n_old), n_pages = (n_old + pt - 1) >> pshift;
 #pragma unroll 1
                     for (int c = 0; c <= n_sl; ++c) {
                         const bool last = c == n_sl;
-                        int n_here = 1;
+                        int n_here = rank == 0 ? 1 : 0, page0 = 0;
                         const unsigned char *sp = nullptr;
                         if (!last) {
                             advance(kv_slot++);
                             sp = reinterpret_cast<const unsigned char *>(slot4) + sub * 16;
-                            n_here = min(kps, n_old - c * kps);
+                            page0 = c << pps_shift;
+                            n_here = min(P.kv_pps, n_pages - page0) << kvr_shift;
                         }
 #pragma unroll 1
                         for (int jj0 = 0; jj0 < n_here; jj0 += 4 * NG) {
                             float4 kk[4], vv[4];
                             float sc[4];
+                            bool live[4];
 #pragma unroll
                             for (int u = 0; u < 4; ++u) {
-                                const int jj = jj0 + u * NG + grp;
+                                const int jj = jj0 + u * NG + grp, pgs = jj >> kvr_shift, row = jj & (kvr - 1);
+                                // position of the row: page, this block's first row of a page, row
+                                live[u] = jj < n_here && (last || ((page0 + pgs) << pshift) + kv_row0 + row < n_old);
                                 kk[u] = vv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                if (jj < n_here) {
+                                if (live[u]) {
                                     if (!last) {
-                                        const unsigned char *kp = sp + (size_t)(jj >> pshift) * 2u * page_k_bytes + (size_t)(jj & (pt - 1)) * hd * 4;
+                                        const unsigned char *kp = sp + (size_t)pgs * 2u * page_k_bytes + (size_t)row * hd * 4;
                                         kk[u] = *reinterpret_cast<const float4 *>(kp);
                                         vv[u] = *reinterpret_cast<const float4 *>(kp + page_k_bytes);
                                     } else {
@@ -747,11 +810,11 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
 #pragma unroll
                                 for (int u = 0; u < 4; ++u) sc[u] += __shfl_xor_sync(0xffffffffu, sc[u], w);
                             }
-                            if (jj0 + grp < n_here) { // this group's first row exists (rows past the end count as -inf)
+                            if (live[0] || live[1] || live[2] || live[3]) {
                                 float mn = m;
 #pragma unroll
                                 for (int u = 0; u < 4; ++u) {
-                                    if (jj0 + u * NG + grp >= n_here) sc[u] = -INFINITY;
+                                    if (!live[u]) sc[u] = -INFINITY;
                                     mn = fmaxf(mn, sc[u]);
                                 }
                                 const float corr = __expf(m - mn);
@@ -771,7 +834,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                     *reinterpret_cast<float4 *>(att_o + grp * hd + sub * 4) = o4;
                     fz_bar();
                     if (warp == 0) {
-                        // weights of the groups' partial results, normalised (NG <= 64: two groups per lane)
+                        // this block's maximum, sum and the groups' weights relative to it (NG <= 64: two groups per lane)
                         const float m0 = lane < NG ? att_m[lane] : -INFINITY, m1 = lane + 32 < NG ? att_m[lane + 32] : -INFINITY;
                         float M = fmaxf(m0, m1);
 #pragma unroll
@@ -779,8 +842,13 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                         const float w0 = m0 == -INFINITY ? 0.f : __expf(m0 - M), w1 = m1 == -INFINITY ? 0.f : __expf(m1 - M);
                         const float Ls = warp_sum((lane < NG ? att_l[lane] * w0 : 0.f) + (lane + 32 < NG ? att_l[lane + 32] * w1 : 0.f));
                         __syncwarp();
-                        if (lane < NG) att_m[lane] = w0 / Ls;
-                        if (lane + 32 < NG) att_m[lane + 32] = w1 / Ls;
+                        if (lane < NG) att_m[lane] = w0;
+                        if (lane + 32 < NG) att_m[lane + 32] = w1;
+                        if (lane < 2) {
+                            const float hv = lane == 0 ? M : Ls;
+                            my_half[b * (hd + 2) + lane] = hv;
+                            if (P.pair) fz_st_remote(peer_pairbuf + (uint32_t)((rank * NB + b) * (hd + 2) + lane) * 4u, hv);
+                        }
                     }
                     fz_bar();
                     if (tid < hd) {
@@ -789,13 +857,31 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                             O0 += att_o[g2 * hd + tid] * att_m[g2];
                             O1 += att_o[(g2 + 1) * hd + tid] * att_m[g2 + 1];
                         }
-                        uint16_t hi, lo;
-                        fz_split(O0 + O1, hi, lo);
-                        ob[(size_t)(2 * b) * P.ob_stride + tid] = hi;
-                        ob[(size_t)(2 * b + 1) * P.ob_stride + tid] = lo;
+                        my_half[b * (hd + 2) + 2 + tid] = O0 + O1;
+                        if (P.pair) fz_st_remote(peer_pairbuf + (uint32_t)((rank * NB + b) * (hd + 2) + 2 + tid) * 4u, O0 + O1);
                     }
                     fz_bar();
                 }
+                // both halves of the head: merged identically by both blocks (first block's half first)
+                if (P.pair) pair_sync();
+                fz_bar();
+                for (int o = tid; o < nb * hd; o += FZ_CTHREADS) {
+                    const int b = o / hd, e = o - b * hd;
+                    const float *h0 = pairbuf + (size_t)b * (hd + 2), *h1 = pairbuf + (size_t)(NB + b) * (hd + 2);
+                    float val;
+                    if (P.pair) {
+                        const float M = fmaxf(h0[0], h1[0]);
+                        const float a0 = h0[0] == -INFINITY ? 0.f : __expf(h0[0] - M), a1 = h1[0] == -INFINITY ? 0.f : __expf(h1[0] - M);
+                        val = (a0 * h0[2 + e] + a1 * h1[2 + e]) / (a0 * h0[1] + a1 * h1[1]);
+                    } else {
+                        val = h0[2 + e] / h0[1];
+                    }
+                    uint16_t hi, lo;
+                    fz_split(val, hi, lo);
+                    ob[(size_t)(2 * b) * P.ob_stride + e] = hi;
+                    ob[(size_t)(2 * b + 1) * P.ob_stride + e] = lo;
+                }
+                fz_bar();
                 lap(FZP_ATTN);
             }
             // ---- second part: tile-split over all d_model rows (partial sums), or the output layer's rows
@@ -806,7 +892,8 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                 int my_slot = slots[0];
 #pragma unroll
                 for (int i = 1; i < NB; ++i) if (q == i) my_slot = slots[i];
-                const int n_t2 = is_head ? wk.n_tiles : d >> 4;
+                const bool is_a2 = ph.kind == FZ_A;
+                const int n_t2 = is_head ? wk.n_tiles : (is_a2 ? wk.row_tiles : d >> 4), row_off = is_a2 ? wk.row_tile0 * 16 : 0;
                 const int ks2 = is_head ? ks : (ph.kind == FZ_A ? hd >> 4 : wk.n_tiles);
                 const uint16_t *opnd = is_head ? xb : (ph.kind == FZ_A ? ob : hb);
                 const int stride = is_head ? P.xb_stride : (ph.kind == FZ_A ? P.ob_stride : P.hb_stride);
@@ -815,8 +902,8 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                     const float y0 = c[0] + c[1], y1 = c[2] + c[3];
                     if (!is_head) {
                         // partial sums over this block's columns, as 64-bit fixed point into the team's accumulator
-                        fz_red_add(acc_w + (size_t)q * d + tile * 16 + g, __float2ll_rn(y0 * FZ_FIX_SCALE));
-                        fz_red_add(acc_w + (size_t)q * d + tile * 16 + g + 8, __float2ll_rn(y1 * FZ_FIX_SCALE));
+                        fz_red_add(acc_w + (size_t)q * d + row_off + tile * 16 + g, __float2ll_rn(y0 * FZ_FIX_SCALE));
+                        fz_red_add(acc_w + (size_t)q * d + row_off + tile * 16 + g + 8, __float2ll_rn(y1 * FZ_FIX_SCALE));
                     } else {
                         const int row = (wk.tile0 + tile) * 16 + g;
                         if (row < P.vocab) {
@@ -912,6 +999,9 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
     if (prof_on)
         for (int i = 0; i < PK_PROF_N; ++i)
             if (i != PF_PROD_WAIT && i != PF_PROD_TOTAL) P.prof[(size_t)blockIdx.x * PK_PROF_N + i] = pf[i];
+    }
+    // no block leaves while its peer may still write into its shared memory
+    fz_cluster_sync_all();
 }
 
 } // namespace mdi

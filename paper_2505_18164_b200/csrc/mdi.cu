@@ -146,7 +146,7 @@ struct mdi_ctx {
     FzBlock *fz_blocks = nullptr;
     FzSeg *fz_segs = nullptr;
     int *fz_units = nullptr, *fz_err = nullptr;
-    int fz_kv_pps = 1;
+    int fz_kv_pps = 1, fz_pair = 0, fz_kv_rows = 16;
     uint4 *fz_stream = nullptr;
     long long *fz_acc = nullptr;
     unsigned *fz_sync = nullptr;
@@ -902,6 +902,22 @@ int fz_setup(mdi_ctx *c) {
     const int n_sm = prop.multiProcessorCount;
     c->fz_nb = c->gmax <= 1 ? 1 : c->gmax <= 2 ? 2 : 4;
     const int NB = c->fz_nb;
+    // Pair mode: a head is served by the two blocks of a cluster (halves of its q,k,v rows, of the rows of every cache
+    // page and of its output rows).  Needs even tile counts, pages of at least two rows, even team sizes with a cluster
+    // per head, and all clusters resident at once.
+    bool pair = !getenv("MDI_FZ_NO_PAIR") && c->page_tokens >= 2 && (3 * hd / 16) % 2 == 0 && (d / 16) % 2 == 0 && n_sm >= 2;
+    if (pair) {
+        for (int nb : {1, 2, 4}) CU(cudaFuncSetAttribute(fz_func(nb), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prop.sharedMemPerBlockOptin));
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(n_sm & ~1); cfg.blockDim = dim3(FZ_THREADS); cfg.dynamicSmemBytes = prop.sharedMemPerBlockOptin;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        int n_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&n_clusters, fz_func(c->fz_nb), &cfg) != cudaSuccess) { cudaGetLastError(); n_clusters = 0; }
+        if (n_clusters < (n_sm & ~1) / 2) pair = false;
+    }
     // team sizes in proportion to the bytes a step streams
     std::vector<double> bytes(K, 0.0);
     const double layer_bytes = 2.0 * (4.0 * d * d + 2.0 * (double)s.d_ff * d);
@@ -910,31 +926,36 @@ int fz_setup(mdi_ctx *c) {
         if (p == K - 1) bytes[p] += 2.0 * (double)s.vocab * d;
     }
     std::vector<int> n_cta(K, 0);
-    {
+    auto team_sizes = [&](bool even) {
         const char *env = getenv("MDI_FZ_TEAM_CTAS");
-        bool from_env = false;
         if (env) {
             std::vector<int> v;
             const char *q = env;
             while (*q) { v.push_back(atoi(q)); while (*q && *q != ',') ++q; if (*q == ',') ++q; }
             int tot = 0;
-            for (int x : v) tot += x;
-            if ((int)v.size() == K && tot <= n_sm && *std::min_element(v.begin(), v.end()) >= 1) { n_cta = v; from_env = true; }
+            bool all_even = true;
+            for (int x : v) { tot += x; all_even = all_even && x % 2 == 0; }
+            if ((int)v.size() == K && tot <= n_sm && *std::min_element(v.begin(), v.end()) >= 1 && (all_even || !even)) { n_cta = v; return; }
         }
-        if (!from_env) {
-            double tot = 0;
-            for (double b : bytes) tot += b;
-            int used = 0, big = 0;
-            for (int p = 0; p < K; ++p) if (bytes[p] > bytes[big]) big = p;
-            for (int p = 0; p < K; ++p) {
-                if (p == big) continue;
-                n_cta[p] = std::max(1, (int)std::floor(n_sm * bytes[p] / tot));
-                used += n_cta[p];
-            }
-            n_cta[big] = n_sm - used;
+        double tot = 0;
+        for (double b : bytes) tot += b;
+        int used = 0, big = 0;
+        for (int p = 0; p < K; ++p) if (bytes[p] > bytes[big]) big = p;
+        for (int p = 0; p < K; ++p) {
+            if (p == big) continue;
+            n_cta[p] = std::max(1, (int)std::floor(n_sm * bytes[p] / tot));
+            if (even) n_cta[p] = std::max(2, n_cta[p] & ~1);
+            used += n_cta[p];
         }
-    }
-    for (int p = 0; p < K; ++p) if (n_cta[p] < H) return no("a team has fewer blocks than the model has heads");
+        n_cta[big] = even ? (n_sm - used) & ~1 : n_sm - used;
+    };
+    team_sizes(pair);
+    for (int p = 0; p < K && pair; ++p)
+        if (n_cta[p] / 2 < H) { pair = false; team_sizes(false); } // not a cluster per head in every team: one block per head
+    for (int p = 0; p < K; ++p)
+        if (n_cta[p] < H) return no("a team has fewer blocks than the model has heads");
+    c->fz_pair = pair;
+    const int pr = pair ? 2 : 1, qkv_tiles = 3 * hd / 16 / pr, out_tiles = d / 16 / pr;
 
     // per team: phases; per block: work items
     c->fz_teams_host.assign(K, FzTeam{});
@@ -957,10 +978,13 @@ int fz_setup(mdi_ctx *c) {
         int next_head_block = 0;
         for (int l = 0; l < Lp; ++l) {
             for (int h = 0; h < H; ++h) {
-                const int b = next_head_block;
-                next_head_block = (next_head_block + 1) % n;
-                wk[b][2 * l].unit = h;
-                wk[b][2 * l].n_tiles = 3 * hd / 16;
+                for (int r = 0; r < pr; ++r) {
+                    FzWork &a = wk[next_head_block + r][2 * l];
+                    a.unit = h;
+                    a.n_tiles = qkv_tiles; a.tile0 = r * qkv_tiles;
+                    a.row_tiles = out_tiles; a.row_tile0 = r * out_tiles;
+                }
+                next_head_block = (next_head_block + pr) % (n / pr * pr);
             }
             // blocks without a head in this layer come first: their rings had the attention phase to fill up
             const int n_units = s.d_ff / 16;
@@ -1003,13 +1027,14 @@ int fz_setup(mdi_ctx *c) {
     }
     // cache rows through the ring: whole pages of one head, as many as fit a slot
     {
-        const size_t page_kv_bytes = (size_t)2 * c->page_tokens * hd * 4;
+        c->fz_kv_rows = c->page_tokens / pr;
+        const size_t page_kv_bytes = (size_t)2 * c->fz_kv_rows * hd * 4; // keys and values of a block's rows of one page of one head
         if (page_kv_bytes > (size_t)FZ_SLOT_BYTES) return no("one head's rows of a cache page exceed a ring slot");
         c->fz_kv_pps = std::min<int>(32, (int)(FZ_SLOT_BYTES / page_kv_bytes));
     }
     // shared memory
     m_max = (m_max + 3) & ~3;
-    const int max_tiles = std::max(3 * hd / 16, m_max);
+    const int max_tiles = std::max(qkv_tiles, m_max);
     c->fz_xb_stride = d + 8; c->fz_hb_stride = 16 * m_max + 8; c->fz_ob_stride = hd + 8;
     c->fz_part_floats = std::max(max_tiles * FZ_CWARPS * 16 * NB, (128 + 16) * FZ_CWARPS); // also the attention scratch
     const size_t fixed = fz_smem_layout(NB, 0, d, hd, c->fz_part_floats, c->pages_per_seq, c->fz_xb_stride, c->fz_hb_stride, c->fz_ob_stride).total;
@@ -1105,13 +1130,16 @@ int fz_build(mdi_ctx *c) {
                 } else if (i % 2 == 0) {
                     if (wk.unit < 0) continue;
                     const int h = wk.unit, tph = hd / 16;
-                    for (int t = 0; t < wk.n_tiles; ++t)
-                        for (int k = 0; k < ks; ++k)
+                    for (int tt = 0; tt < wk.n_tiles; ++tt)
+                        for (int k = 0; k < ks; ++k) {
+                            const int t = wk.tile0 + tt; // row tile of the head's q, k, v rows
                             desc.push_back(FzFbDesc{L.wqkv, d, (t / tph) * qw + h * hd + (t % tph) * 16, 16 * k, 16});
+                        }
                     close_segment(i / 2, h); // this head's cache rows follow in the ring
                     wk.seg1 = (int)segs.size() - FB.seg_begin;
                     wk.fb1 = 0;
-                    rounds(L.wo, qw, d / 16, hd / 16, [&](int t) { return t * 16; }, [&](int k) { return h * hd + 16 * k; }, d);
+                    const int rt0 = wk.row_tile0;
+                    rounds(L.wo, qw, wk.row_tiles, hd / 16, [&](int t) { return (rt0 + t) * 16; }, [&](int k) { return h * hd + 16 * k; }, d);
                 } else {
                     wk.tile0 = (int)c->fz_units_host.size() - FB.unit_begin;
                     for (int u : ul) c->fz_units_host.push_back(u);
@@ -1182,7 +1210,7 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     P.d = s.d_model; P.n_head = s.n_head; P.head_dim = s.head_dim; P.d_ff = s.d_ff; P.vocab = s.vocab; P.act = s.act == MDI_ACT_GELU_ERF;
     P.K = c->K; P.G = G; P.n_samples = n_samples; P.gmax = c->gmax; P.n_pass = n_pass; P.n_slots_ring = c->fz_slots;
     P.xb_stride = c->fz_xb_stride; P.hb_stride = c->fz_hb_stride; P.ob_stride = c->fz_ob_stride; P.part_floats = c->fz_part_floats;
-    P.pages_per_seq = c->pages_per_seq; P.kv_pps = c->fz_kv_pps; P.segs = c->fz_segs;
+    P.pages_per_seq = c->pages_per_seq; P.kv_pps = c->fz_kv_pps; P.pair = c->fz_pair; P.kv_rows = c->fz_kv_rows; P.segs = c->fz_segs;
     P.eps = s.norm_eps; P.scale = 1.0f / std::sqrt((float)s.head_dim);
     P.teams = c->fz_teams; P.phases = c->fz_phases; P.works = c->fz_works; P.blocks = c->fz_blocks; P.units = c->fz_units;
     P.wte = c->wte; P.wpe = c->wpe; P.logits = c->logits; P.head_pv = c->head_pv; P.head_pi = c->head_pi;
@@ -1204,7 +1232,19 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     // the template parameter fixes the accumulator stride, so it is the context's group size, not this call's
     const void *fn = fz_func(c->fz_nb);
     void *args[] = {&P};
-    CU(cudaLaunchCooperativeKernel(fn, dim3(c->fz_grid), dim3(FZ_THREADS), args, c->fz_smem, c->main));
+    if (c->fz_pair) {
+        // cooperative (all blocks resident: teams wait on one another) and in clusters of two (the halves of a head)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(c->fz_grid); cfg.blockDim = dim3(FZ_THREADS); cfg.dynamicSmemBytes = c->fz_smem; cfg.stream = c->main;
+        cudaLaunchAttribute at[2];
+        at[0].id = cudaLaunchAttributeCooperative; at[0].val.cooperative = 1;
+        at[1].id = cudaLaunchAttributeClusterDimension;
+        at[1].val.clusterDim.x = 2; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 2;
+        CU(cudaLaunchKernelExC(&cfg, fn, args));
+    } else {
+        CU(cudaLaunchCooperativeKernel(fn, dim3(c->fz_grid), dim3(FZ_THREADS), args, c->fz_smem, c->main));
+    }
     ++c->st.kernel_launches;
     c->st.stage_steps += (int64_t)c->K * n_pass * G;
     if (trace) {
