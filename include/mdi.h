@@ -90,7 +90,8 @@ typedef struct {
                              scheduler.  Two persistent kernels exist: the fused-phase kernel (GPT block, bf16 weights,
                              fp32 cache, n_kv_head = n_head, d_model <= 1024, groups of at most 4 samples, every team
                              at least n_head blocks: two team barriers per block of the model, weights re-stored per
-                             thread block in tensor-core fragment order) is preferred; the phase-per-matrix kernel
+                             thread block in tensor-core fragment order, a head shared by the two blocks of a
+                             cluster where every team has 2 n_head blocks) is preferred; the phase-per-matrix kernel
                              (groups of at most 4 samples, any block type) comes next;
                           1: always the stream scheduler (one stream per partition, event handoff);
                           2: the phase-per-matrix persistent kernel, or fail;
