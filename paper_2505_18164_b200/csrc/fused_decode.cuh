@@ -853,10 +853,11 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) k_fused_decode(const FzParams P
                     fz_bar();
                     if (tid < hd) {
                         float O0 = 0.f, O1 = 0.f;
-                        for (int g2 = 0; g2 < NG; g2 += 2) {
+                        for (int g2 = 0; g2 + 1 < NG; g2 += 2) {
                             O0 += att_o[g2 * hd + tid] * att_m[g2];
                             O1 += att_o[(g2 + 1) * hd + tid] * att_m[g2 + 1];
                         }
+                        if (NG & 1) O0 += att_o[(NG - 1) * hd + tid] * att_m[NG - 1];
                         my_half[b * (hd + 2) + 2 + tid] = O0 + O1;
                         if (P.pair) fz_st_remote(peer_pairbuf + (uint32_t)((rank * NB + b) * (hd + 2) + 2 + tid) * 4u, O0 + O1);
                     }

@@ -118,3 +118,31 @@ def test_fused_kernel_withheld_handoff_times_out_and_the_context_survives():
         ok = margins[s] > 2 * tol
         assert np.array_equal(out[s][ok], np.asarray(toks[s])[ok])
     ctx.close()
+
+
+def test_fused_kernel_one_or_two_blocks_per_head_agree(monkeypatch):
+    """A head served by one thread block, or shared by the two blocks of a cluster (halves of the q/k/v rows, of each
+    cache page's rows and of the output rows, exchanged through distributed shared memory): same tokens where the
+    oracle's margin is clear, logits equal to rounding, both within tolerance of the oracle."""
+    shape = tiny_shape("gpt", I.DT_BF16, L=4, d=256, H=4, V=523, C=192)
+    orc, w = make_oracle(shape, seed=21, std=0.04)
+    prompts = I.make_prompts(523, 5, 70, seed=8)
+    toks, lgs, margins = oracle_reference(orc, prompts, 60)
+    tol = parity_tolerance(shape)
+    res = []
+    for no_pair in (False, True):
+        if no_pair:
+            monkeypatch.setenv("MDI_FZ_NO_PAIR", "1")
+        ctx = _ctx(shape, [0, 2, 4], 5, w, scheduler=3, page_tokens=32)
+        for s in range(5):
+            ctx.set_teacher_tokens(s, toks[s])
+            ctx.prefill(s, prompts[s])
+        out = ctx.generate(5, 60)
+        lg = np.stack([ctx.get_logits(s) for s in range(5)])
+        for s in range(5):
+            ok = margins[s] > 2 * tol
+            assert np.array_equal(out[s][ok], np.asarray(toks[s])[ok])
+            assert np.abs(lg[s] - lgs[s][-1]).max() <= tol
+        res.append(lg)
+        ctx.close()
+    assert np.abs(res[0] - res[1]).max() < 1e-3
