@@ -192,14 +192,21 @@ int mdi_set_teacher_tokens(mdi_ctx *ctx, int sample, const int32_t *tokens_host,
 int mdi_reset_sample(mdi_ctx *ctx, int sample);
 
 int mdi_get_stats(mdi_ctx *ctx, mdi_stats *out);
-/* Device bytes held by one partition (parameters + key/value pool + buffers), cf. Tables I-II. */
+/* Device bytes held by one partition (parameters + key/value pool + buffers, and once the fused-phase kernel has run its
+ * per-thread-block copy of the partition's matrices), cf. Tables I-II. */
 int64_t mdi_memory_bytes(mdi_ctx *ctx, int partition);
 /* Tracing aid (the paper times token arrival on the starter; here each partition's team of thread
  * blocks times itself).  With MDI_PK_PROFILE set in the environment at mdi_create, the persistent kernel
  * accumulates, per thread block, the nanoseconds spent in: [0] waiting for the input edge, [1] staging
  * and normalising inputs, [2] streaming weight tiles, [3] team barriers, [4] attention, [5] choosing
  * tokens, [6] producer warp waiting for a free ring slot, [7] producer warp total, and within [2]:
- * [8] waiting for a tile to land, [9] multiply-accumulate, [10] reduction and epilogue.  This call averages
+ * [8] waiting for a tile to land, [9] multiply-accumulate, [10] reduction and epilogue.  When the last call ran the
+ * fused-phase kernel the categories are: [0] input edge, [1] norm prologues, [2] row parts (split along k; for the
+ * output layer: unused), [3] bias / activation / cache append after a row part, [4] attention, [5] column parts and the
+ * output layer's rows, [6] and [7] as above, [8] team barriers, [9] end of step (token choice or handoff), [11] time
+ * inside [2], [4], [5] spent waiting for ring slots.  With MDI_FZ_TRACE=<schedule slot> and MDI_FZ_TRACE_FILE=<path>
+ * also set, thread 0 of every block writes a time stamp at every category change of that slot (text, one line per
+ * block, "category:nanoseconds" pairs).  This call averages
  * them over the partition's blocks for the last mdi_generate, in milliseconds, into out_ms[0..n).
  * Returns the number of blocks of the partition (> 0) or a negative error (STATE when timing is off). */
 int mdi_get_partition_times(mdi_ctx *ctx, int partition, double *out_ms, int n);

@@ -152,6 +152,7 @@ struct mdi_ctx {
     unsigned *fz_sync = nullptr;
     unsigned long long *fz_prof = nullptr;
     int64_t fz_stream_bytes = 0;
+    std::vector<int64_t> fz_team_stream_bytes; // per partition: bytes of its blocks' weight streams
     mdi_stats st{};
     std::string err;
 };
@@ -1165,6 +1166,10 @@ int fz_build(mdi_ctx *c) {
     }
     const size_t n_fb = desc.size();
     c->fz_stream_bytes = (int64_t)n_fb * FZ_FB_BYTES;
+    c->fz_team_stream_bytes.assign(K, 0);
+    for (int p = 0; p < K; ++p)
+        for (int b = 0; b < c->fz_teams_host[p].n_cta; ++b)
+            c->fz_team_stream_bytes[p] += (int64_t)c->fz_blocks_host[c->fz_teams_host[p].first_cta + b].n_fb * FZ_FB_BYTES;
     CU(cudaMalloc((void **)&c->fz_stream, std::max<size_t>(n_fb, 1) * FZ_FB_BYTES));
     for (auto &FB : c->fz_blocks_host) FB.stream = c->fz_stream + reinterpret_cast<size_t>(FB.stream) * (FZ_FB_BYTES / 16);
     {
@@ -1897,7 +1902,8 @@ int mdi_get_partition_times(mdi_ctx *c, int p, double *out_ms, int n) {
 
 int64_t mdi_memory_bytes(mdi_ctx *c, int p) {
     if (!c || p < 0 || p >= c->K) return MDI_ERR_ARG;
-    return c->part[p].weight_bytes + (int64_t)c->part[p].kv_bytes + c->part[p].buffer_bytes;
+    return c->part[p].weight_bytes + (int64_t)c->part[p].kv_bytes + c->part[p].buffer_bytes +
+           (p < (int)c->fz_team_stream_bytes.size() ? c->fz_team_stream_bytes[p] : 0);
 }
 
 } // extern "C"
