@@ -312,7 +312,7 @@ def main():
                          "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                          "traffic": ((FZ_TRAFFIC_RATIO if args.scheduler in (0, 3) else PK_TRAFFIC_RATIO)[w.name] * db["total"]
                                      if w.name in PK_TRAFFIC_RATIO and args.scheduler != 1 else None),
-                         "traffic_note": "scaled from a 23-pass ncu capture of the same kernel", "scope": "decode phase of one step (all kernels of mdi_generate)",
+                         "traffic_note": "scaled from a 23-pass ncu capture of the same kernel (fused-phase kernel: captured with one block per head, see profiles/)", "scope": "decode phase of one step (all kernels of mdi_generate)",
                          "algorithmic_bytes": db["total"], "weight_bytes": db["weights"], "kv_bytes": db["kv"]},
             "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(S * P * 4),
                     "d2h_bytes_per_step": int(S * N * 4)},
