@@ -147,6 +147,7 @@ struct mdi_ctx {
     FzSeg *fz_segs = nullptr;
     int *fz_units = nullptr, *fz_err = nullptr;
     int fz_kv_pps = 1, fz_pair = 0, fz_kv_rows = 16;
+    bool fz_no_pair = false; // a cluster launch was refused once: one block per head from then on
     uint4 *fz_stream = nullptr;
     long long *fz_acc = nullptr;
     unsigned *fz_sync = nullptr;
@@ -906,7 +907,7 @@ int fz_setup(mdi_ctx *c) {
     // Pair mode: a head is served by the two blocks of a cluster (halves of its q,k,v rows, of the rows of every cache
     // page and of its output rows).  Needs even tile counts, pages of at least two rows, even team sizes with a cluster
     // per head, and all clusters resident at once.
-    bool pair = !getenv("MDI_FZ_NO_PAIR") && c->page_tokens >= 2 && (3 * hd / 16) % 2 == 0 && (d / 16) % 2 == 0 && n_sm >= 2;
+    bool pair = !c->fz_no_pair && !getenv("MDI_FZ_NO_PAIR") && c->page_tokens >= 2 && (3 * hd / 16) % 2 == 0 && (d / 16) % 2 == 0 && n_sm >= 2;
     if (pair) {
         for (int nb : {1, 2, 4}) CU(cudaFuncSetAttribute(fz_func(nb), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prop.sharedMemPerBlockOptin));
         cudaLaunchConfig_t cfg = {};
@@ -1051,6 +1052,11 @@ int fz_setup(mdi_ctx *c) {
     c->fz_smem = fz_smem_layout(NB, c->fz_slots, d, hd, c->fz_part_floats, c->pages_per_seq, c->fz_xb_stride, c->fz_hb_stride, c->fz_ob_stride).total;
     for (int nb : {1, 2, 4}) CU(cudaFuncSetAttribute(fz_func(nb), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->fz_smem));
     int rc;
+    {   // (a second plan after a refused cluster launch replaces the first one's buffers)
+        void *prev[] = {c->fz_sync, c->fz_err, c->fz_acc, c->fz_prof};
+        for (void *q : prev) if (q) cudaFree(q);
+        c->fz_sync = nullptr; c->fz_err = nullptr; c->fz_acc = nullptr; c->fz_prof = nullptr;
+    }
     if ((rc = dalloc(c, &c->fz_sync, (size_t)K * 64)) != MDI_OK) return rc;
     if ((rc = dalloc(c, &c->fz_err, 1)) != MDI_OK) return rc;
     if ((rc = dalloc(c, &c->fz_acc, (size_t)K * 3 * FZ_MAXNB * d)) != MDI_OK) return rc;
@@ -1252,7 +1258,20 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
         at[1].id = cudaLaunchAttributeClusterDimension;
         at[1].val.clusterDim.x = 2; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 2;
-        CU(cudaLaunchKernelExC(&cfg, fn, args));
+        const cudaError_t le = cudaLaunchKernelExC(&cfg, fn, args);
+        if (le != cudaSuccess) {
+            // The cooperative launch in clusters was refused by the runtime: plan again with one block per head, rebuild
+            // the weight streams and launch that.
+            cudaGetLastError();
+            if (trace) cudaFree(trace);
+            c->fz_no_pair = true;
+            c->fz_ok = false;
+            const int rs = fz_setup(c);
+            if (rs != MDI_OK) return rs;
+            if (!c->fz_ok || c->fz_pair) return fail(c, MDI_ERR_CUDA, "cluster launch refused (%s) and no plan without clusters", cudaGetErrorString(le));
+            c->fz_stale = true;
+            return fz_launch(c, n_samples, G, n_pass);
+        }
     } else {
         CU(cudaLaunchCooperativeKernel(fn, dim3(c->fz_grid), dim3(FZ_THREADS), args, c->fz_smem, c->main));
     }
