@@ -123,7 +123,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
                const mdi_options *opts, mdi_ctx **out);
 void mdi_destroy(mdi_ctx *ctx);
 
-/* "Load model chunk" (Algorithms 1 and 2).  One call per tensor; host_data is row-major
+/* Giving a node its chunk of the model (the loading step that opens Algorithms 1 and 2).  One call per tensor; host_data is row-major
  * [out_features][in_features] for matrices, element type shape.weight_dtype, nbytes its
  * exact size.  Names: "wte" [vocab][d], "wpe" [n_ctx][d] (GPT), "lnf.g", "lnf.b" (GPT),
  * "lm_head" [vocab][d] (untied), and per block i: "h.<i>.ln1.g", "h.<i>.ln1.b" (GPT),
@@ -135,7 +135,8 @@ void mdi_destroy(mdi_ctx *ctx);
  * Errors: ARG (unknown name), SHAPE (nbytes mismatch), CUDA. */
 int mdi_load_weights(mdi_ctx *ctx, const char *tensor_name, const void *host_data, size_t nbytes);
 
-/* First visit of a sample (Algorithm 1 "first iteration", Algorithm 2 "n-th cache is None"):
+/* First visit of a sample (the branch of Algorithm 1 taken on a sample's first iteration, and of Algorithm 2 taken
+ * while the node holds no cache for the sample yet):
  * the whole prompt goes through every partition in turn, filling cache rows 0..n_prompt-1 of
  * the sample's slot; only the last position reaches the output layers, whose result is the
  * sample's first new token (kept pending until mdi_generate returns it).  Work is enqueued

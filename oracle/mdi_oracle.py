@@ -328,7 +328,7 @@ class Oracle:
         out_lg = [[] for _ in range(S)]
         visits = [0] * S                     # starter visits per sample
         trace = []
-        for n in range(S):                   # "Place input tensors in input message queue"
+        for n in range(S):                   # every sample starts in the starter's input queue (Algorithm 1, initialisation)
             queues[0].append((n, None))
         tick = 0
         total_visits = S * (n_new + 1)

@@ -223,9 +223,13 @@ def test_zero_blocks_special_case():
 
 # ---------------- invariants the method relies on ---------------------------------------------
 
-@pytest.mark.parametrize("arch,dtype", [("gpt", I.DT_F32), ("llama", I.DT_BF16)])
-def test_I1_cached_decode_equals_full_recompute(arch, dtype):
-    shape = tiny_shape(arch, dtype)
+@pytest.mark.parametrize("arch,dtype,H,n_kv", [("gpt", I.DT_F32, 2, 2), ("llama", I.DT_BF16, 2, 2),
+                                               ("gpt", I.DT_F32, 4, 2), ("gpt", I.DT_BF16, 4, 1),
+                                               ("llama", I.DT_BF16, 4, 2), ("llama", I.DT_F32, 4, 1)])
+def test_I1_cached_decode_equals_full_recompute(arch, dtype, H, n_kv):
+    """Includes grouped-query shapes (several query heads reading one cached key/value head): the cached path picks
+    the key/value head of a query head by its own index arithmetic, the full-recompute path by another."""
+    shape = tiny_shape(arch, dtype, H=H, n_kv=n_kv)
     orc, _ = make_oracle(shape, std=0.2)
     prompt = [int(t) for t in I.make_prompts(shape.vocab, 1, 5)[0]]
     t_full, l_full = orc.generate_full_recompute(prompt, 10)
@@ -267,9 +271,10 @@ def test_I2_partition_boundaries_do_not_change_logits():
         assert np.array_equal(lg, base), b
 
 
-@pytest.mark.parametrize("S,K", [(1, 1), (1, 3), (2, 3), (3, 3), (5, 3), (3, 2), (5, 2), (2, 1)])
-def test_I3_pipeline_equals_sequential(S, K):
-    shape = tiny_shape("llama", I.DT_BF16, L=3)
+@pytest.mark.parametrize("S,K,n_kv", [(1, 1, 0), (1, 3, 0), (2, 3, 0), (3, 3, 0), (5, 3, 0), (3, 2, 0), (5, 2, 0), (2, 1, 0),
+                                      (3, 3, 2), (5, 2, 1)])
+def test_I3_pipeline_equals_sequential(S, K, n_kv):
+    shape = tiny_shape("llama", I.DT_BF16, L=3, H=4 if n_kv else 2, n_kv=n_kv or None)
     orc, _ = make_oracle(shape, std=0.2)
     bounds = {1: [0, 3], 2: [0, 1, 3], 3: [0, 1, 2, 3]}[K]
     prompts = [[int(t) for t in p[: 2 + s % 3]] for s, p in enumerate(I.make_prompts(shape.vocab, S, 4))]
