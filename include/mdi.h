@@ -96,6 +96,16 @@ typedef struct {
                           1: always the stream scheduler (one stream per partition, event handoff);
                           2: the phase-per-matrix persistent kernel, or fail;
                           3: the fused-phase persistent kernel, or fail */
+    int in_kernel_timing; /* 1: the persistent kernels time themselves (mdi_get_partition_times); costs a few percent */
+    int fused_blocks_per_head; /* fused-phase kernel: 0 (default) two thread blocks of a cluster share a head where every
+                          team has a cluster per head, else one block per head; 1: always one block per head (plain
+                          cooperative launch, no clusters) */
+    int debug_refuse_cluster_launch; /* checking aid: 1 makes the first fused-phase launch in clusters behave as if the
+                          runtime had refused it (nothing is launched), so that the library plans again with one block
+                          per head, as it does after a real refusal */
+    int trace_slot;    /* with in_kernel_timing: s > 0 makes thread 0 of every block of the fused-phase kernel record a
+                          time stamp at every change of timing category while it serves schedule slot s - 1
+                          (mdi_get_trace) */
 } mdi_options;
 
 typedef struct {
@@ -197,20 +207,24 @@ int mdi_get_stats(mdi_ctx *ctx, mdi_stats *out);
  * per-thread-block copy of the partition's matrices), cf. Tables I-II. */
 int64_t mdi_memory_bytes(mdi_ctx *ctx, int partition);
 /* Tracing aid (the paper times token arrival on the starter; here each partition's team of thread
- * blocks times itself).  With MDI_PK_PROFILE set in the environment at mdi_create, the persistent kernel
- * accumulates, per thread block, the nanoseconds spent in: [0] waiting for the input edge, [1] staging
+ * blocks times itself).  With in_kernel_timing set at mdi_create, the persistent kernel accumulates, per
+ * thread block, the nanoseconds spent in: [0] waiting for the input edge, [1] staging
  * and normalising inputs, [2] streaming weight tiles, [3] team barriers, [4] attention, [5] choosing
  * tokens, [6] producer warp waiting for a free ring slot, [7] producer warp total, and within [2]:
  * [8] waiting for a tile to land, [9] multiply-accumulate, [10] reduction and epilogue.  When the last call ran the
  * fused-phase kernel the categories are: [0] input edge, [1] norm prologues, [2] row parts (split along k; for the
  * output layer: unused), [3] bias / activation / cache append after a row part, [4] attention, [5] column parts and the
  * output layer's rows, [6] and [7] as above, [8] team barriers, [9] end of step (token choice or handoff), [11] time
- * inside [2], [4], [5] spent waiting for ring slots.  With MDI_FZ_TRACE=<schedule slot> and MDI_FZ_TRACE_FILE=<path>
- * also set, thread 0 of every block writes a time stamp at every category change of that slot (text, one line per
- * block, "category:nanoseconds" pairs).  This call averages
+ * inside [2], [4], [5] spent waiting for ring slots.  This call averages
  * them over the partition's blocks for the last mdi_generate, in milliseconds, into out_ms[0..n).
  * Returns the number of blocks of the partition (> 0) or a negative error (STATE when timing is off). */
 int mdi_get_partition_times(mdi_ctx *ctx, int partition, double *out_ms, int n);
+/* Time stamps of the traced schedule slot (options.trace_slot) of the last mdi_generate that ran the fused-phase
+ * kernel: per thread block MDI_TRACE_WORDS 64-bit words, each (nanoseconds << 4) | category in the order the
+ * block went through them, 0 = unused.  Copies min(n_words, blocks * MDI_TRACE_WORDS) words to out_host and returns
+ * the number of blocks (> 0), or a negative error (STATE when no trace was taken). */
+#define MDI_TRACE_WORDS 128
+int mdi_get_trace(mdi_ctx *ctx, uint64_t *out_host, int n_words);
 /* Wait for everything enqueued on the context's streams. */
 int mdi_sync(mdi_ctx *ctx);
 /* Greedy token choice for callers that must not allocate.  (The paper has no counterpart: this is a

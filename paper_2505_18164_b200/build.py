@@ -12,7 +12,7 @@ LIB_MDI = os.path.join(_HERE, "libmdi.so")
 LIB_INPUTS = os.path.join(_HERE, "libmdi_inputs.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--use_fast_math=false", "-Xcompiler", "-fPIC", "-shared"]
+              "-Xcompiler", "-fPIC", "-shared"]
 
 
 def _stale(target: str, sources) -> bool:
@@ -36,8 +36,7 @@ def build_mdi(force: bool = False, verbose: bool = False) -> str:
     deps = cu + glob.glob(os.path.join(_CSRC, "*.cuh")) + glob.glob(os.path.join(_ROOT, "include", "*.h"))
     if force or _stale(LIB_MDI, deps):
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
-        cmd = [nvcc] + flags + (["-Xptxas", "-v"] if verbose else []) + \
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
               ["-I", os.path.join(_ROOT, "include"), "-o", LIB_MDI] + cu
         subprocess.check_call(cmd)
     return LIB_MDI

@@ -151,7 +151,9 @@ struct mdi_ctx {
     uint4 *fz_stream = nullptr;
     long long *fz_acc = nullptr;
     unsigned *fz_sync = nullptr;
-    unsigned long long *fz_prof = nullptr;
+    unsigned long long *fz_prof = nullptr, *fz_trace = nullptr;
+    int fz_trace_blocks = 0;
+    bool fz_refusal_faked = false;
     int64_t fz_stream_bytes = 0;
     std::vector<int64_t> fz_team_stream_bytes; // per partition: bytes of its blocks' weight streams
     mdi_stats st{};
@@ -190,28 +192,26 @@ inline void count_launch(mdi_ctx *c) {
     if (c->capturing) ++c->cap_launches; else ++c->st.kernel_launches;
 }
 
-// Launch with the programmatic-serialization attribute when g_pdl is set (the kernels of the tensor-core chain
+// Launch with the programmatic-serialization attribute when pdl is set (the kernels of the tensor-core chain
 // call griddepcontrol.wait before touching their predecessor's results), else as a plain launch.
-bool g_pdl = false;
 template <typename... KArgs, typename... Args>
-void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+void launch_k(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
-    cfg.numAttrs = g_pdl ? 1 : 0;
+    cfg.numAttrs = pdl ? 1 : 0;
     cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 // ---- kernel dispatch ------------------------------------------------------------------------------
 constexpr size_t LIN_SMEM_MAX = 200 * 1024;
 
-// The key/value cache is fp32 unless the context asked for a cache in the (2-byte) weight type.
-bool g_kv_f32_dispatch = true;
-template <int NB, typename WT, int MODE> void lin_launch(const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st) {
-    if (MODE == LIN_QKV && g_kv_f32_dispatch) k_linear<NB, WT, MODE, float><<<grid, LIN_THREADS, smem, st>>>(a, bt);
+// The key/value cache is fp32 (kv_f32) unless the context asked for a cache in the (2-byte) weight type.
+template <int NB, typename WT, int MODE> void lin_launch(const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st, bool kv_f32) {
+    if (MODE == LIN_QKV && kv_f32) k_linear<NB, WT, MODE, float><<<grid, LIN_THREADS, smem, st>>>(a, bt);
     else k_linear<NB, WT, MODE><<<grid, LIN_THREADS, smem, st>>>(a, bt);
 }
 template <int NB, typename WT, int MODE> cudaError_t lin_attr() {
@@ -220,21 +220,21 @@ template <int NB, typename WT, int MODE> cudaError_t lin_attr() {
         e = cudaFuncSetAttribute(k_linear<NB, WT, MODE, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LIN_SMEM_MAX);
     return e;
 }
-template <typename WT, int MODE> void lin_nb(int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st) {
+template <typename WT, int MODE> void lin_nb(int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st, bool kv_f32) {
     switch (nb) {
-        case 1: lin_launch<1, WT, MODE>(a, bt, grid, smem, st); break;
-        case 2: lin_launch<2, WT, MODE>(a, bt, grid, smem, st); break;
-        case 4: lin_launch<4, WT, MODE>(a, bt, grid, smem, st); break;
-        default: lin_launch<8, WT, MODE>(a, bt, grid, smem, st); break;
+        case 1: lin_launch<1, WT, MODE>(a, bt, grid, smem, st, kv_f32); break;
+        case 2: lin_launch<2, WT, MODE>(a, bt, grid, smem, st, kv_f32); break;
+        case 4: lin_launch<4, WT, MODE>(a, bt, grid, smem, st, kv_f32); break;
+        default: lin_launch<8, WT, MODE>(a, bt, grid, smem, st, kv_f32); break;
     }
 }
-template <typename WT> void lin_mode(int mode, int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st) {
+template <typename WT> void lin_mode(int mode, int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st, bool kv_f32) {
     switch (mode) {
-        case LIN_QKV: lin_nb<WT, LIN_QKV>(nb, a, bt, grid, smem, st); break;
-        case LIN_ACT: lin_nb<WT, LIN_ACT>(nb, a, bt, grid, smem, st); break;
-        case LIN_GATEUP: lin_nb<WT, LIN_GATEUP>(nb, a, bt, grid, smem, st); break;
-        case LIN_HEAD: lin_nb<WT, LIN_HEAD>(nb, a, bt, grid, smem, st); break;
-        default: lin_nb<WT, LIN_RESID>(nb, a, bt, grid, smem, st); break;
+        case LIN_QKV: lin_nb<WT, LIN_QKV>(nb, a, bt, grid, smem, st, kv_f32); break;
+        case LIN_ACT: lin_nb<WT, LIN_ACT>(nb, a, bt, grid, smem, st, kv_f32); break;
+        case LIN_GATEUP: lin_nb<WT, LIN_GATEUP>(nb, a, bt, grid, smem, st, kv_f32); break;
+        case LIN_HEAD: lin_nb<WT, LIN_HEAD>(nb, a, bt, grid, smem, st, kv_f32); break;
+        default: lin_nb<WT, LIN_RESID>(nb, a, bt, grid, smem, st, kv_f32); break;
     }
 }
 template <typename WT, int MODE> cudaError_t lin_attr_nb() {
@@ -282,20 +282,19 @@ int linear(mdi_ctx *c, int mode, LinArgs a, const Batch &bt, cudaStream_t st) {
         if (a.x_res) b.x_res = a.x_res + (size_t)first * a.n_rows;
         if (a.x_out) b.x_out = a.x_out + (size_t)first * a.n_rows;
         const size_t smem = (size_t)nb * a.in_dim * 4;
-        g_kv_f32_dispatch = c->kv_f32;
-        if (f32) lin_mode<float>(mode, nb, b, sb, grid, smem, st);
-        else lin_mode<__nv_bfloat16>(mode, nb, b, sb, grid, smem, st);
+        if (f32) lin_mode<float>(mode, nb, b, sb, grid, smem, st, c->kv_f32);
+        else lin_mode<__nv_bfloat16>(mode, nb, b, sb, grid, smem, st, c->kv_f32);
         count_launch(c);
     }
     return MDI_OK;
 }
 
-template <typename KT> void attn_hd(int hd, const AttnArgs &a, const Batch &bt, dim3 grid, cudaStream_t st) {
+template <typename KT> void attn_hd(bool pdl, int hd, const AttnArgs &a, const Batch &bt, dim3 grid, cudaStream_t st) {
     switch (hd) {
-        case 16: launch_k(k_attn_decode<KT, 16>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
-        case 32: launch_k(k_attn_decode<KT, 32>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
-        case 64: launch_k(k_attn_decode<KT, 64>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
-        default: launch_k(k_attn_decode<KT, 128>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
+        case 16: launch_k(pdl, k_attn_decode<KT, 16>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
+        case 32: launch_k(pdl, k_attn_decode<KT, 32>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
+        case 64: launch_k(pdl, k_attn_decode<KT, 64>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
+        default: launch_k(pdl, k_attn_decode<KT, 128>, grid, dim3(ATT_THREADS), 0, st, a, bt); break;
     }
 }
 
@@ -380,7 +379,7 @@ int enqueue_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in
             a.layer_local = l - P.lo; a.n_head = s.n_head; a.n_split = c->n_split; a.pos = P.pos_dev;
             a.scale = 1.0f / std::sqrt((float)s.head_dim);
             dim3 g(s.n_head, c->n_split, bt.n);
-            if (c->kv_f32) attn_hd<float>(s.head_dim, a, bt, g, st); else attn_hd<__nv_bfloat16>(s.head_dim, a, bt, g, st);
+            if (c->kv_f32) attn_hd<float>(false, s.head_dim, a, bt, g, st); else attn_hd<__nv_bfloat16>(false, s.head_dim, a, bt, g, st);
             count_launch(c);
         }
         {   // output projection + residual
@@ -425,7 +424,6 @@ constexpr int PF_SPLIT_MAX = 8; // K splits of the GEMMs with few row tiles (out
 int pf_setup(mdi_ctx *c) {
     const mdi_model_shape &s = c->s;
     c->pf_tc = s.weight_dtype == MDI_DTYPE_BF16 && c->o.prefill_mode != 1;
-    c->pdl = getenv("MDI_NO_PDL") == nullptr;
     // Which decode steps use the tensor-core linear layers (stream scheduler): by default groups of 5 or more
     // samples, and every group when one block's matrices are 48 MB or more (then a step moves enough bytes per
     // kernel for launches not to matter, and TMA-fed GEMM tiles stream faster than the CUDA-core tiles).
@@ -494,7 +492,7 @@ int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, c
     TgArgs a{};
     a.n_rows = n_rows; a.K = K; a.T = T; a.n_tile = n_tile; a.bias = bias; a.resid = resid; a.act = act; a.y = y; a.ldy = n_rows;
     a.err = c->tg_err; a.partial = P.pf_part; a.out_hi = out_hi; a.out_lo = out_lo;
-    launch_k(k_tc_gemm, dim3(grid_x, (T + n_tile - 1) / n_tile, splits), dim3(TG_THREADS), tg_smem_bytes(n_tile), st, *mw, *mhi, *mlo, a);
+    launch_k(c->pdl, k_tc_gemm, dim3(grid_x, (T + n_tile - 1) / n_tile, splits), dim3(TG_THREADS), tg_smem_bytes(n_tile), st, *mw, *mhi, *mlo, a);
     count_launch(c);
     if (pending) {
         pending->splits = splits > 1 ? splits : 0;
@@ -504,13 +502,13 @@ int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, c
     return MDI_OK;
 }
 
-template <typename KT> void pf_attn_hd(int hd, dim3 g, cudaStream_t st, const float *q, __nv_bfloat16 *ohi, __nv_bfloat16 *olo,
+template <typename KT> void pf_attn_hd(bool pdl, int hd, dim3 g, cudaStream_t st, const float *q, __nv_bfloat16 *ohi, __nv_bfloat16 *olo,
                                        const KvView &kv, int ll, int n_head, const int *pos, int slot, float scale) {
     switch (hd) {
-        case 16: launch_k(k_pf_attn<KT, 16>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
-        case 32: launch_k(k_pf_attn<KT, 32>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
-        case 64: launch_k(k_pf_attn<KT, 64>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
-        default: launch_k(k_pf_attn<KT, 128>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        case 16: launch_k(pdl, k_pf_attn<KT, 16>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        case 32: launch_k(pdl, k_pf_attn<KT, 32>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        case 64: launch_k(pdl, k_pf_attn<KT, 64>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
+        default: launch_k(pdl, k_pf_attn<KT, 128>, g, dim3(ATT_THREADS), 0, st, q, ohi, olo, kv, ll, n_head, pos, slot, scale); break;
     }
 }
 
@@ -529,9 +527,9 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
     const float scale = 1.0f / std::sqrt((float)s.head_dim);
     __nv_bfloat16 *hi = (__nv_bfloat16 *)P.pf_hi, *lo = (__nv_bfloat16 *)P.pf_lo;
     int rc;
-    struct PdlScope { PdlScope(bool on) { g_pdl = on; } ~PdlScope() { g_pdl = false; } } pdl_scope(c->pdl);
+    const bool pdl = c->pdl;
     if (!bt && p == 0) {
-        launch_k(k_pf_embed<__nv_bfloat16>, dim3(T), dim3(256), 0, st, (const __nv_bfloat16 *)c->wte, (const __nv_bfloat16 *)c->wpe, d, s.vocab, tok_dev,
+        launch_k(pdl, k_pf_embed<__nv_bfloat16>, dim3(T), dim3(256), 0, st, (const __nv_bfloat16 *)c->wte, (const __nv_bfloat16 *)c->wpe, d, s.vocab, tok_dev,
                                                     P.pos_dev, slot, P.pf_xa);
         count_launch(c);
         x_in = P.pf_xa;
@@ -542,39 +540,39 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
         const int ll = l - P.lo;
         const float *xin_l = l == P.lo ? x_in : x_out;
         // norm 1 (first completing the residual stream if the previous GEMM was split)
-        launch_k(k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, pend.splits ? pend.resid : xin_l, d, norm, L.ln1g, L.ln1b, s.norm_eps, hi, lo, P.pf_part,
+        launch_k(pdl, k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, pend.splits ? pend.resid : xin_l, d, norm, L.ln1g, L.ln1b, s.norm_eps, hi, lo, P.pf_part,
                                                   pend.splits, T, pend.bias, x_out);
         count_launch(c);
         pend = PfPending();
         if ((rc = pf_gemm(c, P, L.wqkv, qw + 2 * kw, d, T, L.bqkv, nullptr, TG_NONE, P.pf_qkv, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
         if (bt) {
-            if (c->kv_f32) launch_k(k_bt_rope_append<float>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
-            else launch_k(k_bt_rope_append<__nv_bfloat16>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
+            if (c->kv_f32) launch_k(pdl, k_bt_rope_append<float>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
+            else launch_k(pdl, k_bt_rope_append<__nv_bfloat16>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
             count_launch(c);
             AttnArgs a{};
             a.q = P.qbuf; a.o = P.obuf; a.part = P.part; a.ticket = P.attn_ticket; a.kv = kv; a.layer_local = ll; a.n_head = s.n_head;
             a.n_split = c->n_split; a.pos = P.pos_dev; a.scale = scale; a.o_hi = hi; a.o_lo = lo;
             const dim3 g(s.n_head, c->n_split, T);
-            if (c->kv_f32) attn_hd<float>(s.head_dim, a, *bt, g, st); else attn_hd<__nv_bfloat16>(s.head_dim, a, *bt, g, st);
+            if (c->kv_f32) attn_hd<float>(pdl, s.head_dim, a, *bt, g, st); else attn_hd<__nv_bfloat16>(pdl, s.head_dim, a, *bt, g, st);
             count_launch(c);
         } else {
-            if (c->kv_f32) launch_k(k_pf_rope_append<float>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
-            else launch_k(k_pf_rope_append<__nv_bfloat16>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
+            if (c->kv_f32) launch_k(pdl, k_pf_rope_append<float>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
+            else launch_k(pdl, k_pf_rope_append<__nv_bfloat16>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
             count_launch(c);
-            if (c->kv_f32) pf_attn_hd<float>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
-            else pf_attn_hd<__nv_bfloat16>(s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
+            if (c->kv_f32) pf_attn_hd<float>(pdl, s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
+            else pf_attn_hd<__nv_bfloat16>(pdl, s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
             count_launch(c);
         }
         // output projection + residual -> x_out (or partial sums, completed by the next kernel)
         PfPending po;
         if ((rc = pf_gemm(c, P, L.wo, d, qw, T, L.bo, xin_l, TG_NONE, x_out, nullptr, nullptr, &po, st)) != MDI_OK) return rc;
-        launch_k(k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, po.splits ? po.resid : x_out, d, norm, L.ln2g, L.ln2b, s.norm_eps, hi, lo, P.pf_part, po.splits, T,
+        launch_k(pdl, k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, po.splits ? po.resid : x_out, d, norm, L.ln2g, L.ln2b, s.norm_eps, hi, lo, P.pf_part, po.splits, T,
                                                   po.bias, x_out);
         count_launch(c);
         if (s.act == MDI_ACT_SWIGLU) {
             if ((rc = pf_gemm(c, P, L.wgate, F, d, T, nullptr, nullptr, TG_NONE, P.pf_h, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
             if ((rc = pf_gemm(c, P, L.wup, F, d, T, nullptr, nullptr, TG_NONE, P.pf_u, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
-            launch_k(k_pf_swiglu_split, dim3(T), dim3(256), 0, st, P.pf_h, P.pf_u, F, hi, lo);
+            launch_k(pdl, k_pf_swiglu_split, dim3(T), dim3(256), 0, st, P.pf_h, P.pf_u, F, hi, lo);
             count_launch(c);
             if ((rc = pf_gemm(c, P, L.wdown, d, F, T, nullptr, x_out, TG_NONE, x_out, nullptr, nullptr, &pend, st)) != MDI_OK) return rc;
         } else {
@@ -582,18 +580,18 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
             if ((rc = pf_gemm(c, P, L.w1, F, d, T, L.b1, nullptr, s.act == MDI_ACT_GELU_ERF ? TG_GELU_ERF : TG_GELU_TANH, P.pf_h, nullptr, nullptr,
                               nullptr, st)) != MDI_OK)
                 return rc;
-            launch_k(k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo, nullptr, 0, T, nullptr, nullptr);
+            launch_k(pdl, k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo, nullptr, 0, T, nullptr, nullptr);
             count_launch(c);
             if ((rc = pf_gemm(c, P, L.w2, d, F, T, L.b2, x_out, TG_NONE, x_out, nullptr, nullptr, &pend, st)) != MDI_OK) return rc;
         }
     }
     if (pend.splits) { // complete the residual stream after the last block
-        launch_k(k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, pend.resid, d, NORM_NONE, nullptr, nullptr, 0.f, nullptr, nullptr, P.pf_part, pend.splits, T,
+        launch_k(pdl, k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, pend.resid, d, NORM_NONE, nullptr, nullptr, 0.f, nullptr, nullptr, P.pf_part, pend.splits, T,
                                                   pend.bias, x_out);
         count_launch(c);
     }
-    if (bt) launch_k(k_bt_advance, dim3(1), dim3(32), 0, st, P.pos_dev, *bt);
-    else launch_k(k_pf_advance, dim3(1), dim3(32), 0, st, P.pos_dev, slot, T);
+    if (bt) launch_k(pdl, k_bt_advance, dim3(1), dim3(32), 0, st, P.pos_dev, *bt);
+    else launch_k(pdl, k_pf_advance, dim3(1), dim3(32), 0, st, P.pos_dev, slot, T);
     count_launch(c);
     return MDI_OK;
 }
@@ -730,17 +728,7 @@ int pk_setup(mdi_ctx *c) {
     }
     // team sizes
     std::vector<int> n_cta(K, 1);
-    const char *env = getenv("MDI_TEAM_CTAS");
-    bool from_env = false;
-    if (env) {
-        std::vector<int> v;
-        const char *q = env;
-        while (*q) { v.push_back(atoi(q)); while (*q && *q != ',') ++q; if (*q == ',') ++q; }
-        int tot = 0;
-        for (int x : v) tot += x;
-        if ((int)v.size() == K && tot <= c->n_sm && *std::min_element(v.begin(), v.end()) >= 1) { n_cta = v; from_env = true; }
-    }
-    if (!from_env) {
+    {
         // Proportional to the bytes a step streams, then rounded down to a size that deals the row blocks of
         // the d_model-row matrices (and the attention items) out evenly - uneven shares make every phase wait
         // for the blocks with one more tile - unless that would give up more than 30% of the share.
@@ -772,7 +760,7 @@ int pk_setup(mdi_ctx *c) {
     if ((rcx = dalloc(c, &c->pk_sync, (size_t)K * 64)) != MDI_OK) return rcx;
     if ((rcx = dalloc(c, &c->pk_err, 1)) != MDI_OK) return rcx;
     if ((rcx = dalloc(c, &c->pk_prof, (size_t)c->n_sm * PK_PROF_N)) != MDI_OK) return rcx;
-    c->pk_prof_on = getenv("MDI_PK_PROFILE") != nullptr;
+    c->pk_prof_on = c->o.in_kernel_timing != 0;
     for (int p = 0; p < K; ++p) {
         Partition &P = c->part[p];
         PkTeam &T = c->pk_teams_host[p];
@@ -892,7 +880,6 @@ int fz_setup(mdi_ctx *c) {
     const bool want = c->scheduler == 3;
     auto no = [&](const char *why) { return want ? fail(c, MDI_ERR_SHAPE, "fused-phase scheduler: %s", why) : MDI_OK; };
     if (c->scheduler == 1 || c->scheduler == 2) return MDI_OK;
-    if (getenv("MDI_NO_FUSED") && !want) return MDI_OK;
     if (s.arch != MDI_ARCH_GPT || s.weight_dtype != MDI_DTYPE_BF16 || !c->kv_f32) return no("needs the GPT block, bf16 weights and an fp32 cache");
     if (s.n_kv_head != H || H * hd != d) return no("needs n_kv_head = n_head and n_head * head_dim = d_model");
     if (d % 16 || s.d_ff % 16 || hd % 16) return no("widths must be multiples of 16");
@@ -907,7 +894,7 @@ int fz_setup(mdi_ctx *c) {
     // Pair mode: a head is served by the two blocks of a cluster (halves of its q,k,v rows, of the rows of every cache
     // page and of its output rows).  Needs even tile counts, pages of at least two rows, even team sizes with a cluster
     // per head, and all clusters resident at once.
-    bool pair = !c->fz_no_pair && !getenv("MDI_FZ_NO_PAIR") && c->page_tokens >= 2 && (3 * hd / 16) % 2 == 0 && (d / 16) % 2 == 0 && n_sm >= 2;
+    bool pair = !c->fz_no_pair && c->o.fused_blocks_per_head != 1 && c->page_tokens >= 2 && (3 * hd / 16) % 2 == 0 && (d / 16) % 2 == 0 && n_sm >= 2;
     if (pair) {
         for (int nb : {1, 2, 4}) CU(cudaFuncSetAttribute(fz_func(nb), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prop.sharedMemPerBlockOptin));
         cudaLaunchConfig_t cfg = {};
@@ -929,16 +916,6 @@ int fz_setup(mdi_ctx *c) {
     }
     std::vector<int> n_cta(K, 0);
     auto team_sizes = [&](bool even) {
-        const char *env = getenv("MDI_FZ_TEAM_CTAS");
-        if (env) {
-            std::vector<int> v;
-            const char *q = env;
-            while (*q) { v.push_back(atoi(q)); while (*q && *q != ',') ++q; if (*q == ',') ++q; }
-            int tot = 0;
-            bool all_even = true;
-            for (int x : v) { tot += x; all_even = all_even && x % 2 == 0; }
-            if ((int)v.size() == K && tot <= n_sm && *std::min_element(v.begin(), v.end()) >= 1 && (all_even || !even)) { n_cta = v; return; }
-        }
         double tot = 0;
         for (double b : bytes) tot += b;
         int used = 0, big = 0;
@@ -1060,7 +1037,7 @@ int fz_setup(mdi_ctx *c) {
     if ((rc = dalloc(c, &c->fz_sync, (size_t)K * 64)) != MDI_OK) return rc;
     if ((rc = dalloc(c, &c->fz_err, 1)) != MDI_OK) return rc;
     if ((rc = dalloc(c, &c->fz_acc, (size_t)K * 3 * FZ_MAXNB * d)) != MDI_OK) return rc;
-    c->fz_prof_on = getenv("MDI_PK_PROFILE") != nullptr;
+    c->fz_prof_on = c->o.in_kernel_timing != 0;
     if (c->fz_prof_on && (rc = dalloc(c, &c->fz_prof, (size_t)c->fz_grid * PK_PROF_N)) != MDI_OK) return rc;
     c->fz_ok = true;
     return MDI_OK;
@@ -1237,14 +1214,18 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     P.withhold_partition = c->withhold_once;
     c->withhold_once = -1;
     P.prof = c->fz_prof_on ? c->fz_prof : nullptr;
-    // MDI_FZ_TRACE=<schedule slot>: with in-kernel timing on, thread 0 of every block also records a time stamp at every
-    // phase boundary of that slot; the stamps are written as text to MDI_FZ_TRACE_FILE after the call (a tuning aid)
-    unsigned long long *trace = nullptr;
-    if (c->fz_prof_on && getenv("MDI_FZ_TRACE") && getenv("MDI_FZ_TRACE_FILE")) {
-        CU(cudaMalloc((void **)&trace, (size_t)c->fz_grid * FZ_TRACE_N * 8));
-        CU(cudaMemsetAsync(trace, 0, (size_t)c->fz_grid * FZ_TRACE_N * 8, c->main));
-        P.trace = trace;
-        P.trace_step = atoi(getenv("MDI_FZ_TRACE"));
+    // trace_slot: with in-kernel timing on, thread 0 of every block also records a time stamp at every category
+    // change while it serves that schedule slot (read back with mdi_get_trace)
+    if (c->fz_prof_on && c->o.trace_slot > 0) {
+        if (!c->fz_trace || c->fz_trace_blocks != c->fz_grid) {
+            if (c->fz_trace) cudaFree(c->fz_trace);
+            c->fz_trace = nullptr;
+            CU(cudaMalloc((void **)&c->fz_trace, (size_t)c->fz_grid * FZ_TRACE_N * 8));
+            c->fz_trace_blocks = c->fz_grid;
+        }
+        CU(cudaMemsetAsync(c->fz_trace, 0, (size_t)c->fz_grid * FZ_TRACE_N * 8, c->main));
+        P.trace = c->fz_trace;
+        P.trace_step = c->o.trace_slot - 1;
     }
     // the template parameter fixes the accumulator stride, so it is the context's group size, not this call's
     const void *fn = fz_func(c->fz_nb);
@@ -1258,12 +1239,14 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
         at[1].id = cudaLaunchAttributeClusterDimension;
         at[1].val.clusterDim.x = 2; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 2;
-        const cudaError_t le = cudaLaunchKernelExC(&cfg, fn, args);
+        // (debug_refuse_cluster_launch: behave once as if the runtime had refused, without launching anything)
+        const bool pretend = c->o.debug_refuse_cluster_launch == 1 && !c->fz_refusal_faked;
+        c->fz_refusal_faked = c->fz_refusal_faked || pretend;
+        const cudaError_t le = pretend ? cudaErrorCooperativeLaunchTooLarge : cudaLaunchKernelExC(&cfg, fn, args);
         if (le != cudaSuccess) {
             // The cooperative launch in clusters was refused by the runtime: plan again with one block per head, rebuild
             // the weight streams and launch that.
             cudaGetLastError();
-            if (trace) cudaFree(trace);
             c->fz_no_pair = true;
             c->fz_ok = false;
             const int rs = fz_setup(c);
@@ -1277,21 +1260,6 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     }
     ++c->st.kernel_launches;
     c->st.stage_steps += (int64_t)c->K * n_pass * G;
-    if (trace) {
-        std::vector<unsigned long long> h((size_t)c->fz_grid * FZ_TRACE_N);
-        cudaStreamSynchronize(c->main);
-        cudaMemcpy(h.data(), trace, h.size() * 8, cudaMemcpyDeviceToHost);
-        cudaFree(trace);
-        if (FILE *f = fopen(getenv("MDI_FZ_TRACE_FILE"), "w")) {
-            for (int b = 0; b < c->fz_grid; ++b) {
-                fprintf(f, "%d", b);
-                for (int i = 0; i < FZ_TRACE_N && h[(size_t)b * FZ_TRACE_N + i]; ++i)
-                    fprintf(f, " %llu:%llu", h[(size_t)b * FZ_TRACE_N + i] & 15ull, h[(size_t)b * FZ_TRACE_N + i] >> 4);
-                fprintf(f, "\n");
-            }
-            fclose(f);
-        }
-    }
     return MDI_OK;
 }
 
@@ -1327,7 +1295,7 @@ void mdi_destroy(mdi_ctx *c) {
     }
     void *ptrs[] = {c->rope_cos, c->rope_sin, c->logits, c->head_pv, c->head_pi, c->head_ticket, c->cur_tok, c->tok_log,
                     c->gen_count, c->teacher, c->n_teacher, c->prompt_buf, c->pk_teams, c->pk_phases, c->pk_sync, c->pk_err, c->pk_prof, c->tg_err,
-                    c->fz_teams, c->fz_phases, c->fz_works, c->fz_blocks, c->fz_segs, c->fz_units, c->fz_err, c->fz_stream, c->fz_acc, c->fz_sync, c->fz_prof};
+                    c->fz_teams, c->fz_phases, c->fz_works, c->fz_blocks, c->fz_segs, c->fz_units, c->fz_err, c->fz_stream, c->fz_acc, c->fz_sync, c->fz_prof, c->fz_trace};
     for (void *q : ptrs) if (q) cudaFree(q);
     cudaEvent_t evs[] = {c->ev_fork, c->ev_fork_cap, c->ev_t0, c->ev_t1, c->ev_pf0, c->ev_pf1};
     for (auto e : evs) if (e) cudaEventDestroy(e);
@@ -1562,8 +1530,11 @@ int mdi_reset_sample(mdi_ctx *c, int sample) {
     if (!c) return MDI_ERR_ARG;
     if (sample < 0 || sample >= c->S) return fail(c, MDI_ERR_ARG, "sample %d out of range", sample);
     CU(cudaSetDevice(c->dev));
-    CU(cudaDeviceSynchronize());
-    const int zero = 0;
+    // No device-wide wait: mdi_generate returns only when its work is done, and whatever a first visit or mdi_step
+    // has left on a partition's stream precedes, on that same stream, both the clearing below and any later work
+    // that could take over the pages given back here (a partition's pool is only ever touched from its stream, or
+    // from a persistent launch that waits for all partition streams).
+    const int K = c->K;
     for (auto &P : c->part) {
         const int Lp = P.hi - P.lo;
         for (int l = 0; l < Lp; ++l)
@@ -1574,10 +1545,11 @@ int mdi_reset_sample(mdi_ctx *c, int sample) {
             }
         P.pages_of_slot[sample] = 0;
         P.pos_host[sample] = 0;
-        CU(cudaMemcpy(P.pos_dev + sample, &zero, 4, cudaMemcpyHostToDevice));
+        CU(cudaMemsetAsync(P.pos_dev + sample, 0, 4, P.stream));
     }
-    CU(cudaMemcpy(c->gen_count + sample, &zero, 4, cudaMemcpyHostToDevice));
-    CU(cudaMemcpy(c->n_teacher + sample, &zero, 4, cudaMemcpyHostToDevice));
+    // counters of the output layers: written by kernels of the last partition's stream
+    CU(cudaMemsetAsync(c->gen_count + sample, 0, 4, c->part[K - 1].stream));
+    CU(cudaMemsetAsync(c->n_teacher + sample, 0, 4, c->part[K - 1].stream));
     c->gen_host[sample] = c->returned_host[sample] = c->prefilled[sample] = 0;
     return MDI_OK;
 }
@@ -1588,8 +1560,11 @@ int mdi_set_teacher_tokens(mdi_ctx *c, int sample, const int32_t *tok, int n) {
     if (n > c->s.n_ctx) return fail(c, MDI_ERR_CONTEXT, "more teacher tokens than n_ctx");
     if (c->prefilled[sample]) return fail(c, MDI_ERR_STATE, "set teacher tokens before the sample's prefill");
     CU(cudaSetDevice(c->dev));
-    if (n) CU(cudaMemcpy(c->teacher + (size_t)sample * c->s.n_ctx, tok, (size_t)n * 4, cudaMemcpyHostToDevice));
-    CU(cudaMemcpy(c->n_teacher + sample, &n, 4, cudaMemcpyHostToDevice));
+    // on the stream whose kernels read them (and after a preceding mdi_reset_sample's clearing on that stream)
+    cudaStream_t st = c->part[c->K - 1].stream;
+    if (n) CU(cudaMemcpyAsync(c->teacher + (size_t)sample * c->s.n_ctx, tok, (size_t)n * 4, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(c->n_teacher + sample, &n, 4, cudaMemcpyHostToDevice, st));
+    CU(cudaStreamSynchronize(st));
     return MDI_OK;
 }
 
@@ -1758,7 +1733,6 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
     if ((rc = pf_check(c)) != MDI_OK) return rc;
     const long total = (long)n_pass * K;        // phase slots per partition
     const long t_total = total ? total + K - 1 : 0;
-    long t = 0;
     // fused-phase kernel where the shape fits it, else the phase-per-matrix kernel, else streams
     const bool small_groups = c->temperature <= 0.f && (n_samples + G - 1) / G <= PK_MAXNB &&
                               !(c->pf_tc && c->scheduler == 0 && (n_samples + G - 1) / G >= c->tc_min_group);
@@ -1766,76 +1740,92 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
     const bool use_pk = !use_fz && c->pk_ok && c->scheduler != 1 && c->scheduler != 3 && small_groups && pk_tile_count_fits(c, n_pass, G);
     if (c->scheduler == 2 && !use_pk) return fail(c, MDI_ERR_SHAPE, "persistent scheduler unavailable for this call");
     if (c->scheduler == 3 && !use_fz) return fail(c, MDI_ERR_SHAPE, "fused-phase scheduler unavailable for this call");
-    if (t_total && use_fz) {
-        if ((rc = fz_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
-        c->last_kernel = 2;
-    } else if (t_total && use_pk) {
-        if ((rc = pk_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
-        c->last_kernel = 1;
-    } else if (t_total) {
-        const int R = c->rounds_per_graph;
-        const long t_steady = K > 1 ? K : 0; // first tick, multiple of K, from which every partition is in steady state
-        // Steady-state windows are replayed from CUDA graphs: first windows of R rounds, then windows of one round
-        // for what is left, so that at most a round (plus fill and drain) is launched kernel by kernel.
-        bool started = false;
-        for (int pass = 0; pass < 2 && R > 0; ++pass) {
-            const long W = pass == 0 ? (long)R * K : (long)K;
-            if (pass == 1 && R == 1) break;
-            if ((started ? t : t_steady) + (pass == 0 ? 2 * W : W) > total) continue;
-            if (!started) {
-                if ((rc = enqueue_ticks(c, n_samples, G, 0, t_steady, total)) != MDI_OK) return rc;
-                t = t_steady;
-                started = true;
+    // From here on work is queued that advances positions and counters on the device; the host's copies follow only
+    // once all of it has run.  A failure half-way leaves the two out of step, so it forgets every sample.
+    auto enqueue_all = [&]() -> int {
+        int rc = MDI_OK;
+        long t = 0;
+        if (t_total && use_fz) {
+            if ((rc = fz_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
+            c->last_kernel = 2;
+        } else if (t_total && use_pk) {
+            if ((rc = pk_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
+            c->last_kernel = 1;
+        } else if (t_total) {
+            const int R = c->rounds_per_graph;
+            const long t_steady = K > 1 ? K : 0; // first tick, multiple of K, from which every partition is in steady state
+            // Steady-state windows are replayed from CUDA graphs: first windows of R rounds, then windows of one round
+            // for what is left, so that at most a round (plus fill and drain) is launched kernel by kernel.
+            bool started = false;
+            for (int pass = 0; pass < 2 && R > 0; ++pass) {
+                const long W = pass == 0 ? (long)R * K : (long)K;
+                if (pass == 1 && R == 1) break;
+                if ((started ? t : t_steady) + (pass == 0 ? 2 * W : W) > total) continue;
+                if (!started) {
+                    if ((rc = enqueue_ticks(c, n_samples, G, 0, t_steady, total)) != MDI_OK) return rc;
+                    t = t_steady;
+                    started = true;
+                }
+                auto key = std::make_pair(n_samples, (int)W);
+                GraphEntry &ge = c->graphs[key];
+                if (!ge.exec) {
+                    cudaGraph_t graph = nullptr;
+                    CU(cudaStreamBeginCapture(c->main, cudaStreamCaptureModeThreadLocal));
+                    c->capturing = true;
+                    c->cap_launches = c->cap_steps = 0;
+                    rc = enqueue_ticks(c, n_samples, G, t_steady, t_steady + W, 1L << 60);
+                    c->capturing = false;
+                    cudaError_t e = cudaStreamEndCapture(c->main, &graph);
+                    if (rc != MDI_OK) { if (graph) cudaGraphDestroy(graph); c->graphs.erase(key); return rc; }
+                    if (e != cudaSuccess) { c->graphs.erase(key); return fail(c, MDI_ERR_CUDA, "graph capture: %s", cudaGetErrorString(e)); }
+                    e = cudaGraphInstantiate(&ge.exec, graph, 0);
+                    cudaGraphDestroy(graph);
+                    if (e != cudaSuccess) { c->graphs.erase(key); return fail(c, MDI_ERR_CUDA, "graph instantiate: %s", cudaGetErrorString(e)); }
+                    ge.launches = c->cap_launches;
+                    ge.steps = c->cap_steps;
+                }
+                while (t + W <= total) {
+                    CU(cudaGraphLaunch(ge.exec, c->main));
+                    c->st.kernel_launches += ge.launches;
+                    c->st.stage_steps += ge.steps;
+                    t += W;
+                }
             }
-            auto key = std::make_pair(n_samples, (int)W);
-            GraphEntry &ge = c->graphs[key];
-            if (!ge.exec) {
-                cudaGraph_t graph = nullptr;
-                CU(cudaStreamBeginCapture(c->main, cudaStreamCaptureModeThreadLocal));
-                c->capturing = true;
-                c->cap_launches = c->cap_steps = 0;
-                rc = enqueue_ticks(c, n_samples, G, t_steady, t_steady + W, 1L << 60);
-                c->capturing = false;
-                cudaError_t e = cudaStreamEndCapture(c->main, &graph);
-                if (rc != MDI_OK) { if (graph) cudaGraphDestroy(graph); c->graphs.erase(key); return rc; }
-                if (e != cudaSuccess) { c->graphs.erase(key); return fail(c, MDI_ERR_CUDA, "graph capture: %s", cudaGetErrorString(e)); }
-                e = cudaGraphInstantiate(&ge.exec, graph, 0);
-                cudaGraphDestroy(graph);
-                if (e != cudaSuccess) { c->graphs.erase(key); return fail(c, MDI_ERR_CUDA, "graph instantiate: %s", cudaGetErrorString(e)); }
-                ge.launches = c->cap_launches;
-                ge.steps = c->cap_steps;
-            }
-            while (t + W <= total) {
-                CU(cudaGraphLaunch(ge.exec, c->main));
-                c->st.kernel_launches += ge.launches;
-                c->st.stage_steps += ge.steps;
-                t += W;
-            }
+            if ((rc = enqueue_ticks(c, n_samples, G, t, t_total, total)) != MDI_OK) return rc;
         }
-        if ((rc = enqueue_ticks(c, n_samples, G, t, t_total, total)) != MDI_OK) return rc;
-    }
-    CU(cudaEventRecord(c->ev_t1, c->main));
-    CU(cudaGetLastError());
-    // tokens: entries [returned, returned + n_new) of each sample's log
-    for (int smp = 0; smp < n_samples; ++smp) {
-        if (n_new)
+        CU(cudaEventRecord(c->ev_t1, c->main));
+        CU(cudaGetLastError());
+        // tokens: entries [returned, returned + n_new) of each sample's log
+        for (int smp = 0; smp < n_samples && n_new; ++smp)
             CU(cudaMemcpyAsync(out + (size_t)smp * n_new, c->tok_log + (size_t)smp * c->s.n_ctx + c->returned_host[smp], (size_t)n_new * 4,
                                on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, c->main));
-        for (int p = 0; p < K; ++p) c->part[p].pos_host[smp] += n_pass;
-        c->gen_host[smp] += n_pass;
-        c->returned_host[smp] += n_new;
-        c->st.tokens_generated += n_pass;
+        CU(cudaStreamSynchronize(c->main));
+        return MDI_OK;
+    };
+    auto forget_all = [&]() {
+        cudaDeviceSynchronize();
+        cudaGetLastError();
+        for (int smp = 0; smp < c->S; ++smp) mdi_reset_sample(c, smp);
+    };
+    if ((rc = enqueue_all()) != MDI_OK) {
+        const std::string why = c->err;
+        forget_all();
+        return fail(c, rc, "%s; all samples were reset", why.c_str());
     }
-    CU(cudaStreamSynchronize(c->main));
     if (t_total && (use_pk || use_fz)) {
         int kerr = 0;
         CU(cudaMemcpy(&kerr, use_fz ? c->fz_err : c->pk_err, sizeof(int), cudaMemcpyDeviceToHost));
         if (kerr) {
-            // the pipeline stopped half-way: positions, caches and counters no longer agree, so every sample is
-            // forgotten (like mdi_reset_sample); the context itself stays usable
-            for (int smp = 0; smp < c->S; ++smp) mdi_reset_sample(c, smp);
+            // the pipeline stopped half-way: positions, caches and counters no longer agree
+            forget_all();
             return fail(c, MDI_ERR_TIMEOUT, "persistent decode kernel gave up waiting (code %d: 1 edge flag, 2 team barrier, 3 weight tile, 4 ring slot); all samples were reset", kerr);
         }
+    }
+    for (int smp = 0; smp < n_samples; ++smp) {
+        for (int p = 0; p < K; ++p) c->part[p].pos_host[smp] += n_pass;
+        c->gen_host[smp] += n_pass;
+        c->returned_host[smp] += n_new;
+        c->st.tokens_generated += n_pass;
     }
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, c->ev_t0, c->ev_t1) == cudaSuccess) c->st.last_generate_ms = ms;
@@ -1856,6 +1846,9 @@ int mdi_set_sampling(mdi_ctx *c, float temperature, int top_k, uint64_t seed) {
     if (!(temperature == temperature)) return fail(c, MDI_ERR_ARG, "temperature is not a number");
     CU(cudaSetDevice(c->dev));
     CU(cudaDeviceSynchronize());
+    // the captured windows of the stream scheduler carry the token-choice parameters in their kernel arguments
+    for (auto &g : c->graphs) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
+    c->graphs.clear();
     c->temperature = temperature > 0.f ? temperature : 0.f;
     c->top_k = top_k;
     c->sample_seed = seed;
@@ -1904,7 +1897,7 @@ int mdi_get_partition_times(mdi_ctx *c, int p, double *out_ms, int n) {
     if (p < 0 || p >= c->K || n < 1) return fail(c, MDI_ERR_ARG, "partition out of range");
     const bool fz = c->last_kernel == 2;
     if (fz ? !(c->fz_ok && c->fz_prof_on) : !(c->pk_ok && c->pk_prof_on))
-        return fail(c, MDI_ERR_STATE, "in-kernel timing is off (set MDI_PK_PROFILE=1 before mdi_create; persistent schedulers only)");
+        return fail(c, MDI_ERR_STATE, "in-kernel timing is off (options.in_kernel_timing at mdi_create; persistent schedulers only)");
     CU(cudaSetDevice(c->dev));
     CU(cudaDeviceSynchronize());
     const int first_cta = fz ? c->fz_teams_host[p].first_cta : c->pk_teams_host[p].first_cta;
@@ -1917,6 +1910,17 @@ int mdi_get_partition_times(mdi_ctx *c, int p, double *out_ms, int n) {
         out_ms[i] = acc / n_cta * 1e-6;
     }
     return n_cta;
+}
+
+int mdi_get_trace(mdi_ctx *c, uint64_t *out_host, int n_words) {
+    if (!c || !out_host || n_words < 1) return fail(c, MDI_ERR_ARG, "null argument");
+    static_assert(FZ_TRACE_N == MDI_TRACE_WORDS, "trace record size");
+    if (!c->fz_trace || c->last_kernel != 2) return fail(c, MDI_ERR_STATE, "no trace was taken (in_kernel_timing and trace_slot at mdi_create; fused-phase kernel only)");
+    CU(cudaSetDevice(c->dev));
+    CU(cudaDeviceSynchronize());
+    const size_t n = std::min<size_t>((size_t)n_words, (size_t)c->fz_trace_blocks * FZ_TRACE_N);
+    CU(cudaMemcpy(out_host, c->fz_trace, n * 8, cudaMemcpyDeviceToHost));
+    return c->fz_trace_blocks;
 }
 
 int64_t mdi_memory_bytes(mdi_ctx *c, int p) {

@@ -16,13 +16,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmdi.so")
 
 MDI_OK = 0
+TRACE_WORDS = 128
 ERR_ARG, ERR_SHAPE, ERR_OOM, ERR_CONTEXT, ERR_STATE, ERR_TIMEOUT, ERR_CUDA = -1, -2, -3, -4, -5, -6, -7
 _ERR_NAMES = {ERR_ARG: "MDI_ERR_ARG", ERR_SHAPE: "MDI_ERR_SHAPE", ERR_OOM: "MDI_ERR_OOM", ERR_CONTEXT: "MDI_ERR_CONTEXT",
               ERR_STATE: "MDI_ERR_STATE", ERR_TIMEOUT: "MDI_ERR_TIMEOUT", ERR_CUDA: "MDI_ERR_CUDA"}
 
 EXPORTS = ["mdi_create", "mdi_destroy", "mdi_load_weights", "mdi_prefill", "mdi_prefill_dev", "mdi_step",
            "mdi_generate", "mdi_generate_dev", "mdi_get_logits", "mdi_set_sampling", "mdi_set_teacher_tokens", "mdi_reset_sample",
-           "mdi_get_stats", "mdi_get_partition_times", "mdi_memory_bytes", "mdi_sync", "mdi_last_error", "mdi_greedy_argmax_static"]
+           "mdi_get_stats", "mdi_get_partition_times", "mdi_get_trace", "mdi_memory_bytes", "mdi_sync", "mdi_last_error", "mdi_greedy_argmax_static"]
 
 
 class MdiError(RuntimeError):
@@ -41,7 +42,8 @@ class ModelShape(ctypes.Structure):
 class Options(ctypes.Structure):
     _fields_ = [("page_tokens", ctypes.c_int), ("kv_pool_tokens", ctypes.c_int), ("attn_splits", ctypes.c_int),
                 ("rounds_per_graph", ctypes.c_int), ("kv_cache_bf16", ctypes.c_int), ("prefill_mode", ctypes.c_int), ("tc_min_group", ctypes.c_int), ("wait_limit_ms", ctypes.c_int), ("debug_withhold_handoff", ctypes.c_int),
-                ("scheduler", ctypes.c_int)]
+                ("scheduler", ctypes.c_int), ("in_kernel_timing", ctypes.c_int), ("fused_blocks_per_head", ctypes.c_int),
+                ("debug_refuse_cluster_launch", ctypes.c_int), ("trace_slot", ctypes.c_int)]
 
 
 class Stats(ctypes.Structure):
@@ -80,6 +82,7 @@ def lib():
         L.mdi_reset_sample.argtypes = [vp, ci]
         L.mdi_get_stats.argtypes = [vp, ctypes.POINTER(Stats)]
         L.mdi_get_partition_times.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_double), ci]
+        L.mdi_get_trace.argtypes = [vp, vp, ci]
         L.mdi_memory_bytes.argtypes = [vp, ci]
         L.mdi_memory_bytes.restype = ctypes.c_int64
         L.mdi_sync.argtypes = [vp]
@@ -115,7 +118,8 @@ class Context:
     def __init__(self, shape, part_bounds: Sequence[int], n_samples: int, page_tokens: int = 0,
                  kv_pool_tokens: int = 0, attn_splits: int = 0, rounds_per_graph: int = 0, scheduler: int = 0,
                  kv_cache_bf16: int = 0, prefill_mode: int = 0, tc_min_group: int = 0,
-                 wait_limit_ms: int = 0, debug_withhold_handoff: int = 0):
+                 wait_limit_ms: int = 0, debug_withhold_handoff: int = 0, in_kernel_timing: int = 0,
+                 fused_blocks_per_head: int = 0, debug_refuse_cluster_launch: int = 0, trace_slot: int = 0):
         self._h = None
         self.shape = shape
         self.K = len(part_bounds) - 1
@@ -123,7 +127,8 @@ class Context:
         cs = ModelShape(**{n: getattr(shape, n) for n, _ in ModelShape._fields_})
         bounds = (ctypes.c_int * len(part_bounds))(*part_bounds)
         opts = Options(page_tokens, kv_pool_tokens, attn_splits, rounds_per_graph, kv_cache_bf16, prefill_mode, tc_min_group,
-                       wait_limit_ms, debug_withhold_handoff, scheduler)
+                       wait_limit_ms, debug_withhold_handoff, scheduler, in_kernel_timing, fused_blocks_per_head,
+                       debug_refuse_cluster_launch, trace_slot)
         h = ctypes.c_void_p()
         rc = lib().mdi_create(ctypes.byref(cs), bounds, self.K, n_samples, ctypes.byref(opts), ctypes.byref(h))
         if rc != MDI_OK:
@@ -202,6 +207,14 @@ class Context:
         if rc < 0:
             self._check(rc)
         return rc, list(out)
+
+    def trace(self) -> np.ndarray:
+        """[blocks][TRACE_WORDS] uint64 time stamps of the traced schedule slot ((ns << 4) | category, 0 = unused)."""
+        buf = np.zeros(1024 * TRACE_WORDS, np.uint64)
+        rc = lib().mdi_get_trace(self._h, buf.ctypes.data, buf.size)
+        if rc < 0:
+            self._check(rc)
+        return buf[: rc * TRACE_WORDS].reshape(rc, TRACE_WORDS)
 
     def memory_bytes(self, partition: int) -> int:
         return lib().mdi_memory_bytes(self._h, partition)

@@ -53,3 +53,37 @@ def test_sampled_tokens_reproduce_from_the_logits(arch, dtype, V, top_k, tempera
         ctx.set_sampling(1.0, 65, 1)
     assert e.value.code == mdi.ERR_ARG
     ctx.close()
+
+
+def test_sampling_parameters_reach_replayed_graph_windows():
+    """The stream scheduler replays captured windows of the schedule; the token-choice parameters travel in kernel
+    arguments, so a change of them must not be answered from a window captured before it.  Sample with seed A over
+    several windows, then switch to seed B, then to greedy, and check every token against the oracle's sampler
+    (or the argmax) applied to the library's own logits."""
+    from paper_2505_18164_b200 import mdi
+    shape = tiny_shape("gpt", I.DT_F32, L=2, d=64, H=4, V=97, C=64)
+    _, w = make_oracle(shape, seed=13, std=0.08)
+    S, P, n = 3, 4, 6
+    prompts = I.make_prompts(97, S, P, seed=9)
+    ctx = mdi.Context(shape, [0, 1, 2], S, scheduler=1, rounds_per_graph=2)
+    ctx.load_all(w)
+    launches_before = None
+    for temperature, top_k, seed in ((1.3, 20, 111), (1.3, 20, 222), (0.0, 0, 0), (0.9, 7, 222)):
+        ctx.set_sampling(temperature, top_k, seed)
+        for s in range(S):
+            ctx.reset_sample(s)
+            ctx.prefill(s, prompts[s])
+        # one call over several windows, then token by token so that every step's logits can be read back
+        block = ctx.generate(S, n).copy()
+        for s in range(S):
+            ctx.reset_sample(s)
+            ctx.set_teacher_tokens(s, block[s])
+            ctx.prefill(s, prompts[s])
+        for i in range(n):
+            out = ctx.generate(S, 1)
+            for s in range(S):
+                lg = ctx.get_logits(s)
+                want = (O.sample_top_k(lg, top_k, temperature, O.sample_uniform(seed, s, i)) if temperature > 0
+                        else int(np.argmax(lg)))
+                assert out[s, 0] == want == block[s, i], (temperature, seed, s, i)
+    ctx.close()
