@@ -9,6 +9,16 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def pytest_addoption(parser):
+    parser.addoption("--full-lengths", action="store_true", default=False,
+                     help="run the largest workload's oracle comparison over its whole generation length")
+
+
+@pytest.fixture
+def full_lengths(request):
+    return request.config.getoption("--full-lengths")
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run on a B200)")
     # native pieces that need no GPU to build: input generator, CPU checker, CUDA library (cross-compiled)

@@ -1,9 +1,9 @@
 """The five named workloads against the CPU oracle, through the C ABI.
 
-gpt2_small runs at its full size (3 samples, 64-token prompts, 512 new tokens) in the launch
-configuration bench.py times; the larger shapes keep their full model shape, partitioning and number of
-samples in flight but shorter prompts and generations, and the oracle follows a stated subset of the
-samples (first and last slot), so that the CPU side finishes in seconds to a few minutes.
+Every workload runs at its full model shape, partitioning, number of samples in flight and prompt length, in the
+launch configuration bench.py times; the generation length is the workload's own (the Llama-7B shape: 256 of its
+512 new tokens unless pytest is given --full-lengths).  For the three large shapes the oracle follows a stated
+subset of the samples (first and last slot), so that the CPU side finishes in a few minutes.
 
 Protocol as in test_gpu_parity.py: checked samples are teacher-forced with the oracle's tokens; every
 token must equal the oracle's where its top-1/top-2 margin exceeds twice the logit tolerance; logits are
@@ -72,16 +72,24 @@ def test_gpt2_small_stream_scheduler_short():
     _run("gpt2_small", n_new=40, chunk=20, scheduler=1)
 
 
-def test_gpt2_medium_shape():
-    _run("gpt2_medium", n_prompt=32, n_new=24, check=[0, 7])
+def test_gpt2_medium_full_size():
+    """Full prompts and generation length (128 + 768): caches grow over seven 128-row pages with two samples per
+    group; first and last slot follow the oracle."""
+    _run("gpt2_medium", check=[0, 7], chunk=64)
 
 
-def test_gpt2_xl_shape_uneven_groups():
-    _run("gpt2_xl", n_prompt=16, n_new=12, check=[0, 15], chunk=6)
+def test_gpt2_xl_full_size_ends_at_the_context_limit():
+    """256-token prompts + 768 new tokens = n_ctx: the last token is produced from position 1022 and never fed, so
+    1023 rows are cached; groups of 3,3,3,3,2,2 samples; every attention split holds rows."""
+    w = I.ALL_WORKLOADS["gpt2_xl"]
+    assert w.n_prompt + w.n_new == w.shape.n_ctx
+    _run("gpt2_xl", check=[0, 15], chunk=64)
 
 
-def test_llama_7b_shape_groups_of_eight():
-    _run("llama_7b", n_prompt=8, n_new=6, check=[0, 63], chunk=3)
+def test_llama_7b_long(full_lengths):
+    """Full 128-token prompts, groups of eight on the tensor cores, slots 0 and 63 against the oracle; 256 new tokens
+    by default, all 512 with --full-lengths."""
+    _run("llama_7b", n_new=None if full_lengths else 256, check=[0, 63], chunk=32)
 
 
 @pytest.mark.parametrize("name", ["nanollama_3nodes", "nanollama_2nodes", "tinyllama_3nodes"])

@@ -118,3 +118,29 @@ def test_reference_arm_prints_its_json_line():
     d = json.loads([ln for ln in out.stdout.splitlines() if ln.startswith("{")][-1])
     assert d["impl"] == "reference" and d["unit"] == "tokens/s" and d["value"] > 0
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_bench_byte_counts_and_cpu_sample_plans():
+    """Bytes a round of the schedule must move (every group streams the model once, every sample reads its cache at
+    the weights' width), against figures worked out by hand from the shapes: 12 d^2 + 13 d parameters per GPT block,
+    4 d^2 + 3 d F + 2 d per Llama block, V d + norm vectors for the output layers, cache rows of 2 d elements."""
+    import bench
+    for name, kv_bpe, gb in (("tiny_gpt_fp32", 4, 0.1308), ("gpt2_small", 2, 0.7774), ("gpt2_medium", 2, 3.234), ("llama_7b", 2, 118.64)):
+        w = I.WORKLOADS[name]
+        s = w.shape
+        bpe = 4 if s.weight_dtype == I.DT_F32 else 2
+        block = (12 * s.d_model ** 2 + 13 * s.d_model) if s.arch == I.ARCH_GPT else (4 * s.d_model ** 2 + 3 * s.d_model * s.d_ff + 2 * s.d_model)
+        head = s.vocab * s.d_model + (2 if s.arch == I.ARCH_GPT else 1) * s.d_model
+        G = min(w.n_samples, w.n_partitions)
+        n_pass = w.n_new - 1
+        mean_rows = w.n_prompt + (n_pass - 1) / 2 + 1                      # rows read per pass, averaged, plus the one written
+        want = G * (s.n_layer * block + head) * bpe + w.n_samples * s.n_layer * 2 * s.d_model * (mean_rows + 1) * kv_bpe
+        got = bench.decode_bytes(w, w.n_samples, kv_bpe)
+        assert got["passes"] == n_pass and abs(got["total"] / n_pass - want) < 1e-6 * want
+        assert abs(got["total"] / n_pass / 1e9 - gb) < 2e-3 * gb
+    assert bench.oracle_sample_plan(I.WORKLOADS["tiny_gpt_fp32"], 16) == ("full",)
+    kind, p_s, n_s = bench.oracle_sample_plan(I.WORKLOADS["llama_7b"], 16)
+    assert kind == "slot0" and 8 <= p_s <= 128 and 8 <= n_s <= 511
+    for name in I.WORKLOAD_ORDER:                                         # the two arms describe the workload alike
+        w = I.WORKLOADS[name]
+        assert bench.workload_config(w, 1)["workload"] == name and bench.workload_config(w, 1) == bench.workload_config(w, 1)
