@@ -248,7 +248,7 @@ def run_workload(w: I.Workload, args, steps: int, warmup: int, e2e_steps: int, w
     s = w.shape
     S, P, N = w.n_samples, w.n_prompt, w.n_new
     ctx = mdi.Context(s, list(w.part_bounds), S, kv_pool_tokens=S * ((P + N + 15) // 16 * 16), rounds_per_graph=args.rounds_per_graph,
-                      scheduler=args.scheduler, tc_min_group=args.tc_min_group, kv_cache_bf16=args.kv_cache_bf16)
+                      scheduler=args.scheduler, tc_min_group=args.tc_min_group, kv_cache_dtype=args.kv_cache_dtype)
     weights = {}
     for name, a in I.iter_weights(s, w.weight_seed):
         ctx.load_weights(name, a)
@@ -310,7 +310,7 @@ def run_workload(w: I.Workload, args, steps: int, warmup: int, e2e_steps: int, w
         e2e_s = [step_host() for _ in range(e2e_steps)]
         barrier()
         assert np.array_equal(out_np, tokens_dev), "host and device entry points disagree"
-    kv_stored_bpe = 2 if (args.kv_cache_bf16 and s.weight_dtype == I.DT_BF16) else 4
+    kv_stored_bpe = int(st1.kv_element_bytes)
     res = {"run_ms": run_ms, "gen_ms": gen_ms, "pf_ms": pf_ms, "e2e_s": e2e_s, "clocks": clocks,
            "launches": int(st1.kernel_launches - st0.kernel_launches), "kv_stored_bpe": kv_stored_bpe}
     ctx.close()
@@ -355,7 +355,7 @@ def main():
     ap.add_argument("--rounds-per-graph", type=int, default=0)
     ap.add_argument("--scheduler", type=int, default=0, help="0 auto (a persistent kernel when the shape fits), 1 streams, 2 phase-per-matrix persistent kernel, 3 fused-phase persistent kernel")
     ap.add_argument("--tc-min-group", type=int, default=0, help="smallest group whose decode steps run on the tensor cores (0 = library default)")
-    ap.add_argument("--kv-cache-bf16", type=int, default=0)
+    ap.add_argument("--kv-cache-dtype", type=int, default=0, help="0 library default, 1 bf16, 2 fp16, 3 fp32")
     ap.add_argument("--n-new", type=int, default=0, help="shorter generation (profiler captures only; not the headline)")
     ap.add_argument("--n-prompt", type=int, default=0, help="shorter prompts (profiler captures only)")
     ap.add_argument("--n-layer", type=int, default=0, help="fewer blocks, one partition (profiler captures only)")

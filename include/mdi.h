@@ -44,6 +44,7 @@ enum {
 enum { MDI_ARCH_GPT = 0, MDI_ARCH_LLAMA = 1 };
 enum { MDI_DTYPE_F32 = 0, MDI_DTYPE_BF16 = 1 };
 enum { MDI_ACT_GELU_TANH = 0, MDI_ACT_GELU_ERF = 1, MDI_ACT_SWIGLU = 2 };
+enum { MDI_KV_DEFAULT = 0, MDI_KV_BF16 = 1, MDI_KV_F16 = 2, MDI_KV_F32 = 3 };
 
 typedef struct mdi_ctx mdi_ctx;
 
@@ -70,9 +71,11 @@ typedef struct {
     int attn_splits;   /* sequence splits of decode attention (default: chosen from n_ctx) */
     int rounds_per_graph; /* stream scheduler: rounds of the recurrent schedule captured per CUDA graph
                              (default 16; <0: no graphs) */
-    int kv_cache_bf16; /* 0 (default): the key/value cache holds fp32; 1: with bf16 weights, hold bf16 instead - half the
-                          cache bytes, at about 2e-3 relative error per block on the activations (measured), which on a
-                          32-block model exceeds a 3e-2 absolute logit tolerance */
+    int kv_cache_dtype; /* MDI_KV_*: element type of the key/value cache when the weights are bf16 (fp32 weights always
+                          keep an fp32 cache).  DEFAULT = F32.  BF16 halves the cache bytes at about 2e-3 relative error
+                          per block on the activations (measured), which on a 32-block model exceeds a 3e-2 absolute
+                          logit tolerance; F16 halves them at an eighth of that error (three more mantissa bits; keys and
+                          values of these models are far inside its range) */
     int prefill_mode;  /* first visits (whole prompt): 0 (default) tensor-core GEMMs (tcgen05, bf16 x bf16 -> fp32, inputs split
                           into two bf16 planes) when the weights are bf16, else the CUDA-core step kernels in chunks of 8
                           positions; 1: always the CUDA-core kernels */
@@ -95,7 +98,11 @@ typedef struct {
                              (groups of at most 4 samples, any block type) comes next;
                           1: always the stream scheduler (one stream per partition, event handoff);
                           2: the phase-per-matrix persistent kernel, or fail;
-                          3: the fused-phase persistent kernel, or fail */
+                          3: the fused-phase persistent kernel, or fail;
+                          4: the tensor-core persistent kernel, or fail (bf16 weights, groups of at most 8 samples, widths
+                             that are multiples of 64: one cooperative launch, a team per partition, every linear layer a
+                             tcgen05 contraction fed by a TMA weight ring; what scheduler 0 picks where it would otherwise run
+                             tensor-core steps on the stream scheduler, greedy token choice only) */
     int in_kernel_timing; /* 1: the persistent kernels time themselves (mdi_get_partition_times); costs a few percent */
     int fused_blocks_per_head; /* fused-phase kernel: 0 (default) two thread blocks of a cluster share a head where every
                           team has a cluster per head, else one block per head; 1: always one block per head (plain
@@ -120,6 +127,7 @@ typedef struct {
                                    end of the last one (events on the partition streams) */
     float last_generate_ms;     /* device time of the last mdi_generate, first to last partition step */
     float last_run_ms;          /* device time from that first mdi_prefill to the end of the last mdi_generate */
+    int kv_element_bytes;       /* bytes per element of the key/value cache (4, or 2 for a bf16 / fp16 cache) */
 } mdi_stats;
 
 /* Set-up of the nodes (Section III-A: the starter assigns each node its chunk).

@@ -19,6 +19,7 @@
 #include "persistent_decode.cuh"
 #include "prefill_kernels.cuh"
 #include "step_kernels.cuh"
+#include "tc_decode.cuh"
 #include "tc_gemm.cuh"
 
 using namespace mdi;
@@ -85,6 +86,7 @@ struct mdi_ctx {
     int page_tokens = 16, page_shift = 4, pages_per_seq = 0, n_split = 1, gmax = 1, rounds_per_graph = 16;
     size_t page_elems = 0, esize = 2, kv_esize = 4;
     bool kv_f32 = true;
+    int kv_kind = 0; // KV_F32 / KV_BF16 / KV_F16
     std::vector<Partition> part;
     std::vector<LayerW> layer;
     void *wte = nullptr, *wpe = nullptr, *lm_head = nullptr;
@@ -156,6 +158,21 @@ struct mdi_ctx {
     bool fz_refusal_faked = false;
     int64_t fz_stream_bytes = 0;
     std::vector<int64_t> fz_team_stream_bytes; // per partition: bytes of its blocks' weight streams
+    // persistent tensor-core decode kernel (bf16 weights, groups of up to 8 samples): plan at creation, tables at first use
+    bool td_ok = false, td_stale = true;
+    int td_grid = 0;
+    size_t td_smem = 0;
+    std::vector<TdTeam> td_teams_host;
+    std::vector<TdPhase> td_phases_host;
+    std::vector<int> td_phase_begin, td_phase_count;
+    TdTeam *td_teams = nullptr;
+    TdPhase *td_phases = nullptr;
+    CUtensorMap *td_maps = nullptr;
+    float *td_buf = nullptr;       // all scratch of the kernel (residual copies, partial sums), one allocation
+    unsigned *td_sync = nullptr;
+    int *td_err = nullptr;
+    unsigned long long *td_prof = nullptr;
+    int64_t td_buf_bytes = 0;
     mdi_stats st{};
     std::string err;
 };
@@ -209,32 +226,43 @@ void launch_k(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t 
 // ---- kernel dispatch ------------------------------------------------------------------------------
 constexpr size_t LIN_SMEM_MAX = 200 * 1024;
 
-// The key/value cache is fp32 (kv_f32) unless the context asked for a cache in the (2-byte) weight type.
-template <int NB, typename WT, int MODE> void lin_launch(const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st, bool kv_f32) {
-    if (MODE == LIN_QKV && kv_f32) k_linear<NB, WT, MODE, float><<<grid, LIN_THREADS, smem, st>>>(a, bt);
+// Element type of the key/value cache: fp32 (always with fp32 weights), or with bf16 weights a 2-byte type on request.
+enum { KV_F32 = 0, KV_BF16 = 1, KV_F16 = 2 };
+// Runs `call` with KT bound to the cache's element type.
+#define KV_DISPATCH(kind, call)                                          \
+    do {                                                                 \
+        if ((kind) == KV_F32) { using KT = float; call; }                \
+        else if ((kind) == KV_F16) { using KT = __half; call; }          \
+        else { using KT = __nv_bfloat16; call; }                         \
+    } while (0)
+template <int NB, typename WT, int MODE> void lin_launch(const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st, int kv_kind) {
+    if (MODE == LIN_QKV && kv_kind == KV_F32) k_linear<NB, WT, MODE, float><<<grid, LIN_THREADS, smem, st>>>(a, bt);
+    else if (MODE == LIN_QKV && kv_kind == KV_F16) k_linear<NB, WT, MODE, __half><<<grid, LIN_THREADS, smem, st>>>(a, bt);
     else k_linear<NB, WT, MODE><<<grid, LIN_THREADS, smem, st>>>(a, bt);
 }
 template <int NB, typename WT, int MODE> cudaError_t lin_attr() {
     cudaError_t e = cudaFuncSetAttribute(k_linear<NB, WT, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LIN_SMEM_MAX);
     if (e == cudaSuccess && MODE == LIN_QKV)
         e = cudaFuncSetAttribute(k_linear<NB, WT, MODE, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LIN_SMEM_MAX);
+    if (e == cudaSuccess && MODE == LIN_QKV)
+        e = cudaFuncSetAttribute(k_linear<NB, WT, MODE, __half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LIN_SMEM_MAX);
     return e;
 }
-template <typename WT, int MODE> void lin_nb(int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st, bool kv_f32) {
+template <typename WT, int MODE> void lin_nb(int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st, int kv_kind) {
     switch (nb) {
-        case 1: lin_launch<1, WT, MODE>(a, bt, grid, smem, st, kv_f32); break;
-        case 2: lin_launch<2, WT, MODE>(a, bt, grid, smem, st, kv_f32); break;
-        case 4: lin_launch<4, WT, MODE>(a, bt, grid, smem, st, kv_f32); break;
-        default: lin_launch<8, WT, MODE>(a, bt, grid, smem, st, kv_f32); break;
+        case 1: lin_launch<1, WT, MODE>(a, bt, grid, smem, st, kv_kind); break;
+        case 2: lin_launch<2, WT, MODE>(a, bt, grid, smem, st, kv_kind); break;
+        case 4: lin_launch<4, WT, MODE>(a, bt, grid, smem, st, kv_kind); break;
+        default: lin_launch<8, WT, MODE>(a, bt, grid, smem, st, kv_kind); break;
     }
 }
-template <typename WT> void lin_mode(int mode, int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st, bool kv_f32) {
+template <typename WT> void lin_mode(int mode, int nb, const LinArgs &a, const Batch &bt, int grid, size_t smem, cudaStream_t st, int kv_kind) {
     switch (mode) {
-        case LIN_QKV: lin_nb<WT, LIN_QKV>(nb, a, bt, grid, smem, st, kv_f32); break;
-        case LIN_ACT: lin_nb<WT, LIN_ACT>(nb, a, bt, grid, smem, st, kv_f32); break;
-        case LIN_GATEUP: lin_nb<WT, LIN_GATEUP>(nb, a, bt, grid, smem, st, kv_f32); break;
-        case LIN_HEAD: lin_nb<WT, LIN_HEAD>(nb, a, bt, grid, smem, st, kv_f32); break;
-        default: lin_nb<WT, LIN_RESID>(nb, a, bt, grid, smem, st, kv_f32); break;
+        case LIN_QKV: lin_nb<WT, LIN_QKV>(nb, a, bt, grid, smem, st, kv_kind); break;
+        case LIN_ACT: lin_nb<WT, LIN_ACT>(nb, a, bt, grid, smem, st, kv_kind); break;
+        case LIN_GATEUP: lin_nb<WT, LIN_GATEUP>(nb, a, bt, grid, smem, st, kv_kind); break;
+        case LIN_HEAD: lin_nb<WT, LIN_HEAD>(nb, a, bt, grid, smem, st, kv_kind); break;
+        default: lin_nb<WT, LIN_RESID>(nb, a, bt, grid, smem, st, kv_kind); break;
     }
 }
 template <typename WT, int MODE> cudaError_t lin_attr_nb() {
@@ -282,8 +310,8 @@ int linear(mdi_ctx *c, int mode, LinArgs a, const Batch &bt, cudaStream_t st) {
         if (a.x_res) b.x_res = a.x_res + (size_t)first * a.n_rows;
         if (a.x_out) b.x_out = a.x_out + (size_t)first * a.n_rows;
         const size_t smem = (size_t)nb * a.in_dim * 4;
-        if (f32) lin_mode<float>(mode, nb, b, sb, grid, smem, st, c->kv_f32);
-        else lin_mode<__nv_bfloat16>(mode, nb, b, sb, grid, smem, st, c->kv_f32);
+        if (f32) lin_mode<float>(mode, nb, b, sb, grid, smem, st, KV_F32);
+        else lin_mode<__nv_bfloat16>(mode, nb, b, sb, grid, smem, st, c->kv_kind);
         count_launch(c);
     }
     return MDI_OK;
@@ -379,7 +407,7 @@ int enqueue_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in
             a.layer_local = l - P.lo; a.n_head = s.n_head; a.n_split = c->n_split; a.pos = P.pos_dev;
             a.scale = 1.0f / std::sqrt((float)s.head_dim);
             dim3 g(s.n_head, c->n_split, bt.n);
-            if (c->kv_f32) attn_hd<float>(false, s.head_dim, a, bt, g, st); else attn_hd<__nv_bfloat16>(false, s.head_dim, a, bt, g, st);
+            KV_DISPATCH(c->kv_kind, attn_hd<KT>(false, s.head_dim, a, bt, g, st));
             count_launch(c);
         }
         {   // output projection + residual
@@ -546,21 +574,18 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
         pend = PfPending();
         if ((rc = pf_gemm(c, P, L.wqkv, qw + 2 * kw, d, T, L.bqkv, nullptr, TG_NONE, P.pf_qkv, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
         if (bt) {
-            if (c->kv_f32) launch_k(pdl, k_bt_rope_append<float>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
-            else launch_k(pdl, k_bt_rope_append<__nv_bfloat16>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf);
+            KV_DISPATCH(c->kv_kind, launch_k(pdl, k_bt_rope_append<KT>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf));
             count_launch(c);
             AttnArgs a{};
             a.q = P.qbuf; a.o = P.obuf; a.part = P.part; a.ticket = P.attn_ticket; a.kv = kv; a.layer_local = ll; a.n_head = s.n_head;
             a.n_split = c->n_split; a.pos = P.pos_dev; a.scale = scale; a.o_hi = hi; a.o_lo = lo;
             const dim3 g(s.n_head, c->n_split, T);
-            if (c->kv_f32) attn_hd<float>(pdl, s.head_dim, a, *bt, g, st); else attn_hd<__nv_bfloat16>(pdl, s.head_dim, a, *bt, g, st);
+            KV_DISPATCH(c->kv_kind, attn_hd<KT>(pdl, s.head_dim, a, *bt, g, st));
             count_launch(c);
         } else {
-            if (c->kv_f32) launch_k(pdl, k_pf_rope_append<float>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
-            else launch_k(pdl, k_pf_rope_append<__nv_bfloat16>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q);
+            KV_DISPATCH(c->kv_kind, launch_k(pdl, k_pf_rope_append<KT>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, slot, P.pf_q));
             count_launch(c);
-            if (c->kv_f32) pf_attn_hd<float>(pdl, s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
-            else pf_attn_hd<__nv_bfloat16>(pdl, s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale);
+            KV_DISPATCH(c->kv_kind, pf_attn_hd<KT>(pdl, s.head_dim, dim3(s.n_head, T), st, P.pf_q, hi, lo, kv, ll, s.n_head, P.pos_dev, slot, scale));
             count_launch(c);
         }
         // output projection + residual -> x_out (or partial sums, completed by the next kernel)
@@ -662,7 +687,7 @@ template <typename WT, typename KT> const void *pk_func(int nb) {
 }
 const void *pk_func_for(const mdi_ctx *c, int nb) {
     if (c->s.weight_dtype == MDI_DTYPE_F32) return pk_func<float, float>(nb);
-    return c->kv_f32 ? pk_func<__nv_bfloat16, float>(nb) : pk_func<__nv_bfloat16, __nv_bfloat16>(nb);
+    return c->kv_kind == KV_F32 ? pk_func<__nv_bfloat16, float>(nb) : c->kv_kind == KV_F16 ? pk_func<__nv_bfloat16, __half>(nb) : pk_func<__nv_bfloat16, __nv_bfloat16>(nb);
 }
 
 // Phase list of every partition, team sizes (blocks per partition, in proportion to the bytes a step
@@ -674,7 +699,7 @@ int pk_setup(mdi_ctx *c) {
     cudaDeviceProp prop;
     CU(cudaGetDeviceProperties(&prop, c->dev));
     c->n_sm = prop.multiProcessorCount;
-    if (c->scheduler == 1 || c->scheduler == 3) return MDI_OK;
+    if (c->scheduler == 1 || c->scheduler == 3 || c->scheduler == 4) return MDI_OK;
     const bool want = c->scheduler == 2;
     if (c->gmax > PK_MAXNB) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: at most %d samples per group", PK_MAXNB) : MDI_OK;
     if (K > 32 || K > c->n_sm) return want ? fail(c, MDI_ERR_SHAPE, "persistent scheduler: too many partitions") : MDI_OK;
@@ -691,7 +716,8 @@ int pk_setup(mdi_ctx *c) {
     {
         cudaError_t ea;
         if (s.weight_dtype == MDI_DTYPE_F32) ea = pk_attr<float, float>(c->pk_smem);
-        else if (c->kv_f32) ea = pk_attr<__nv_bfloat16, float>(c->pk_smem);
+        else if (c->kv_kind == KV_F32) ea = pk_attr<__nv_bfloat16, float>(c->pk_smem);
+        else if (c->kv_kind == KV_F16) ea = pk_attr<__nv_bfloat16, __half>(c->pk_smem);
         else ea = pk_attr<__nv_bfloat16, __nv_bfloat16>(c->pk_smem);
         CU(ea);
     }
@@ -879,7 +905,7 @@ int fz_setup(mdi_ctx *c) {
     const int K = c->K, d = s.d_model, hd = s.head_dim, H = s.n_head;
     const bool want = c->scheduler == 3;
     auto no = [&](const char *why) { return want ? fail(c, MDI_ERR_SHAPE, "fused-phase scheduler: %s", why) : MDI_OK; };
-    if (c->scheduler == 1 || c->scheduler == 2) return MDI_OK;
+    if (c->scheduler == 1 || c->scheduler == 2 || c->scheduler == 4) return MDI_OK;
     if (s.arch != MDI_ARCH_GPT || s.weight_dtype != MDI_DTYPE_BF16 || !c->kv_f32) return no("needs the GPT block, bf16 weights and an fp32 cache");
     if (s.n_kv_head != H || H * hd != d) return no("needs n_kv_head = n_head and n_head * head_dim = d_model");
     if (d % 16 || s.d_ff % 16 || hd % 16) return no("widths must be multiples of 16");
@@ -1263,6 +1289,290 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     return MDI_OK;
 }
 
+
+// ---- persistent tensor-core decode kernel: plan, tables and launch ----------------------------------------
+template <typename KT> cudaError_t td_attr(size_t smem) {
+    return cudaFuncSetAttribute(k_tc_decode<KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+}
+const void *td_func(const mdi_ctx *c) {
+    return c->kv_kind == KV_F32 ? (const void *)k_tc_decode<float> : c->kv_kind == KV_F16 ? (const void *)k_tc_decode<__half> : (const void *)k_tc_decode<__nv_bfloat16>;
+}
+
+// How many ranges of k-blocks a contraction with `tiles` row tiles (all its matrices together) and n_kb k-blocks is
+// cut into for a team of n_cta blocks: at least so many that a range fits the resident B operand, then the first
+// count at which the units deal out evenly (a phase ends in a team barrier, so the block with most units sets its time).
+void td_choose_split(int tiles, int n_kb, int n_cta, int *n_split, int *kb_per_split) {
+    int best_s = 0, best_k = 0;
+    double best = -1.0;
+    for (int s0 = (n_kb + TD_B_KB - 1) / TD_B_KB; s0 <= std::min(n_kb, 16); ++s0) {
+        const int kbps = (n_kb + s0 - 1) / s0, s = (n_kb + kbps - 1) / kbps;
+        if (kbps < 2 && s0 > (n_kb + TD_B_KB - 1) / TD_B_KB) break;
+        const long units = (long)s * tiles;
+        const long most = (units + n_cta - 1) / n_cta;
+        // work of the busiest block against the mean, counting that every unit is charged a full range
+        const double eff = (double)tiles * n_kb / ((double)most * kbps * n_cta);
+        if (eff > best + 0.02) { best = eff; best_s = s; best_k = kbps; }
+        if (eff >= 0.93) break;
+    }
+    *n_split = best_s;
+    *kb_per_split = best_k;
+}
+
+int td_setup(mdi_ctx *c) {
+    const mdi_model_shape &s = c->s;
+    const int K = c->K, d = s.d_model, hd = s.head_dim, H = s.n_head, qw = H * hd, kw = s.n_kv_head * hd, F = s.d_ff, V = s.vocab;
+    const bool want = c->scheduler == 4;
+    auto no = [&](const char *why) { return want ? fail(c, MDI_ERR_SHAPE, "tensor-core persistent scheduler: %s", why) : MDI_OK; };
+    if (c->scheduler != 0 && c->scheduler != 4) return MDI_OK;
+    if (s.weight_dtype != MDI_DTYPE_BF16) return no("needs bf16 weights");
+    if (c->gmax > TD_MAXB) return no("at most 8 samples per group");
+    if (d % 64 || qw % 64 || F % 64) return no("d_model, n_head * head_dim and d_ff must be multiples of 64");
+    if (hd != 32 && hd != 64 && hd != 128) return no("head_dim must be 32, 64 or 128");
+    if (K > 32) return no("too many partitions");
+    if (!tg_encoder()) return no("no tensor-map encoder (driver too old)");
+    cudaDeviceProp prop;
+    CU(cudaGetDeviceProperties(&prop, c->dev));
+    const int n_sm = prop.multiProcessorCount;
+    if (n_sm < K) return no("fewer SMs than partitions");
+    c->td_smem = td_smem_layout().total;
+    if (c->td_smem > (size_t)prop.sharedMemPerBlockOptin) return no("not enough shared memory per block");
+    {
+        cudaError_t ea = c->kv_kind == KV_F32 ? td_attr<float>(c->td_smem) : c->kv_kind == KV_F16 ? td_attr<__half>(c->td_smem) : td_attr<__nv_bfloat16>(c->td_smem);
+        CU(ea);
+    }
+    for (int p = 0; p < K; ++p)
+        if (5 * (c->part[p].hi - c->part[p].lo) + 2 > TD_MAX_PHASES) return no("too many blocks of the model in one partition");
+    // team sizes in proportion to the bytes a partition step streams
+    const double layer_bytes = 2.0 * ((double)(qw + 2 * kw) * d + (double)d * qw + (double)(s.act == MDI_ACT_SWIGLU ? 3 : 2) * F * d);
+    std::vector<double> bytes(K);
+    double tot = 0;
+    for (int p = 0; p < K; ++p) {
+        bytes[p] = layer_bytes * (c->part[p].hi - c->part[p].lo) + (p == K - 1 ? 2.0 * V * d : 0.0);
+        tot += bytes[p];
+    }
+    std::vector<int> n_cta(K);
+    int used = 0, big = 0;
+    for (int p = 0; p < K; ++p) if (bytes[p] > bytes[big]) big = p;
+    for (int p = 0; p < K; ++p) {
+        if (p == big) continue;
+        n_cta[p] = std::max(1, (int)std::floor(n_sm * bytes[p] / tot));
+        used += n_cta[p];
+    }
+    if (n_sm - used < 1) return no("not enough SMs");
+    n_cta[big] = n_sm - used;
+    // phases (addresses follow in td_build)
+    c->td_phases_host.clear();
+    c->td_teams_host.assign(K, TdTeam{});
+    c->td_phase_begin.assign(K, 0);
+    c->td_phase_count.assign(K, 0);
+    int first = 0;
+    for (int p = 0; p < K; ++p) {
+        const int n = n_cta[p], Lp = c->part[p].hi - c->part[p].lo;
+        c->td_phase_begin[p] = (int)c->td_phases_host.size();
+        auto gemm = [&](int kind, int ll, int n_mat, int rows, int Kd, int pro) {
+            TdPhase q{};
+            q.kind = kind; q.layer_local = ll; q.n_mat = n_mat; q.n_rows = rows; q.K = Kd; q.pro = pro;
+            q.n_tiles = (rows + TG_BM - 1) / TG_BM; q.n_kb = Kd / TG_BK;
+            td_choose_split(n_mat * q.n_tiles, q.n_kb, n, &q.n_split, &q.kb_per_split);
+            q.n_units = q.n_split * n_mat * q.n_tiles;
+            c->td_phases_host.push_back(q);
+        };
+        for (int l = 0; l < Lp; ++l) {
+            gemm(TD_QKV, l, 1, qw + 2 * kw, d, TDP_NORM);
+            c->td_phases_host.back().first_of_step = l == 0;
+            TdPhase a{}; a.kind = TD_ATTN; a.layer_local = l; c->td_phases_host.push_back(a);
+            gemm(TD_OUT, l, 1, d, qw, TDP_MERGE);
+            gemm(TD_UP, l, s.act == MDI_ACT_SWIGLU ? 2 : 1, F, d, TDP_NORM);
+            gemm(TD_DOWN, l, 1, d, F, TDP_ACT);
+        }
+        if (p == K - 1) gemm(TD_HEAD, Lp, 1, V, d, TDP_NORM);
+        else { TdPhase f{}; f.kind = TD_FIN; f.layer_local = Lp; c->td_phases_host.push_back(f); }
+        c->td_phase_count[p] = (int)c->td_phases_host.size() - c->td_phase_begin[p];
+        TdTeam &T = c->td_teams_host[p];
+        T.first_cta = first; T.n_cta = n; first += n;
+        T.phase_begin = c->td_phase_begin[p]; T.n_phases = c->td_phase_count[p];
+        T.is_first = p == 0; T.is_last = p == K - 1;
+        // attention units (sample, head, split) over the team's warps: the split count that deals them out most evenly
+        {
+            const int warps = n * TD_CWARPS, pairs = c->gmax * H;
+            int best_s = 1;
+            double best = -1.0;
+            for (int sp = 1; sp <= TD_MAX_SPLITS; sp *= 2) {
+                const long units = (long)pairs * sp, most = (units + warps - 1) / warps;
+                const double eff = (double)units / ((double)most * warps);
+                if (eff > best + 0.03) { best = eff; best_s = sp; }
+            }
+            T.n_att_split = best_s;
+        }
+    }
+    c->td_grid = first;
+    int rc;
+    if ((rc = dalloc(c, &c->td_sync, (size_t)K * 64)) != MDI_OK) return rc;
+    if ((rc = dalloc(c, &c->td_err, 1)) != MDI_OK) return rc;
+    if (c->o.in_kernel_timing && (rc = dalloc(c, &c->td_prof, (size_t)c->td_grid * PK_PROF_N)) != MDI_OK) return rc;
+    c->td_ok = true;
+    return MDI_OK;
+}
+
+// Scratch, tensor maps and phase tables; runs before the first launch and again after weights were replaced.
+int td_build(mdi_ctx *c) {
+    if (!c->td_stale) return MDI_OK;
+    const mdi_model_shape &s = c->s;
+    const int K = c->K, d = s.d_model, hd = s.head_dim, H = s.n_head, qw = H * hd, kw = s.n_kv_head * hd, F = s.d_ff, V = s.vocab;
+    void *old[] = {c->td_teams, c->td_phases, c->td_maps, c->td_buf};
+    for (void *q : old) if (q) cudaFree(q);
+    c->td_teams = nullptr; c->td_phases = nullptr; c->td_maps = nullptr; c->td_buf = nullptr;
+    // one allocation for all scratch: first count, then carve
+    std::vector<CUtensorMap> maps;
+    size_t floats = 0;
+    auto take = [&](size_t n) { const size_t r = floats; floats += (n + 3) & ~(size_t)3; return r; };
+    struct Off { size_t x0, x1, att; std::vector<size_t> out; };
+    std::vector<Off> offs(K);
+    for (int p = 0; p < K; ++p) {
+        offs[p].x0 = take((size_t)TD_MAXB * d);
+        offs[p].x1 = take((size_t)TD_MAXB * d);
+        offs[p].att = take((size_t)TD_MAXB * H * c->td_teams_host[p].n_att_split * (hd + 2));
+        for (int i = 0; i < c->td_phase_count[p]; ++i) {
+            const TdPhase &q = c->td_phases_host[c->td_phase_begin[p] + i];
+            offs[p].out.push_back(td_is_gemm(q.kind) ? take((size_t)q.n_mat * q.n_split * TD_MAXB * q.n_rows) : 0);
+        }
+    }
+    c->td_buf_bytes = (int64_t)floats * 4;
+    CU(cudaMalloc((void **)&c->td_buf, std::max<size_t>(floats, 4) * 4));
+    CU(cudaMemset(c->td_buf, 0, std::max<size_t>(floats, 4) * 4));
+    auto add_map = [&](const void *W, int rows, int cols, int *idx) -> int {
+        CUtensorMap m;
+        const CUresult r = tg_make_map(&m, W, (uint64_t)rows, (uint64_t)cols, TG_BM);
+        if (r != CUDA_SUCCESS) return fail(c, MDI_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) for a %d x %d matrix", (int)r, rows, cols);
+        *idx = (int)maps.size();
+        maps.push_back(m);
+        return MDI_OK;
+    };
+    std::vector<std::pair<int, int>> map_idx(c->td_phases_host.size(), {-1, -1});
+    for (int p = 0; p < K; ++p) {
+        Partition &P = c->part[p];
+        for (int i = 0; i < c->td_phase_count[p]; ++i) {
+            const int gi = c->td_phase_begin[p] + i;
+            TdPhase &q = c->td_phases_host[gi];
+            if (!td_is_gemm(q.kind)) continue;
+            int rc = MDI_OK;
+            if (q.kind == TD_HEAD) rc = add_map(s.tied_lm_head ? c->wte : c->lm_head, V, d, &map_idx[gi].first);
+            else {
+                const LayerW &L = c->layer[P.lo + q.layer_local];
+                if (q.kind == TD_QKV) rc = add_map(L.wqkv, qw + 2 * kw, d, &map_idx[gi].first);
+                else if (q.kind == TD_OUT) rc = add_map(L.wo, d, qw, &map_idx[gi].first);
+                else if (q.kind == TD_UP && s.act == MDI_ACT_SWIGLU) {
+                    rc = add_map(L.wgate, F, d, &map_idx[gi].first);
+                    if (rc == MDI_OK) rc = add_map(L.wup, F, d, &map_idx[gi].second);
+                } else if (q.kind == TD_UP) rc = add_map(L.w1, F, d, &map_idx[gi].first);
+                else rc = add_map(s.act == MDI_ACT_SWIGLU ? L.wdown : L.w2, d, F, &map_idx[gi].first);
+            }
+            if (rc != MDI_OK) return rc;
+        }
+    }
+    CU(cudaMalloc((void **)&c->td_maps, std::max<size_t>(maps.size(), 1) * sizeof(CUtensorMap)));
+    CU(cudaMemcpy(c->td_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice));
+    for (int p = 0; p < K; ++p) {
+        Partition &P = c->part[p];
+        const Off &o = offs[p];
+        float *x0 = c->td_buf + o.x0, *x1 = c->td_buf + o.x1;
+        const int Lp = P.hi - P.lo;
+        // out buffer and split count of the phase of a given kind in local layer ll
+        auto find = [&](int kind, int ll) {
+            for (int i = 0; i < c->td_phase_count[p]; ++i) {
+                const TdPhase &q = c->td_phases_host[c->td_phase_begin[p] + i];
+                if (q.kind == kind && q.layer_local == ll) return i;
+            }
+            return -1;
+        };
+        for (int i = 0; i < c->td_phase_count[p]; ++i) {
+            const int gi = c->td_phase_begin[p] + i;
+            TdPhase &q = c->td_phases_host[gi];
+            const int ll = q.layer_local;
+            if (td_is_gemm(q.kind)) {
+                q.out = c->td_buf + o.out[i];
+                q.wmap[0] = map_idx[gi].first >= 0 ? c->td_maps + map_idx[gi].first : nullptr;
+                q.wmap[1] = map_idx[gi].second >= 0 ? c->td_maps + map_idx[gi].second : nullptr;
+            }
+            // the MLP-down sums of the previous block (if any) complete the residual stream that enters block ll
+            auto from_down = [&](int prev_ll) {
+                const int di = find(TD_DOWN, prev_ll);
+                const TdPhase &dn = c->td_phases_host[c->td_phase_begin[p] + di];
+                q.src = x1; q.part_in = c->td_buf + o.out[di]; q.s_in = dn.n_split; q.ld_in = d;
+                q.bias_in = s.has_bias ? c->layer[P.lo + prev_ll].b2 : nullptr;
+            };
+            if (q.kind == TD_QKV) {
+                const LayerW &L = c->layer[P.lo + ll];
+                q.gamma = L.ln1g; q.beta = L.ln1b; q.dst = x0;
+                if (ll > 0) from_down(ll - 1);
+            } else if (q.kind == TD_ATTN) {
+                const int qi = find(TD_QKV, ll);
+                const TdPhase &qq = c->td_phases_host[c->td_phase_begin[p] + qi];
+                q.part_in = c->td_buf + o.out[qi]; q.s_in = qq.n_split; q.ld_in = qw + 2 * kw;
+                q.bias_in = s.has_bias ? c->layer[P.lo + ll].bqkv : nullptr;
+            } else if (q.kind == TD_UP) {
+                const LayerW &L = c->layer[P.lo + ll];
+                const int oi = find(TD_OUT, ll);
+                const TdPhase &oo = c->td_phases_host[c->td_phase_begin[p] + oi];
+                q.gamma = L.ln2g; q.beta = L.ln2b; q.src = x0; q.dst = x1;
+                q.part_in = c->td_buf + o.out[oi]; q.s_in = oo.n_split; q.ld_in = d;
+                q.bias_in = s.has_bias ? L.bo : nullptr;
+            } else if (q.kind == TD_DOWN) {
+                const int ui = find(TD_UP, ll);
+                const TdPhase &uu = c->td_phases_host[c->td_phase_begin[p] + ui];
+                q.part_in = c->td_buf + o.out[ui]; q.s_in = uu.n_split; q.ld_in = F;
+                q.bias_in = s.has_bias ? c->layer[P.lo + ll].b1 : nullptr;
+            } else if (q.kind == TD_HEAD) {
+                q.gamma = c->lnfg; q.beta = c->lnfb; q.dst = nullptr;
+                from_down(Lp - 1);
+            } else if (q.kind == TD_FIN) {
+                from_down(Lp - 1);
+            }
+        }
+        TdTeam &T = c->td_teams_host[p];
+        T.kv = kv_view(c, P);
+        T.ring_in = p > 0 ? c->part[p - 1].ring : nullptr;
+        T.ring_out = p < K - 1 ? P.ring : nullptr;
+        T.att_part = c->td_buf + o.att;
+        T.pos = P.pos_dev;
+        T.bar = c->td_sync + (size_t)p * 64;
+        T.flag_out = c->td_sync + (size_t)p * 64 + 32;
+        T.flag_in = c->td_sync + (size_t)((p + K - 1) % K) * 64 + 32;
+    }
+    CU(cudaMalloc((void **)&c->td_teams, sizeof(TdTeam) * K));
+    CU(cudaMemcpy(c->td_teams, c->td_teams_host.data(), sizeof(TdTeam) * K, cudaMemcpyHostToDevice));
+    CU(cudaMalloc((void **)&c->td_phases, sizeof(TdPhase) * c->td_phases_host.size()));
+    CU(cudaMemcpy(c->td_phases, c->td_phases_host.data(), sizeof(TdPhase) * c->td_phases_host.size(), cudaMemcpyHostToDevice));
+    c->td_stale = false;
+    return MDI_OK;
+}
+
+int td_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
+    const mdi_model_shape &s = c->s;
+    int rc = td_build(c);
+    if (rc != MDI_OK) return rc;
+    CU(cudaMemsetAsync(c->td_sync, 0, (size_t)c->K * 64 * sizeof(unsigned), c->main));
+    CU(cudaMemsetAsync(c->td_err, 0, sizeof(int), c->main));
+    if (c->td_prof) CU(cudaMemsetAsync(c->td_prof, 0, (size_t)c->td_grid * PK_PROF_N * 8, c->main));
+    TdParams P{};
+    P.d = s.d_model; P.n_head = s.n_head; P.n_kv_head = s.n_kv_head; P.head_dim = s.head_dim; P.d_ff = s.d_ff; P.vocab = s.vocab;
+    P.norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS; P.act = s.act; P.rope = s.arch == MDI_ARCH_LLAMA;
+    P.K = c->K; P.G = G; P.n_samples = n_samples; P.gmax = c->gmax; P.n_pass = n_pass;
+    P.eps = s.norm_eps; P.scale = 1.0f / std::sqrt((float)s.head_dim);
+    P.teams = c->td_teams; P.phases = c->td_phases; P.wte = c->wte; P.wpe = c->wpe; P.rope_cos = c->rope_cos; P.rope_sin = c->rope_sin;
+    P.logits = c->logits; P.head_pv = c->head_pv; P.head_pi = c->head_pi; P.cur_tok = c->cur_tok; P.tok_log = c->tok_log;
+    P.gen_count = c->gen_count; P.teacher = c->teacher; P.n_teacher = c->n_teacher; P.log_stride = s.n_ctx; P.err = c->td_err;
+    P.wait_ns = c->o.wait_limit_ms > 0 ? (unsigned long long)c->o.wait_limit_ms * 1000000ull : PK_WAIT_NS;
+    P.withhold_partition = c->withhold_once;
+    c->withhold_once = -1;
+    P.prof = c->td_prof;
+    void *args[] = {&P};
+    CU(cudaLaunchCooperativeKernel(td_func(c), dim3(c->td_grid), dim3(TD_THREADS), args, c->td_smem, c->main));
+    ++c->st.kernel_launches;
+    c->st.stage_steps += (int64_t)c->K * n_pass * G;
+    return MDI_OK;
+}
+
 } // namespace
 
 // Used by entry points that take no context (other files of the library): text for mdi_last_error(NULL).
@@ -1295,7 +1605,8 @@ void mdi_destroy(mdi_ctx *c) {
     }
     void *ptrs[] = {c->rope_cos, c->rope_sin, c->logits, c->head_pv, c->head_pi, c->head_ticket, c->cur_tok, c->tok_log,
                     c->gen_count, c->teacher, c->n_teacher, c->prompt_buf, c->pk_teams, c->pk_phases, c->pk_sync, c->pk_err, c->pk_prof, c->tg_err,
-                    c->fz_teams, c->fz_phases, c->fz_works, c->fz_blocks, c->fz_segs, c->fz_units, c->fz_err, c->fz_stream, c->fz_acc, c->fz_sync, c->fz_prof, c->fz_trace};
+                    c->fz_teams, c->fz_phases, c->fz_works, c->fz_blocks, c->fz_segs, c->fz_units, c->fz_err, c->fz_stream, c->fz_acc, c->fz_sync, c->fz_prof, c->fz_trace,
+                    c->td_teams, c->td_phases, c->td_maps, c->td_buf, c->td_sync, c->td_err, c->td_prof};
     for (void *q : ptrs) if (q) cudaFree(q);
     cudaEvent_t evs[] = {c->ev_fork, c->ev_fork_cap, c->ev_t0, c->ev_t1, c->ev_pf0, c->ev_pf1};
     for (auto e : evs) if (e) cudaEventDestroy(e);
@@ -1344,8 +1655,9 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     // default page: 16 rows; 128 rows where the fused-phase kernel can run (GPT block, bf16 weights, fp32 cache), which
     // copies one head's rows of a page with one bulk copy each for keys and values and wants those copies large
     {
-        const bool fused_candidate = s.arch == MDI_ARCH_GPT && s.weight_dtype == MDI_DTYPE_BF16 && !c->o.kv_cache_bf16 &&
-                                     s.n_kv_head == s.n_head && c->o.scheduler != 1 && c->o.scheduler != 2 && s.head_dim <= 64;
+        const bool fused_candidate = s.arch == MDI_ARCH_GPT && s.weight_dtype == MDI_DTYPE_BF16 &&
+                                     (c->o.kv_cache_dtype == MDI_KV_DEFAULT || c->o.kv_cache_dtype == MDI_KV_F32) &&
+                                     s.n_kv_head == s.n_head && c->o.scheduler != 1 && c->o.scheduler != 2 && c->o.scheduler != 4 && s.head_dim <= 64;
         c->page_tokens = c->o.page_tokens > 0 ? c->o.page_tokens : (fused_candidate ? 128 : 16);
     }
     if (c->page_tokens & (c->page_tokens - 1)) return bail(fail(c, MDI_ERR_ARG, "page_tokens must be a power of two"));
@@ -1353,7 +1665,9 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     while ((1 << c->page_shift) < c->page_tokens) ++c->page_shift;
     c->pages_per_seq = (s.n_ctx + c->page_tokens - 1) / c->page_tokens;
     c->esize = s.weight_dtype == MDI_DTYPE_F32 ? 4 : 2;
-    c->kv_f32 = !(c->o.kv_cache_bf16 && s.weight_dtype == MDI_DTYPE_BF16);
+    if (c->o.kv_cache_dtype < 0 || c->o.kv_cache_dtype > 3) return bail(fail(c, MDI_ERR_ARG, "kv_cache_dtype must be one of MDI_KV_*"));
+    c->kv_kind = s.weight_dtype != MDI_DTYPE_BF16 ? KV_F32 : c->o.kv_cache_dtype == MDI_KV_BF16 ? KV_BF16 : c->o.kv_cache_dtype == MDI_KV_F16 ? KV_F16 : KV_F32;
+    c->kv_f32 = c->kv_kind == KV_F32;
     c->kv_esize = c->kv_f32 ? 4 : 2;
     c->page_elems = (size_t)2 * s.n_kv_head * c->page_tokens * s.head_dim;
     c->n_split = c->o.attn_splits > 0 ? c->o.attn_splits : std::max(1, std::min(16, s.n_ctx / 128));
@@ -1362,7 +1676,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     if (c->o.debug_withhold_handoff < 0 || c->o.debug_withhold_handoff > K) return bail(fail(c, MDI_ERR_ARG, "debug_withhold_handoff must name a partition (1-based) or be 0"));
     c->withhold_once = c->o.debug_withhold_handoff - 1;
     c->scheduler = c->o.scheduler;
-    if (c->scheduler < 0 || c->scheduler > 3) return bail(fail(c, MDI_ERR_ARG, "scheduler must be 0, 1, 2 or 3"));
+    if (c->scheduler < 0 || c->scheduler > 4) return bail(fail(c, MDI_ERR_ARG, "scheduler must be 0, 1, 2, 3 or 4"));
     const int G = std::min(n_samples, K);
     c->gmax = (n_samples + G - 1) / G;
     const long pool_tokens = c->o.kv_pool_tokens > 0 ? c->o.kv_pool_tokens : (long)n_samples * s.n_ctx;
@@ -1493,6 +1807,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     TRY(pk_setup(c));
     TRY(pf_setup(c));
     TRY(fz_setup(c));
+    TRY(td_setup(c));
     CUB(cudaDeviceSynchronize());
 #undef TRY
 #undef CUB
@@ -1523,6 +1838,7 @@ int mdi_load_weights(mdi_ctx *c, const char *name, const void *host, size_t nbyt
     if (!t.loaded) { t.loaded = true; ++c->n_loaded; }
     c->pk_tables_stale = true;
     c->fz_stale = true;
+    c->td_stale = true;
     return MDI_OK;
 }
 
@@ -1737,9 +2053,14 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
     const bool small_groups = c->temperature <= 0.f && (n_samples + G - 1) / G <= PK_MAXNB &&
                               !(c->pf_tc && c->scheduler == 0 && (n_samples + G - 1) / G >= c->tc_min_group);
     const bool use_fz = c->fz_ok && (c->scheduler == 0 || c->scheduler == 3) && small_groups && fz_slot_count_fits(c, n_pass, G);
-    const bool use_pk = !use_fz && c->pk_ok && c->scheduler != 1 && c->scheduler != 3 && small_groups && pk_tile_count_fits(c, n_pass, G);
+    const bool use_pk = !use_fz && c->pk_ok && c->scheduler != 1 && c->scheduler != 3 && c->scheduler != 4 && small_groups && pk_tile_count_fits(c, n_pass, G);
+    // the tensor-core persistent kernel: large blocks of the model or groups of 5 to 8 samples (what the stream scheduler
+    // would run as tensor-core steps), greedy token choice
+    const bool use_td = !use_fz && !use_pk && c->td_ok && c->temperature <= 0.f && (n_samples + G - 1) / G <= TD_MAXB &&
+                        (c->scheduler == 4 || (c->scheduler == 0 && !small_groups));
     if (c->scheduler == 2 && !use_pk) return fail(c, MDI_ERR_SHAPE, "persistent scheduler unavailable for this call");
     if (c->scheduler == 3 && !use_fz) return fail(c, MDI_ERR_SHAPE, "fused-phase scheduler unavailable for this call");
+    if (c->scheduler == 4 && !use_td) return fail(c, MDI_ERR_SHAPE, "tensor-core persistent scheduler unavailable for this call");
     // From here on work is queued that advances positions and counters on the device; the host's copies follow only
     // once all of it has run.  A failure half-way leaves the two out of step, so it forgets every sample.
     auto enqueue_all = [&]() -> int {
@@ -1751,6 +2072,9 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
         } else if (t_total && use_pk) {
             if ((rc = pk_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
             c->last_kernel = 1;
+        } else if (t_total && use_td) {
+            if ((rc = td_launch(c, n_samples, G, n_pass)) != MDI_OK) return rc;
+            c->last_kernel = 3;
         } else if (t_total) {
             const int R = c->rounds_per_graph;
             const long t_steady = K > 1 ? K : 0; // first tick, multiple of K, from which every partition is in steady state
@@ -1812,9 +2136,9 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
         forget_all();
         return fail(c, rc, "%s; all samples were reset", why.c_str());
     }
-    if (t_total && (use_pk || use_fz)) {
+    if (t_total && (use_pk || use_fz || use_td)) {
         int kerr = 0;
-        CU(cudaMemcpy(&kerr, use_fz ? c->fz_err : c->pk_err, sizeof(int), cudaMemcpyDeviceToHost));
+        CU(cudaMemcpy(&kerr, use_fz ? c->fz_err : use_td ? c->td_err : c->pk_err, sizeof(int), cudaMemcpyDeviceToHost));
         if (kerr) {
             // the pipeline stopped half-way: positions, caches and counters no longer agree
             forget_all();
@@ -1883,6 +2207,7 @@ int mdi_get_stats(mdi_ctx *c, mdi_stats *out) {
     c->st.n_partitions = c->K;
     c->st.n_samples = c->S;
     c->st.n_groups = std::min(c->S, c->K);
+    c->st.kv_element_bytes = (int)c->kv_esize;
     for (int p = 0; p < c->K && p < 16; ++p) {
         c->st.weight_bytes[p] = c->part[p].weight_bytes;
         c->st.kv_pool_bytes[p] = (int64_t)c->part[p].kv_bytes;
@@ -1895,15 +2220,15 @@ int mdi_get_stats(mdi_ctx *c, mdi_stats *out) {
 int mdi_get_partition_times(mdi_ctx *c, int p, double *out_ms, int n) {
     if (!c || !out_ms) return fail(c, MDI_ERR_ARG, "null argument");
     if (p < 0 || p >= c->K || n < 1) return fail(c, MDI_ERR_ARG, "partition out of range");
-    const bool fz = c->last_kernel == 2;
-    if (fz ? !(c->fz_ok && c->fz_prof_on) : !(c->pk_ok && c->pk_prof_on))
+    const bool fz = c->last_kernel == 2, td = c->last_kernel == 3;
+    if (td ? !(c->td_ok && c->td_prof) : fz ? !(c->fz_ok && c->fz_prof_on) : !(c->pk_ok && c->pk_prof_on))
         return fail(c, MDI_ERR_STATE, "in-kernel timing is off (options.in_kernel_timing at mdi_create; persistent schedulers only)");
     CU(cudaSetDevice(c->dev));
     CU(cudaDeviceSynchronize());
-    const int first_cta = fz ? c->fz_teams_host[p].first_cta : c->pk_teams_host[p].first_cta;
-    const int n_cta = fz ? c->fz_teams_host[p].n_cta : c->pk_teams_host[p].n_cta;
+    const int first_cta = td ? c->td_teams_host[p].first_cta : fz ? c->fz_teams_host[p].first_cta : c->pk_teams_host[p].first_cta;
+    const int n_cta = td ? c->td_teams_host[p].n_cta : fz ? c->fz_teams_host[p].n_cta : c->pk_teams_host[p].n_cta;
     std::vector<unsigned long long> h((size_t)n_cta * PK_PROF_N);
-    CU(cudaMemcpy(h.data(), (fz ? c->fz_prof : c->pk_prof) + (size_t)first_cta * PK_PROF_N, h.size() * 8, cudaMemcpyDeviceToHost));
+    CU(cudaMemcpy(h.data(), (td ? c->td_prof : fz ? c->fz_prof : c->pk_prof) + (size_t)first_cta * PK_PROF_N, h.size() * 8, cudaMemcpyDeviceToHost));
     for (int i = 0; i < n; ++i) {
         double acc = 0;
         for (int k = 0; k < n_cta && i < PK_PROF_N; ++k) acc += (double)h[(size_t)k * PK_PROF_N + i];
@@ -1926,7 +2251,7 @@ int mdi_get_trace(mdi_ctx *c, uint64_t *out_host, int n_words) {
 int64_t mdi_memory_bytes(mdi_ctx *c, int p) {
     if (!c || p < 0 || p >= c->K) return MDI_ERR_ARG;
     return c->part[p].weight_bytes + (int64_t)c->part[p].kv_bytes + c->part[p].buffer_bytes +
-           (p < (int)c->fz_team_stream_bytes.size() ? c->fz_team_stream_bytes[p] : 0);
+           (p < (int)c->fz_team_stream_bytes.size() ? c->fz_team_stream_bytes[p] : 0) + (c->K ? c->td_buf_bytes / c->K : 0);
 }
 
 } // extern "C"

@@ -205,6 +205,16 @@ template <int ES> __device__ __forceinline__ void pk_unpack(const uint4 &v, floa
     }
 }
 
+// 16 bytes of cache elements widened to fp32
+template <typename KT> __device__ __forceinline__ void kv_unpack(const uint4 &v, float *w) {
+    if constexpr (sizeof(KT) == 4) pk_unpack<4>(v, w);
+    else if constexpr (std::is_same<KT, __half>::value) {
+        const __half2 *h = reinterpret_cast<const __half2 *>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { const float2 f = __half22float2(h[i]); w[2 * i] = f.x; w[2 * i + 1] = f.y; }
+    } else pk_unpack<2>(v, w);
+}
+
 // Position of logical column i inside an item's staged input row.  For 2-byte weights a lane consumes
 // 8 consecutive columns per step as two float4 reads; columns are laid out so that each of those reads
 // is contiguous across the 32 lanes (no bank conflicts): within every group of 256 columns, first the
@@ -419,8 +429,8 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
                             const KT *vp = kp + (size_t)T.kv.n_kv_head * T.kv.page_tokens * hd;
                             float kf[EPL], vf[EPL];
                             const uint4 kk = __ldcg(reinterpret_cast<const uint4 *>(kp)), vv = __ldcg(reinterpret_cast<const uint4 *>(vp));
-                            pk_unpack<(int)sizeof(KT)>(kk, kf);
-                            pk_unpack<(int)sizeof(KT)>(vv, vf);
+                            kv_unpack<KT>(kk, kf);
+                            kv_unpack<KT>(vv, vf);
                             float s = 0.f;
 #pragma unroll
                             for (int e = 0; e < EPL; ++e) s = fmaf(q[e], kf[e], s);

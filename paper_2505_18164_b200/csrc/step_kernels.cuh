@@ -8,6 +8,7 @@
 // visit of a sample they are consecutive prompt positions of one slot.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -108,6 +109,21 @@ template <> struct WVec<__nv_bfloat16> {
     }
 };
 
+template <> struct WVec<__half> {     // key/value cache rows only
+    static constexpr int N = 8;
+    uint4 v;
+    __device__ __forceinline__ void load(const __half *p) { v = __ldg(reinterpret_cast<const uint4 *>(p)); }
+    __device__ __forceinline__ void unpack(float *w) const {
+        const __half2 *h = reinterpret_cast<const __half2 *>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(h[i]);
+            w[2 * i] = f.x;
+            w[2 * i + 1] = f.y;
+        }
+    }
+};
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -134,6 +150,7 @@ __device__ __forceinline__ float silu_f(float x) { return x / (1.f + expf(-x)); 
 template <typename KT> __device__ __forceinline__ void kv_store(KT *p, float v);
 template <> __device__ __forceinline__ void kv_store<float>(float *p, float v) { *p = v; }
 template <> __device__ __forceinline__ void kv_store<__nv_bfloat16>(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ void kv_store<__half>(__half *p, float v) { *p = __float2half_rn(v); }
 
 // Element address of (K or V, kv head, row, e) of a slot's cache in one local layer.
 template <typename KT>

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libmdi.so")
 
 MDI_OK = 0
 TRACE_WORDS = 128
+KV_DEFAULT, KV_BF16, KV_F16, KV_F32 = 0, 1, 2, 3
 ERR_ARG, ERR_SHAPE, ERR_OOM, ERR_CONTEXT, ERR_STATE, ERR_TIMEOUT, ERR_CUDA = -1, -2, -3, -4, -5, -6, -7
 _ERR_NAMES = {ERR_ARG: "MDI_ERR_ARG", ERR_SHAPE: "MDI_ERR_SHAPE", ERR_OOM: "MDI_ERR_OOM", ERR_CONTEXT: "MDI_ERR_CONTEXT",
               ERR_STATE: "MDI_ERR_STATE", ERR_TIMEOUT: "MDI_ERR_TIMEOUT", ERR_CUDA: "MDI_ERR_CUDA"}
@@ -41,7 +42,7 @@ class ModelShape(ctypes.Structure):
 
 class Options(ctypes.Structure):
     _fields_ = [("page_tokens", ctypes.c_int), ("kv_pool_tokens", ctypes.c_int), ("attn_splits", ctypes.c_int),
-                ("rounds_per_graph", ctypes.c_int), ("kv_cache_bf16", ctypes.c_int), ("prefill_mode", ctypes.c_int), ("tc_min_group", ctypes.c_int), ("wait_limit_ms", ctypes.c_int), ("debug_withhold_handoff", ctypes.c_int),
+                ("rounds_per_graph", ctypes.c_int), ("kv_cache_dtype", ctypes.c_int), ("prefill_mode", ctypes.c_int), ("tc_min_group", ctypes.c_int), ("wait_limit_ms", ctypes.c_int), ("debug_withhold_handoff", ctypes.c_int),
                 ("scheduler", ctypes.c_int), ("in_kernel_timing", ctypes.c_int), ("fused_blocks_per_head", ctypes.c_int),
                 ("debug_refuse_cluster_launch", ctypes.c_int), ("trace_slot", ctypes.c_int)]
 
@@ -52,7 +53,7 @@ class Stats(ctypes.Structure):
                 ("kv_pages_in_use", ctypes.c_int64 * 16), ("tokens_generated", ctypes.c_int64),
                 ("stage_steps", ctypes.c_int64), ("kernel_launches", ctypes.c_int64),
                 ("last_prefill_ms", ctypes.c_float), ("last_generate_ms", ctypes.c_float),
-                ("last_run_ms", ctypes.c_float)]
+                ("last_run_ms", ctypes.c_float), ("kv_element_bytes", ctypes.c_int)]
 
 
 _lib = None
@@ -117,7 +118,7 @@ class Context:
 
     def __init__(self, shape, part_bounds: Sequence[int], n_samples: int, page_tokens: int = 0,
                  kv_pool_tokens: int = 0, attn_splits: int = 0, rounds_per_graph: int = 0, scheduler: int = 0,
-                 kv_cache_bf16: int = 0, prefill_mode: int = 0, tc_min_group: int = 0,
+                 kv_cache_dtype: int = 0, prefill_mode: int = 0, tc_min_group: int = 0,
                  wait_limit_ms: int = 0, debug_withhold_handoff: int = 0, in_kernel_timing: int = 0,
                  fused_blocks_per_head: int = 0, debug_refuse_cluster_launch: int = 0, trace_slot: int = 0):
         self._h = None
@@ -126,7 +127,7 @@ class Context:
         self.n_samples = n_samples
         cs = ModelShape(**{n: getattr(shape, n) for n, _ in ModelShape._fields_})
         bounds = (ctypes.c_int * len(part_bounds))(*part_bounds)
-        opts = Options(page_tokens, kv_pool_tokens, attn_splits, rounds_per_graph, kv_cache_bf16, prefill_mode, tc_min_group,
+        opts = Options(page_tokens, kv_pool_tokens, attn_splits, rounds_per_graph, kv_cache_dtype, prefill_mode, tc_min_group,
                        wait_limit_ms, debug_withhold_handoff, scheduler, in_kernel_timing, fused_blocks_per_head,
                        debug_refuse_cluster_launch, trace_slot)
         h = ctypes.c_void_p()

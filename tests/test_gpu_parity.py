@@ -64,11 +64,14 @@ CASES = [
     ("gpt", I.DT_F32, 4, 64, 4, None, 97, 64, [0, 4], 1, 5, 12, {}),
     ("gpt", I.DT_F32, 4, 64, 4, None, 97, 64, [0, 1, 2, 4], 3, 7, 20, dict(page_tokens=4, attn_splits=3)),
     ("gpt", I.DT_BF16, 4, 64, 4, None, 97, 64, [0, 2, 4], 5, 9, 16, dict(page_tokens=8, attn_splits=2)),
-    ("gpt", I.DT_BF16, 4, 64, 4, None, 97, 64, [0, 2, 4], 5, 9, 16, dict(page_tokens=8, attn_splits=2, kv_cache_bf16=1)),
+    ("gpt", I.DT_BF16, 4, 64, 4, None, 97, 64, [0, 2, 4], 5, 9, 16, dict(page_tokens=8, attn_splits=2, kv_cache_dtype=1)),
     ("gpt", I.DT_BF16, 3, 128, 2, None, 131, 96, [0, 1, 2, 3], 2, 17, 30, dict(attn_splits=4)),
     ("gpt", I.DT_BF16, 3, 128, 2, None, 131, 96, [0, 1, 2, 3], 2, 17, 30, dict(attn_splits=4, prefill_mode=1)),
     ("llama", I.DT_BF16, 4, 64, 4, None, 101, 64, [0, 2, 3, 4], 3, 6, 20, dict(page_tokens=4, attn_splits=2)),
-    ("llama", I.DT_BF16, 4, 64, 4, None, 101, 64, [0, 2, 3, 4], 3, 6, 20, dict(page_tokens=4, attn_splits=2, kv_cache_bf16=1)),
+    ("llama", I.DT_BF16, 4, 64, 4, None, 101, 64, [0, 2, 3, 4], 3, 6, 20, dict(page_tokens=4, attn_splits=2, kv_cache_dtype=1)),
+    ("gpt", I.DT_BF16, 4, 64, 4, None, 97, 64, [0, 2, 4], 5, 9, 16, dict(page_tokens=8, attn_splits=2, kv_cache_dtype=2)),   # fp16 cache
+    ("llama", I.DT_BF16, 4, 64, 4, 2, 101, 64, [0, 2, 3, 4], 3, 6, 20, dict(page_tokens=4, attn_splits=2, kv_cache_dtype=2)),
+    ("llama", I.DT_BF16, 2, 256, 2, 1, 300, 40, [0, 2], 11, 3, 10, dict(kv_cache_dtype=2)),   # fp16 cache, tensor-core steps
     ("llama", I.DT_F32, 2, 128, 4, 2, 67, 48, [0, 1, 2], 4, 11, 14, dict(attn_splits=3)),
     ("llama", I.DT_BF16, 2, 256, 2, 1, 300, 40, [0, 2], 11, 3, 10, {}),         # one partition, group > 8 items
     ("llama", I.DT_BF16, 2, 256, 2, 1, 300, 40, [0, 2], 11, 3, 10, dict(prefill_mode=1)),   # the same on the CUDA-core kernels

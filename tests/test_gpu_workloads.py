@@ -19,14 +19,14 @@ from helpers import parity_tolerance
 pytestmark = pytest.mark.gpu
 
 
-def _run(name, n_prompt=None, n_new=None, check=None, chunk=8, scheduler=0):
+def _run(name, n_prompt=None, n_new=None, check=None, chunk=8, scheduler=0, **ctx_opts):
     from paper_2505_18164_b200 import mdi
     w = I.ALL_WORKLOADS[name]
     w = I.scaled(w, n_prompt=n_prompt or w.n_prompt, n_new=n_new or w.n_new)
     s, S, P, N = w.shape, w.n_samples, w.n_prompt, w.n_new
     check = list(range(S)) if check is None else check
     tol = parity_tolerance(s)
-    ctx = mdi.Context(s, list(w.part_bounds), S, kv_pool_tokens=S * ((P + N + 15) // 16 * 16), scheduler=scheduler)
+    ctx = mdi.Context(s, list(w.part_bounds), S, kv_pool_tokens=S * ((P + N + 15) // 16 * 16), scheduler=scheduler, **ctx_opts)
     weights = {}
     for nm, a in I.iter_weights(s, w.weight_seed):
         ctx.load_weights(nm, a)
@@ -57,6 +57,7 @@ def _run(name, n_prompt=None, n_new=None, check=None, chunk=8, scheduler=0):
           f"{ctx.stats().kernel_launches} launches")
     assert worst <= tol, worst
     ctx.close()
+    return worst
 
 
 @pytest.mark.parametrize("scheduler", [0, 1], ids=["persistent", "streams"])
