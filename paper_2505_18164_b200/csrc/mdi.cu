@@ -168,7 +168,9 @@ struct mdi_ctx {
     TdTeam *td_teams = nullptr;
     TdPhase *td_phases = nullptr;
     CUtensorMap *td_maps = nullptr;
-    float *td_buf = nullptr;       // all scratch of the kernel (residual copies, partial sums), one allocation
+    float *td_buf = nullptr;       // all float scratch of the kernel (residual copies, partial and finished sums), one allocation
+    int *td_ints = nullptr;        // tickets and argmax candidates
+    size_t td_n_ints = 0;
     unsigned *td_sync = nullptr;
     int *td_err = nullptr;
     unsigned long long *td_prof = nullptr;
@@ -1341,7 +1343,11 @@ int td_setup(mdi_ctx *c) {
         CU(ea);
     }
     for (int p = 0; p < K; ++p)
-        if (5 * (c->part[p].hi - c->part[p].lo) + 2 > TD_MAX_PHASES) return no("too many blocks of the model in one partition");
+        if (5 * (c->part[p].hi - c->part[p].lo) + 1 > TD_MAX_PHASES) return no("too many blocks of the model in one partition");
+    // a warp hands out the page-table entries of its sequence split by shuffles: a split may span at most 32 pages
+    int min_att_split = 1;
+    while (min_att_split < TD_MAX_SPLITS && (c->pages_per_seq + min_att_split - 1) / min_att_split + 2 > 32) min_att_split *= 2;
+    if ((c->pages_per_seq + min_att_split - 1) / min_att_split + 2 > 32) return no("too many cache pages per sequence (use larger pages)");
     // team sizes in proportion to the bytes a partition step streams
     const double layer_bytes = 2.0 * ((double)(qw + 2 * kw) * d + (double)d * qw + (double)(s.act == MDI_ACT_SWIGLU ? 3 : 2) * F * d);
     std::vector<double> bytes(K);
@@ -1381,12 +1387,11 @@ int td_setup(mdi_ctx *c) {
             gemm(TD_QKV, l, 1, qw + 2 * kw, d, TDP_NORM);
             c->td_phases_host.back().first_of_step = l == 0;
             TdPhase a{}; a.kind = TD_ATTN; a.layer_local = l; c->td_phases_host.push_back(a);
-            gemm(TD_OUT, l, 1, d, qw, TDP_MERGE);
+            gemm(TD_OUT, l, 1, d, qw, TDP_COPY);
             gemm(TD_UP, l, s.act == MDI_ACT_SWIGLU ? 2 : 1, F, d, TDP_NORM);
             gemm(TD_DOWN, l, 1, d, F, TDP_ACT);
         }
         if (p == K - 1) gemm(TD_HEAD, Lp, 1, V, d, TDP_NORM);
-        else { TdPhase f{}; f.kind = TD_FIN; f.layer_local = Lp; c->td_phases_host.push_back(f); }
         c->td_phase_count[p] = (int)c->td_phases_host.size() - c->td_phase_begin[p];
         TdTeam &T = c->td_teams_host[p];
         T.first_cta = first; T.n_cta = n; first += n;
@@ -1395,9 +1400,9 @@ int td_setup(mdi_ctx *c) {
         // attention units (sample, head, split) over the team's warps: the split count that deals them out most evenly
         {
             const int warps = n * TD_CWARPS, pairs = c->gmax * H;
-            int best_s = 1;
+            int best_s = min_att_split;
             double best = -1.0;
-            for (int sp = 1; sp <= TD_MAX_SPLITS; sp *= 2) {
+            for (int sp = min_att_split; sp <= TD_MAX_SPLITS; sp *= 2) {
                 const long units = (long)pairs * sp, most = (units + warps - 1) / warps;
                 const double eff = (double)units / ((double)most * warps);
                 if (eff > best + 0.03) { best = eff; best_s = sp; }
@@ -1419,27 +1424,41 @@ int td_build(mdi_ctx *c) {
     if (!c->td_stale) return MDI_OK;
     const mdi_model_shape &s = c->s;
     const int K = c->K, d = s.d_model, hd = s.head_dim, H = s.n_head, qw = H * hd, kw = s.n_kv_head * hd, F = s.d_ff, V = s.vocab;
-    void *old[] = {c->td_teams, c->td_phases, c->td_maps, c->td_buf};
+    void *old[] = {c->td_teams, c->td_phases, c->td_maps, c->td_buf, c->td_ints};
     for (void *q : old) if (q) cudaFree(q);
-    c->td_teams = nullptr; c->td_phases = nullptr; c->td_maps = nullptr; c->td_buf = nullptr;
-    // one allocation for all scratch: first count, then carve
+    c->td_teams = nullptr; c->td_phases = nullptr; c->td_maps = nullptr; c->td_buf = nullptr; c->td_ints = nullptr;
+    // one allocation for all float scratch and one for all integers: first count, then carve
     std::vector<CUtensorMap> maps;
-    size_t floats = 0;
+    size_t floats = 0, ints = 0;
     auto take = [&](size_t n) { const size_t r = floats; floats += (n + 3) & ~(size_t)3; return r; };
-    struct Off { size_t x0, x1, att; std::vector<size_t> out; };
+    auto take_i = [&](size_t n) { const size_t r = ints; ints += (n + 3) & ~(size_t)3; return r; };
+    struct Off { size_t x0, x1, qkv, u, att_part, att_out, att_ticket, head_pv, head_pi; std::vector<size_t> part, ticket; };
     std::vector<Off> offs(K);
     for (int p = 0; p < K; ++p) {
-        offs[p].x0 = take((size_t)TD_MAXB * d);
-        offs[p].x1 = take((size_t)TD_MAXB * d);
-        offs[p].att = take((size_t)TD_MAXB * H * c->td_teams_host[p].n_att_split * (hd + 2));
+        Off &o = offs[p];
+        const TdTeam &T = c->td_teams_host[p];
+        o.x0 = take((size_t)TD_MAXB * d);
+        o.x1 = take((size_t)TD_MAXB * d);
+        o.qkv = take((size_t)TD_MAXB * (qw + 2 * kw));
+        o.u = take((size_t)2 * TD_MAXB * F);
+        o.att_part = take((size_t)TD_MAXB * H * T.n_att_split * (hd + 4));
+        o.att_out = take((size_t)TD_MAXB * qw);
+        o.att_ticket = take_i((size_t)TD_MAXB * H);
+        o.head_pv = o.head_pi = 0;
         for (int i = 0; i < c->td_phase_count[p]; ++i) {
             const TdPhase &q = c->td_phases_host[c->td_phase_begin[p] + i];
-            offs[p].out.push_back(td_is_gemm(q.kind) ? take((size_t)q.n_mat * q.n_split * TD_MAXB * q.n_rows) : 0);
+            const bool split = td_is_gemm(q.kind) && q.n_split > 1;
+            o.part.push_back(split ? take((size_t)q.n_mat * q.n_split * TD_MAXB * q.n_rows) : 0);
+            o.ticket.push_back(split ? take_i((size_t)q.n_mat * q.n_tiles) : 0);
+            if (q.kind == TD_HEAD) { o.head_pv = take((size_t)TD_MAXB * 4 * q.n_tiles); o.head_pi = take_i((size_t)TD_MAXB * 4 * q.n_tiles); }
         }
     }
-    c->td_buf_bytes = (int64_t)floats * 4;
+    c->td_buf_bytes = (int64_t)floats * 4 + (int64_t)ints * 4;
+    c->td_n_ints = ints;
     CU(cudaMalloc((void **)&c->td_buf, std::max<size_t>(floats, 4) * 4));
     CU(cudaMemset(c->td_buf, 0, std::max<size_t>(floats, 4) * 4));
+    CU(cudaMalloc((void **)&c->td_ints, std::max<size_t>(ints, 4) * 4));
+    CU(cudaMemset(c->td_ints, 0, std::max<size_t>(ints, 4) * 4));
     auto add_map = [&](const void *W, int rows, int cols, int *idx) -> int {
         CUtensorMap m;
         const CUresult r = tg_make_map(&m, W, (uint64_t)rows, (uint64_t)cols, TG_BM);
@@ -1475,65 +1494,55 @@ int td_build(mdi_ctx *c) {
     for (int p = 0; p < K; ++p) {
         Partition &P = c->part[p];
         const Off &o = offs[p];
-        float *x0 = c->td_buf + o.x0, *x1 = c->td_buf + o.x1;
+        float *x0 = c->td_buf + o.x0, *x1 = c->td_buf + o.x1, *qkv = c->td_buf + o.qkv, *u = c->td_buf + o.u;
         const int Lp = P.hi - P.lo;
-        // out buffer and split count of the phase of a given kind in local layer ll
-        auto find = [&](int kind, int ll) {
-            for (int i = 0; i < c->td_phase_count[p]; ++i) {
-                const TdPhase &q = c->td_phases_host[c->td_phase_begin[p] + i];
-                if (q.kind == kind && q.layer_local == ll) return i;
-            }
-            return -1;
-        };
         for (int i = 0; i < c->td_phase_count[p]; ++i) {
             const int gi = c->td_phase_begin[p] + i;
             TdPhase &q = c->td_phases_host[gi];
             const int ll = q.layer_local;
             if (td_is_gemm(q.kind)) {
-                q.out = c->td_buf + o.out[i];
                 q.wmap[0] = map_idx[gi].first >= 0 ? c->td_maps + map_idx[gi].first : nullptr;
                 q.wmap[1] = map_idx[gi].second >= 0 ? c->td_maps + map_idx[gi].second : nullptr;
+                q.part = q.n_split > 1 ? c->td_buf + o.part[i] : nullptr;
+                q.ticket = q.n_split > 1 ? c->td_ints + o.ticket[i] : nullptr;
             }
-            // the MLP-down sums of the previous block (if any) complete the residual stream that enters block ll
-            auto from_down = [&](int prev_ll) {
-                const int di = find(TD_DOWN, prev_ll);
-                const TdPhase &dn = c->td_phases_host[c->td_phase_begin[p] + di];
-                q.src = x1; q.part_in = c->td_buf + o.out[di]; q.s_in = dn.n_split; q.ld_in = d;
-                q.bias_in = s.has_bias ? c->layer[P.lo + prev_ll].b2 : nullptr;
-            };
-            if (q.kind == TD_QKV) {
-                const LayerW &L = c->layer[P.lo + ll];
-                q.gamma = L.ln1g; q.beta = L.ln1b; q.dst = x0;
-                if (ll > 0) from_down(ll - 1);
-            } else if (q.kind == TD_ATTN) {
-                const int qi = find(TD_QKV, ll);
-                const TdPhase &qq = c->td_phases_host[c->td_phase_begin[p] + qi];
-                q.part_in = c->td_buf + o.out[qi]; q.s_in = qq.n_split; q.ld_in = qw + 2 * kw;
-                q.bias_in = s.has_bias ? c->layer[P.lo + ll].bqkv : nullptr;
-            } else if (q.kind == TD_UP) {
-                const LayerW &L = c->layer[P.lo + ll];
-                const int oi = find(TD_OUT, ll);
-                const TdPhase &oo = c->td_phases_host[c->td_phase_begin[p] + oi];
-                q.gamma = L.ln2g; q.beta = L.ln2b; q.src = x0; q.dst = x1;
-                q.part_in = c->td_buf + o.out[oi]; q.s_in = oo.n_split; q.ld_in = d;
-                q.bias_in = s.has_bias ? L.bo : nullptr;
-            } else if (q.kind == TD_DOWN) {
-                const int ui = find(TD_UP, ll);
-                const TdPhase &uu = c->td_phases_host[c->td_phase_begin[p] + ui];
-                q.part_in = c->td_buf + o.out[ui]; q.s_in = uu.n_split; q.ld_in = F;
-                q.bias_in = s.has_bias ? c->layer[P.lo + ll].b1 : nullptr;
-            } else if (q.kind == TD_HEAD) {
-                q.gamma = c->lnfg; q.beta = c->lnfb; q.dst = nullptr;
-                from_down(Lp - 1);
-            } else if (q.kind == TD_FIN) {
-                from_down(Lp - 1);
+            const LayerW *L = ll < Lp ? &c->layer[P.lo + ll] : nullptr;
+            switch (q.kind) {
+                case TD_QKV:   // input: the residual stream entering the block (ring slot or embedding for the first block)
+                    q.src = x0; q.dst = (p == 0 && ll == 0) ? x0 : nullptr; q.gamma = L->ln1g; q.beta = L->ln1b;
+                    q.fin = qkv; q.fin_bias = s.has_bias ? L->bqkv : nullptr;
+                    break;
+                case TD_ATTN:
+                    q.src = qkv;
+                    break;
+                case TD_OUT:   // x1 = x0 + bo + Wo . attention
+                    q.src = c->td_buf + o.att_out;
+                    q.fin = x1; q.fin_bias = s.has_bias ? L->bo : nullptr;
+                    q.fin_resid = x0; q.fin_resid_ring = (ll == 0 && p > 0) ? 1 : 0;
+                    break;
+                case TD_UP:
+                    q.src = x1; q.gamma = L->ln2g; q.beta = L->ln2b;
+                    q.fin = u; q.fin_bias = s.has_bias ? L->b1 : nullptr;
+                    break;
+                case TD_DOWN:  // x0 (or the ring slot after the partition's last block) = x1 + b2 + W2 . hidden
+                    q.src = u;
+                    q.fin = x0; q.fin_bias = s.has_bias ? L->b2 : nullptr; q.fin_resid = x1;
+                    q.fin_ring = (ll == Lp - 1 && p < K - 1) ? 1 : 0;
+                    break;
+                default:       // TD_HEAD
+                    q.src = x0; q.gamma = c->lnfg; q.beta = c->lnfb;
+                    break;
             }
         }
         TdTeam &T = c->td_teams_host[p];
         T.kv = kv_view(c, P);
         T.ring_in = p > 0 ? c->part[p - 1].ring : nullptr;
         T.ring_out = p < K - 1 ? P.ring : nullptr;
-        T.att_part = c->td_buf + o.att;
+        T.att_part = c->td_buf + o.att_part;
+        T.att_out = c->td_buf + o.att_out;
+        T.att_ticket = c->td_ints + o.att_ticket;
+        T.head_pv = p == K - 1 ? c->td_buf + o.head_pv : nullptr;
+        T.head_pi = p == K - 1 ? c->td_ints + o.head_pi : nullptr;
         T.pos = P.pos_dev;
         T.bar = c->td_sync + (size_t)p * 64;
         T.flag_out = c->td_sync + (size_t)p * 64 + 32;
@@ -1553,6 +1562,7 @@ int td_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     if (rc != MDI_OK) return rc;
     CU(cudaMemsetAsync(c->td_sync, 0, (size_t)c->K * 64 * sizeof(unsigned), c->main));
     CU(cudaMemsetAsync(c->td_err, 0, sizeof(int), c->main));
+    CU(cudaMemsetAsync(c->td_ints, 0, std::max<size_t>(c->td_n_ints, 4) * 4, c->main)); // tickets start at zero (a timed-out call may have left some)
     if (c->td_prof) CU(cudaMemsetAsync(c->td_prof, 0, (size_t)c->td_grid * PK_PROF_N * 8, c->main));
     TdParams P{};
     P.d = s.d_model; P.n_head = s.n_head; P.n_kv_head = s.n_kv_head; P.head_dim = s.head_dim; P.d_ff = s.d_ff; P.vocab = s.vocab;
@@ -1560,7 +1570,7 @@ int td_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     P.K = c->K; P.G = G; P.n_samples = n_samples; P.gmax = c->gmax; P.n_pass = n_pass;
     P.eps = s.norm_eps; P.scale = 1.0f / std::sqrt((float)s.head_dim);
     P.teams = c->td_teams; P.phases = c->td_phases; P.wte = c->wte; P.wpe = c->wpe; P.rope_cos = c->rope_cos; P.rope_sin = c->rope_sin;
-    P.logits = c->logits; P.head_pv = c->head_pv; P.head_pi = c->head_pi; P.cur_tok = c->cur_tok; P.tok_log = c->tok_log;
+    P.logits = c->logits; P.cur_tok = c->cur_tok; P.tok_log = c->tok_log;
     P.gen_count = c->gen_count; P.teacher = c->teacher; P.n_teacher = c->n_teacher; P.log_stride = s.n_ctx; P.err = c->td_err;
     P.wait_ns = c->o.wait_limit_ms > 0 ? (unsigned long long)c->o.wait_limit_ms * 1000000ull : PK_WAIT_NS;
     P.withhold_partition = c->withhold_once;
@@ -1606,7 +1616,7 @@ void mdi_destroy(mdi_ctx *c) {
     void *ptrs[] = {c->rope_cos, c->rope_sin, c->logits, c->head_pv, c->head_pi, c->head_ticket, c->cur_tok, c->tok_log,
                     c->gen_count, c->teacher, c->n_teacher, c->prompt_buf, c->pk_teams, c->pk_phases, c->pk_sync, c->pk_err, c->pk_prof, c->tg_err,
                     c->fz_teams, c->fz_phases, c->fz_works, c->fz_blocks, c->fz_segs, c->fz_units, c->fz_err, c->fz_stream, c->fz_acc, c->fz_sync, c->fz_prof, c->fz_trace,
-                    c->td_teams, c->td_phases, c->td_maps, c->td_buf, c->td_sync, c->td_err, c->td_prof};
+                    c->td_teams, c->td_phases, c->td_maps, c->td_buf, c->td_ints, c->td_sync, c->td_err, c->td_prof};
     for (void *q : ptrs) if (q) cudaFree(q);
     cudaEvent_t evs[] = {c->ev_fork, c->ev_fork_cap, c->ev_t0, c->ev_t1, c->ev_pf0, c->ev_pf1};
     for (auto e : evs) if (e) cudaEventDestroy(e);
@@ -1658,7 +1668,10 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
         const bool fused_candidate = s.arch == MDI_ARCH_GPT && s.weight_dtype == MDI_DTYPE_BF16 &&
                                      (c->o.kv_cache_dtype == MDI_KV_DEFAULT || c->o.kv_cache_dtype == MDI_KV_F32) &&
                                      s.n_kv_head == s.n_head && c->o.scheduler != 1 && c->o.scheduler != 2 && c->o.scheduler != 4 && s.head_dim <= 64;
-        c->page_tokens = c->o.page_tokens > 0 ? c->o.page_tokens : (fused_candidate ? 128 : 16);
+        // ... and 64 rows where the tensor-core persistent kernel may run (a warp hands out the page-table entries of
+        // its sequence split by shuffles: fewer, larger pages)
+        const bool td_candidate = s.weight_dtype == MDI_DTYPE_BF16 && (c->o.scheduler == 0 || c->o.scheduler == 4);
+        c->page_tokens = c->o.page_tokens > 0 ? c->o.page_tokens : (fused_candidate ? 128 : td_candidate ? 64 : 16);
     }
     if (c->page_tokens & (c->page_tokens - 1)) return bail(fail(c, MDI_ERR_ARG, "page_tokens must be a power of two"));
     c->page_shift = 0;

@@ -12,16 +12,17 @@
 // instruction serves both and the two column halves of D are added when the accumulator is read back.
 //
 // Work of a linear layer is cut into units (matrix, 128-row tile, range of k-blocks) dealt out evenly over the
-// team's blocks; a unit leaves a raw partial sum in global memory.  Everything that is not a contraction happens
-// where those sums are consumed: the next phase's prologue adds the partial sums in a fixed order (so results do
-// not depend on timing), adds bias and residual, normalises, applies GELU / SwiGLU or merges the attention splits,
-// and writes its own range of the B operand straight into shared memory in the swizzled layout the tensor core
-// reads.  A block of the model therefore costs five team barriers: q/k/v rows | attention | output projection |
-// MLP up | MLP down.
+// team's blocks.  A unit leaves a raw partial sum in global memory and takes a ticket of its row tile; the unit that
+// arrives last adds the tile's partial sums in a fixed order (so results do not depend on timing), adds bias and
+// residual, and writes the finished rows: the residual stream, the q/k/v rows, the pre-activations, the logits.
+// Everything else that is not a contraction happens in the next phase's prologue, which reads finished values
+// only: it normalises, applies GELU / SwiGLU, splits into bf16 pairs and writes its own range of the B operand
+// straight into shared memory in the swizzled layout the tensor core reads.  A block of the model costs five team
+// barriers: q/k/v rows | attention | output projection | MLP up | MLP down.
 //
 // Attention (rotary embedding of q and k, append of the new cache row, online softmax over the slot's cached
 // rows) runs on the CUDA cores: (sample, head, sequence split) units dealt out over the team's warps, sixteen
-// cache rows in flight per warp.
+// cache rows in flight per warp, page-table entries fetched once per unit; the last split to arrive merges.
 //
 // Every wait (flag, team barrier, mbarrier) is bounded in wall time as in k_persistent_decode: when a limit is hit
 // an error word is set, nobody waits any more, tensor memory is freed and the kernel returns.
@@ -43,23 +44,27 @@ constexpr int TD_ACC = 4;                       // accumulators in tensor memory
 constexpr int TD_MAX_PHASES = 64;
 constexpr int TD_MAX_SPLITS = 16;               // attention splits over the sequence
 
-enum TdKind { TD_QKV = 0, TD_ATTN = 1, TD_OUT = 2, TD_UP = 3, TD_DOWN = 4, TD_HEAD = 5, TD_FIN = 6 };
-enum TdPro { TDP_NORM = 0, TDP_MERGE = 1, TDP_ACT = 2 };
+enum TdKind { TD_QKV = 0, TD_ATTN = 1, TD_OUT = 2, TD_UP = 3, TD_DOWN = 4, TD_HEAD = 5 };
+enum TdPro { TDP_NORM = 0, TDP_COPY = 1, TDP_ACT = 2 };
 
 struct TdPhase {
     int kind, layer_local;
     // contraction: n_mat matrices [n_rows][K] (2: gate and up), n_tiles row tiles, n_split ranges of kb_per_split k-blocks
     int n_mat, n_rows, K, n_tiles, n_kb, n_split, kb_per_split, n_units;
     const CUtensorMap *wmap[2];
-    float *out;              // raw partial sums [n_mat][n_split][TD_MAXB][n_rows]
-    // prologue (what the B operand is made of)
+    float *part;             // raw partial sums [n_mat][n_split][TD_MAXB][n_rows] (unused when n_split == 1)
+    int *ticket;             // [n_mat * n_tiles] arrivals per (matrix, row tile), zero between uses (unused when n_split == 1)
+    // what the unit that completes a row tile does: fin[mat][i][row] = sum + fin_bias[row] + resid[i][row]
+    const float *fin_bias;   // [n_rows] or null
+    const float *fin_resid;  // [TD_MAXB][n_rows] or null
+    int fin_resid_ring;      // 1: the residual is the previous partition's ring slot (first block of a step)
+    float *fin;              // [n_mat][TD_MAXB][n_rows] (output layer: the context's logits, by slot)
+    int fin_ring;            // 1: the result goes to this partition's ring slot (last block of a step)
+    // prologue: what the B operand is made of
     int pro;                 // TdPro
     int first_of_step;       // NORM: the input is the previous partition's ring slot, or the token embedding
-    const float *src;        // NORM: residual stream before this phase's addends [TD_MAXB][d]
-    float *dst;              // NORM: where the completed residual stream goes [TD_MAXB][d] (null: nowhere)
-    const float *part_in;    // partial sums to add up: [s_in][TD_MAXB][ld_in]  (ACT with two matrices: gate then up)
-    int s_in, ld_in;
-    const float *bias_in;    // bias that completes the incoming sums (null: none)
+    const float *src;        // NORM: residual stream [TD_MAXB][d]; COPY: [TD_MAXB][K]; ACT: [n_mat][TD_MAXB][K]; attention: q/k/v rows
+    float *dst;              // NORM of the very first block: where the embedded tokens are kept [TD_MAXB][d]
     const float *gamma, *beta;
 };
 
@@ -68,7 +73,11 @@ struct TdTeam {
     KvView kv;
     const float *ring_in;
     float *ring_out;
-    float *att_part;         // [TD_MAXB][n_head][n_att_split][head_dim + 2]
+    float *att_part;         // [TD_MAXB][n_head][n_att_split][head_dim + 4]: max, sum, -, -, o[head_dim]
+    float *att_out;          // [TD_MAXB][n_head * head_dim]
+    int *att_ticket;         // [TD_MAXB][n_head]
+    float *head_pv;          // last partition: argmax candidates [TD_MAXB][4 * row tiles of the vocabulary]
+    int *head_pi;
     int *pos;
     unsigned *bar, *flag_out;
     const unsigned *flag_in;
@@ -81,8 +90,7 @@ struct TdParams {
     const TdPhase *phases;
     const void *wte, *wpe;
     const float *rope_cos, *rope_sin;
-    float *logits, *head_pv;
-    int *head_pi;
+    float *logits;
     int *cur_tok, *tok_log, *gen_count;
     const int *teacher, *n_teacher;
     int log_stride;
@@ -94,7 +102,7 @@ struct TdParams {
 };
 
 struct TdSmem {
-    size_t ring, b, stats, red, best_v, best_i, s_dead, bars, tmem_slot, s_ph, total;
+    size_t ring, b, stats, red, s_flag, s_dead, bars, tmem_slot, s_ph, total;
 };
 __host__ __device__ inline TdSmem td_smem_layout() {
     TdSmem L;
@@ -104,8 +112,7 @@ __host__ __device__ inline TdSmem td_smem_layout() {
     L.b = take(TD_B_BYTES, 1024);
     L.stats = take(4 * 2 * TD_MAXB, 16);
     L.red = take(4 * 2 * TD_MAXB * TD_CWARPS, 16);
-    L.best_v = take(4 * TD_MAXB * TD_CWARPS, 16);
-    L.best_i = take(4 * TD_MAXB * TD_CWARPS, 16);
+    L.s_flag = take(8, 8);
     L.s_dead = take(8, 8);
     L.bars = take(8 * (2 * TD_STAGES + 2 * TD_ACC + 1), 8);
     L.tmem_slot = take(8, 8);
@@ -116,6 +123,7 @@ __host__ __device__ inline TdSmem td_smem_layout() {
 
 __host__ __device__ inline bool td_is_gemm(int kind) { return kind == TD_QKV || kind == TD_OUT || kind == TD_UP || kind == TD_DOWN || kind == TD_HEAD; }
 __device__ __forceinline__ void td_bar() { asm volatile("bar.sync 1, %0;" ::"n"(TD_CTHREADS) : "memory"); }
+__device__ __forceinline__ void td_epi_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); } // warps 4..7
 
 // unit u of a phase -> (k range, matrix, row tile); units are ordered k-range-major so that a block's units share B
 struct TdUnit { int ks, mat, tile, kb_lo, kb_hi; };
@@ -159,122 +167,178 @@ __device__ __forceinline__ float4 td_bf16x4(const __nv_bfloat16 *p) {
 }
 
 // ---- attention of one (sample, head, sequence split) by one warp ------------------------------------------------
-// q, and the new row's k and v, come from the raw sums of the q/k/v contraction (ph.part_in, ph.bias_in); rotary
-// embedding is applied here; the warp whose split ends at the new row uses it from registers, and for the first query
-// head of a key/value head also appends it to the cache.  Leaves (max, sum, o[head_dim]) of the split in att_part.
+// q, and the new row's k and v, are finished rows of the q/k/v contraction (bias included); rotary embedding is
+// applied here; the warp whose split ends at the new row uses it from registers, and for the first query head of a
+// key/value head also appends it to the cache.  Leaves (max, sum, o[head_dim]) of the split in att_part; the split
+// that arrives last merges all of them (in split order) into att_out.
 template <typename KT, int HD>
 __device__ __forceinline__ void td_attn_unit(const TdParams &P, const TdTeam &T, const TdPhase &ph, int i, int slot, int pos, int h, int sp,
                                              int lane) {
-    constexpr int EPL = 16 / (int)sizeof(KT), LPR = HD / EPL, RPW = 32 / LPR, U = 16 / RPW < 8 ? 16 / RPW : 8; // rows in flight: RPW * U
+    constexpr int EPL = 16 / (int)sizeof(KT), LPR = HD / EPL, RPW = 32 / LPR, U = 16 / RPW; // 16 cache rows in flight per warp
     static_assert(LPR >= 2 && LPR <= 32, "head_dim");
     const int sub = lane % LPR, grp = lane / LPR;
-    const int qw = P.n_head * HD, kw = P.n_kv_head * HD;
+    const int qw = P.n_head * HD, kw = P.n_kv_head * HD, rows_all = qw + 2 * kw;
     const int kvh = h / (P.n_head / P.n_kv_head);
     const int nsp = T.n_att_split;
     const int n_keys = pos + 1;
     const int per = (n_keys + nsp - 1) / nsp;
     const int lo = sp * per, hi = min(n_keys, lo + per);
-    float *part = T.att_part + (((size_t)i * P.n_head + h) * nsp + sp) * (HD + 2);
-    if (lo >= hi) {
-        for (int e = lane; e < HD + 2; e += 32) part[e] = e == 0 ? -INFINITY : 0.f;
-        return;
-    }
-    // one row of the q/k/v sums: elements [sub * EPL, + EPL) of the row block starting at `row0`
-    auto fetch = [&](int row0, float *out, bool rotate) {
+    float *part = T.att_part + (((size_t)i * P.n_head + h) * nsp + sp) * (HD + 4);
+    float m = -INFINITY, l = 0.f, o[EPL];
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) out[e] = ph.bias_in ? ph.bias_in[row0 + sub * EPL + e] : 0.f;
-        for (int ks = 0; ks < ph.s_in; ++ks) {
-            const float *p = ph.part_in + ((size_t)ks * TD_MAXB + i) * ph.ld_in + row0 + sub * EPL;
+    for (int e = 0; e < EPL; ++e) o[e] = 0.f;
+    if (lo < hi) {
+        const bool has_new = hi == n_keys;
+        const float *src = ph.src + (size_t)i * rows_all;
+        float q[EPL], kn[EPL], vn[EPL];
+        // all three rows are requested before any is used
 #pragma unroll
-            for (int e4 = 0; e4 < EPL / 4; ++e4) {
-                const float4 v = td_ldcg4(p + 4 * e4);
-                out[4 * e4] += v.x; out[4 * e4 + 1] += v.y; out[4 * e4 + 2] += v.z; out[4 * e4 + 3] += v.w;
+        for (int e4 = 0; e4 < EPL / 4; ++e4) {
+            const float4 a = td_ldcg4(src + h * HD + sub * EPL + 4 * e4);
+            q[4 * e4] = a.x; q[4 * e4 + 1] = a.y; q[4 * e4 + 2] = a.z; q[4 * e4 + 3] = a.w;
+            if (has_new) {
+                const float4 b = td_ldcg4(src + qw + kvh * HD + sub * EPL + 4 * e4), c = td_ldcg4(src + qw + kw + kvh * HD + sub * EPL + 4 * e4);
+                kn[4 * e4] = b.x; kn[4 * e4 + 1] = b.y; kn[4 * e4 + 2] = b.z; kn[4 * e4 + 3] = b.w;
+                vn[4 * e4] = c.x; vn[4 * e4 + 1] = c.y; vn[4 * e4 + 2] = c.z; vn[4 * e4 + 3] = c.w;
+            } else {
+                kn[4 * e4] = kn[4 * e4 + 1] = kn[4 * e4 + 2] = kn[4 * e4 + 3] = 0.f;
+                vn[4 * e4] = vn[4 * e4 + 1] = vn[4 * e4 + 2] = vn[4 * e4 + 3] = 0.f;
             }
         }
-        if (rotate) {
+        // page-table entries of the split's rows: one per lane, handed out by shuffles (a split spans at most 32 pages,
+        // which the host's choice of splits guarantees)
+        const int pg_lo = lo >> T.kv.page_shift;
+        const int my_pg = min(pg_lo + lane, T.kv.pages_per_seq - 1);
+        const int my_entry = T.kv.page_table[((size_t)slot * T.kv.n_layers_local + ph.layer_local) * T.kv.pages_per_seq + my_pg];
+        if (P.rope) {
             // split-halves pairing: element e pairs with e + HD/2, which another lane of the row holds
 #pragma unroll
             for (int e = 0; e < EPL; ++e) {
                 const int idx = sub * EPL + e, ir = idx & (HD / 2 - 1);
                 const float c = P.rope_cos[(size_t)pos * (HD / 2) + ir], s = P.rope_sin[(size_t)pos * (HD / 2) + ir];
-                const float oth = __shfl_xor_sync(0xffffffffu, out[e], LPR / 2);
-                out[e] = idx < HD / 2 ? out[e] * c - oth * s : out[e] * c + oth * s;
+                const float oq = __shfl_xor_sync(0xffffffffu, q[e], LPR / 2), ok = __shfl_xor_sync(0xffffffffu, kn[e], LPR / 2);
+                q[e] = idx < HD / 2 ? q[e] * c - oq * s : q[e] * c + oq * s;
+                kn[e] = idx < HD / 2 ? kn[e] * c - ok * s : kn[e] * c + ok * s;
             }
         }
-    };
-    float q[EPL];
-    fetch(h * HD, q, P.rope != 0);
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) q[e] *= P.scale;
-    const bool has_new = hi == n_keys;
-    float kn[EPL], vn[EPL];
-    if (has_new) {
-        fetch(qw + kvh * HD, kn, P.rope != 0);
-        fetch(qw + kw + kvh * HD, vn, false);
-        if (h % (P.n_head / P.n_kv_head) == 0 && grp == 0) {
-            KT *kp = kv_addr<KT>(T.kv, slot, ph.layer_local, 0, kvh, pos, sub * EPL);
+        for (int e = 0; e < EPL; ++e) q[e] *= P.scale;
+        auto row_ptr = [&](int row) -> const KT * {
+            const int entry = __shfl_sync(0xffffffffu, my_entry, (row >> T.kv.page_shift) - pg_lo);
+            return reinterpret_cast<const KT *>(T.kv.pool) + (size_t)entry * T.kv.page_elems +
+                   ((size_t)kvh * T.kv.page_tokens + (row & (T.kv.page_tokens - 1))) * HD + sub * EPL;
+        };
+        if (has_new && h % (P.n_head / P.n_kv_head) == 0) {
+            KT *kp = const_cast<KT *>(row_ptr(pos));
             KT *vp = kp + (size_t)T.kv.n_kv_head * T.kv.page_tokens * HD;
+            if (grp == 0) {
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) { kv_store<KT>(kp + e, kn[e]); kv_store<KT>(vp + e, vn[e]); }
+                for (int e = 0; e < EPL; ++e) { kv_store<KT>(kp + e, kn[e]); kv_store<KT>(vp + e, vn[e]); }
+            }
         }
-    }
-    const int hi_old = has_new ? hi - 1 : hi;
-    float m = -INFINITY, l = 0.f, o[EPL];
+        const int hi_old = has_new ? hi - 1 : hi;
+        auto fold = [&](float s, const float *vf) {
+            const float mn = fmaxf(m, s), corr = expf(m - mn), pr = expf(s - mn);
+            l = l * corr + pr;
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) o[e] = 0.f;
-    auto fold = [&](float s, const float *vf) {
-        const float mn = fmaxf(m, s), corr = expf(m - mn), pr = expf(s - mn);
-        l = l * corr + pr;
+            for (int e = 0; e < EPL; ++e) o[e] = o[e] * corr + pr * vf[e];
+            m = mn;
+        };
+        for (int j0 = lo; j0 < hi_old; j0 += RPW * U) {
+            uint4 kk[U], vv[U];
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) o[e] = o[e] * corr + pr * vf[e];
-        m = mn;
-    };
-    for (int j0 = lo; j0 < hi_old; j0 += RPW * U) {
-        uint4 kk[U], vv[U];
+            for (int u = 0; u < U; ++u) {
+                const int jr = j0 + u * RPW + grp;
+                const KT *kp = row_ptr(jr < hi_old ? jr : lo);
+                const KT *vp = kp + (size_t)T.kv.n_kv_head * T.kv.page_tokens * HD;
+                kk[u] = __ldcg(reinterpret_cast<const uint4 *>(kp));
+                vv[u] = __ldcg(reinterpret_cast<const uint4 *>(vp));
+            }
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int jr = j0 + u * RPW + grp;
-            const KT *kp = kv_addr<KT>(T.kv, slot, ph.layer_local, 0, kvh, jr < hi_old ? jr : lo, sub * EPL);
-            const KT *vp = kp + (size_t)T.kv.n_kv_head * T.kv.page_tokens * HD;
-            kk[u] = __ldcg(reinterpret_cast<const uint4 *>(kp));
-            vv[u] = __ldcg(reinterpret_cast<const uint4 *>(vp));
+            for (int u = 0; u < U; ++u) {
+                float kf[EPL], vf[EPL];
+                kv_unpack<KT>(kk[u], kf);
+                kv_unpack<KT>(vv[u], vf);
+                float s = 0.f;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) s = fmaf(q[e], kf[e], s);
+#pragma unroll
+                for (int w = LPR / 2; w > 0; w >>= 1) s += __shfl_xor_sync(0xffffffffu, s, w);
+                if (j0 + u * RPW + grp < hi_old) fold(s, vf);
+            }
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            float kf[EPL], vf[EPL];
-            kv_unpack<KT>(kk[u], kf);
-            kv_unpack<KT>(vv[u], vf);
+        if (has_new) {
             float s = 0.f;
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) s = fmaf(q[e], kf[e], s);
+            for (int e = 0; e < EPL; ++e) s = fmaf(q[e], kn[e], s);
 #pragma unroll
             for (int w = LPR / 2; w > 0; w >>= 1) s += __shfl_xor_sync(0xffffffffu, s, w);
-            if (j0 + u * RPW + grp < hi_old) fold(s, vf);
+            if (grp == 0) fold(s, vn);
+        }
+        // merge the row groups of the warp
+#pragma unroll
+        for (int w = LPR; w < 32; w <<= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, m, w), l2 = __shfl_xor_sync(0xffffffffu, l, w);
+            const float mn = fmaxf(m, m2);
+            const float c1 = m == -INFINITY ? 0.f : expf(m - mn), c2 = m2 == -INFINITY ? 0.f : expf(m2 - mn);
+            l = l * c1 + l2 * c2;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) o[e] = o[e] * c1 + __shfl_xor_sync(0xffffffffu, o[e], w) * c2;
+            m = mn;
         }
     }
-    if (has_new) {
-        float s = 0.f;
+    float *out = T.att_out + (size_t)i * qw + h * HD;
+    if (nsp == 1) {
+        if (grp == 0) {
+            const float inv = 1.f / l;
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) s = fmaf(q[e], kn[e], s);
-#pragma unroll
-        for (int w = LPR / 2; w > 0; w >>= 1) s += __shfl_xor_sync(0xffffffffu, s, w);
-        if (grp == 0) fold(s, vn);
-    }
-    // merge the row groups of the warp
-#pragma unroll
-    for (int w = LPR; w < 32; w <<= 1) {
-        const float m2 = __shfl_xor_sync(0xffffffffu, m, w), l2 = __shfl_xor_sync(0xffffffffu, l, w);
-        const float mn = fmaxf(m, m2);
-        const float c1 = m == -INFINITY ? 0.f : expf(m - mn), c2 = m2 == -INFINITY ? 0.f : expf(m2 - mn);
-        l = l * c1 + l2 * c2;
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) o[e] = o[e] * c1 + __shfl_xor_sync(0xffffffffu, o[e], w) * c2;
-        m = mn;
+            for (int e = 0; e < EPL; ++e) out[sub * EPL + e] = o[e] * inv;
+        }
+        return;
     }
     if (grp == 0) {
         if (sub == 0) { part[0] = m; part[1] = l; }
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) part[2 + sub * EPL + e] = o[e];
+        for (int e = 0; e < EPL; ++e) part[4 + sub * EPL + e] = o[e];
+    }
+    __threadfence();
+    __syncwarp();
+    int last = 0;
+    if (lane == 0) {
+        int *tk = T.att_ticket + i * P.n_head + h;
+        last = atomicAdd(tk, 1) == nsp - 1;
+        if (last) *tk = 0;
+    }
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (!last) return;
+    __threadfence();
+    // every lane reads all split headers, then its four output elements of every split (HD <= 128: lanes 0 .. HD/4-1)
+    const float *pb = T.att_part + ((size_t)i * P.n_head + h) * nsp * (HD + 4);
+    float ms[TD_MAX_SPLITS], ls[TD_MAX_SPLITS];
+    float4 os[TD_MAX_SPLITS];
+    const bool act = 4 * lane < HD;
+#pragma unroll
+    for (int s2 = 0; s2 < TD_MAX_SPLITS; ++s2) {
+        if (s2 < nsp) {
+            const float2 hdr = __ldcg(reinterpret_cast<const float2 *>(pb + (size_t)s2 * (HD + 4)));
+            ms[s2] = hdr.x; ls[s2] = hdr.y;
+            os[s2] = act ? td_ldcg4(pb + (size_t)s2 * (HD + 4) + 4 + 4 * lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+        } else { ms[s2] = -INFINITY; ls[s2] = 0.f; os[s2] = make_float4(0.f, 0.f, 0.f, 0.f); }
+    }
+    float M = -INFINITY;
+#pragma unroll
+    for (int s2 = 0; s2 < TD_MAX_SPLITS; ++s2) M = fmaxf(M, ms[s2]);
+    float Ls = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int s2 = 0; s2 < TD_MAX_SPLITS; ++s2) {
+        const float w = ms[s2] == -INFINITY ? 0.f : expf(ms[s2] - M);
+        Ls += ls[s2] * w;
+        acc.x += os[s2].x * w; acc.y += os[s2].y * w; acc.z += os[s2].z * w; acc.w += os[s2].w * w;
+    }
+    if (act) {
+        const float inv = 1.f / Ls;
+        *reinterpret_cast<float4 *>(out + 4 * lane) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
     }
 }
 
@@ -296,8 +360,7 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
     unsigned char *Bsm = smem + L.b;
     float *stats = reinterpret_cast<float *>(smem + L.stats);   // [TD_MAXB][2]: mean, 1/std
     float *red = reinterpret_cast<float *>(smem + L.red);       // [TD_CWARPS][TD_MAXB][2]
-    float *best_v = reinterpret_cast<float *>(smem + L.best_v); // [TD_CWARPS][TD_MAXB]
-    int *best_i = reinterpret_cast<int *>(smem + L.best_i);
+    volatile int *s_flag = reinterpret_cast<volatile int *>(smem + L.s_flag);
     int *s_dead = reinterpret_cast<int *>(smem + L.s_dead);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L.tmem_slot);
@@ -401,7 +464,7 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
             td_bar();
             if (*(volatile int *)s_dead) dead = true;
         };
-        // ring and accumulator cursors (kept by the MMA thread and, for the accumulators, by the reading warps)
+        // ring cursor (kept by the MMA thread) and accumulator count (the same in every thread)
         int stage = 0;
         uint32_t spar = 0;
         unsigned acc_cnt = 0;
@@ -429,19 +492,15 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
 #pragma unroll
             for (int i = 0; i < TD_MAXB; ++i) pos[i] = __ldcg(T.pos + slots[i]) + (int)r;
             const float *ring_in = T.is_first ? nullptr : T.ring_in + (size_t)j * P.gmax * d;
+            float *ring_out = T.is_last ? nullptr : T.ring_out + (size_t)j * P.gmax * d;
 
-            // value of the residual stream entering phase ph at (sample i, columns 4*c4..): source + partial sums + bias
+            // residual stream entering a normalising phase at (sample i, columns 4*c4..)
             auto x_in4 = [&](const TdPhase &ph, int i, int c4) -> float4 {
-                float4 x;
-                if (ph.first_of_step) {
-                    if (T.is_first) {
-                        const int tok = min(max(__ldcg(P.cur_tok + slots[i]), 0), P.vocab - 1);
-                        x = td_bf16x4(reinterpret_cast<const __nv_bfloat16 *>(P.wte) + (size_t)tok * d + 4 * c4);
-                        if (P.wpe) x = td_add4(x, td_bf16x4(reinterpret_cast<const __nv_bfloat16 *>(P.wpe) + (size_t)pos[i] * d + 4 * c4));
-                    } else x = td_ldcg4(ring_in + (size_t)i * d + 4 * c4);
-                } else x = td_ldcg4(ph.src + (size_t)i * d + 4 * c4);
-                for (int ks = 0; ks < ph.s_in; ++ks) x = td_add4(x, td_ldcg4(ph.part_in + ((size_t)ks * TD_MAXB + i) * ph.ld_in + 4 * c4));
-                if (ph.bias_in) x = td_add4(x, *reinterpret_cast<const float4 *>(ph.bias_in + 4 * c4));
+                if (!ph.first_of_step) return td_ldcg4(ph.src + (size_t)i * d + 4 * c4);
+                if (!T.is_first) return td_ldcg4(ring_in + (size_t)i * d + 4 * c4);
+                const int tok = min(max(__ldcg(P.cur_tok + slots[i]), 0), P.vocab - 1);
+                float4 x = td_bf16x4(reinterpret_cast<const __nv_bfloat16 *>(P.wte) + (size_t)tok * d + 4 * c4);
+                if (P.wpe) x = td_add4(x, td_bf16x4(reinterpret_cast<const __nv_bfloat16 *>(P.wpe) + (size_t)pos[i] * d + 4 * c4));
                 return x;
             };
 
@@ -462,116 +521,99 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
                     lap(3);
                     continue;
                 }
-                if (ph.kind == TD_FIN) {
-                    // ---------------- the partition's output: completed residual stream into the ring slot
-                    float *ring_out = T.ring_out + (size_t)j * P.gmax * d;
-                    const int n4 = nb * (d >> 2);
-                    for (int e = cta * TD_CTHREADS + ct; e < n4; e += T.n_cta * TD_CTHREADS) {
-                        const int i = e / (d >> 2), c4 = e - i * (d >> 2);
-                        *reinterpret_cast<float4 *>(ring_out + (size_t)i * d + 4 * c4) = x_in4(ph, i, c4);
-                    }
-                    lap(1);
-                    team_barrier();
-                    lap(3);
-                    continue;
-                }
                 // ---------------- contraction phase
                 const int u0 = (int)((long)cta * ph.n_units / T.n_cta), u1 = (int)((long)(cta + 1) * ph.n_units / T.n_cta);
-                // Residual stream of a normalising phase: every block of the team adds up its columns' share of the completed
-                // stream (so that the copy in ph.dst is whole whether or not the block has units) and, if it has units, the
-                // moments of every sample's row.
-                if (ph.pro == TDP_NORM && (u0 < u1 || ph.dst)) {
+                const bool keep_embedding = ph.pro == TDP_NORM && ph.first_of_step && T.is_first; // the first block's residual input
+                if (ph.pro == TDP_NORM && (u0 < u1 || keep_embedding)) {
+                    // moments of every sample's row (blocks with units); a copy of the embedded tokens, every block its columns
                     float s1[TD_MAXB], s2[TD_MAXB];
 #pragma unroll
                     for (int i = 0; i < TD_MAXB; ++i) s1[i] = s2[i] = 0.f;
                     const int n4 = d >> 2, w_lo = (int)((long)cta * n4 / T.n_cta), w_hi = (int)((long)(cta + 1) * n4 / T.n_cta);
-                    // (a block without units only needs its own columns)
-                    for (int c4 = (u0 < u1 ? 0 : w_lo) + ct; c4 < (u0 < u1 ? n4 : w_hi); c4 += TD_CTHREADS) {
+                    const int c_beg = u0 < u1 ? 0 : w_lo, c_end = u0 < u1 ? n4 : w_hi;
+                    for (int c4 = c_beg + ct; c4 < c_end; c4 += 2 * TD_CTHREADS) {
+                        float4 xa[TD_MAXB], xb[TD_MAXB];
+                        const bool two = c4 + TD_CTHREADS < c_end;
 #pragma unroll
                         for (int i = 0; i < TD_MAXB; ++i) {
-                            if (i >= nb) break;
-                            const float4 x = x_in4(ph, i, c4);
-                            if (ph.dst && c4 >= w_lo && c4 < w_hi) *reinterpret_cast<float4 *>(ph.dst + (size_t)i * d + 4 * c4) = x;
-                            s1[i] += (x.x + x.y) + (x.z + x.w);
-                            s2[i] += (x.x * x.x + x.y * x.y) + (x.z * x.z + x.w * x.w);
+                            xa[i] = i < nb ? x_in4(ph, i, c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                            xb[i] = (i < nb && two) ? x_in4(ph, i, c4 + TD_CTHREADS) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int i = 0; i < TD_MAXB; ++i) {
+                            if (i < nb) {
+                                if (keep_embedding && c4 >= w_lo && c4 < w_hi) *reinterpret_cast<float4 *>(ph.dst + (size_t)i * d + 4 * c4) = xa[i];
+                                if (keep_embedding && two && c4 + TD_CTHREADS >= w_lo && c4 + TD_CTHREADS < w_hi)
+                                    *reinterpret_cast<float4 *>(ph.dst + (size_t)i * d + 4 * (c4 + TD_CTHREADS)) = xb[i];
+                                s1[i] += ((xa[i].x + xa[i].y) + (xa[i].z + xa[i].w)) + ((xb[i].x + xb[i].y) + (xb[i].z + xb[i].w));
+                                s2[i] += ((xa[i].x * xa[i].x + xa[i].y * xa[i].y) + (xa[i].z * xa[i].z + xa[i].w * xa[i].w)) +
+                                         ((xb[i].x * xb[i].x + xb[i].y * xb[i].y) + (xb[i].z * xb[i].z + xb[i].w * xb[i].w));
+                            }
                         }
                     }
+                    if (u0 < u1) {
 #pragma unroll
-                    for (int i = 0; i < TD_MAXB; ++i) {
-                        s1[i] = warp_sum(s1[i]);
-                        s2[i] = warp_sum(s2[i]);
-                        if (lane == 0) { red[((warp - 1) * TD_MAXB + i) * 2] = s1[i]; red[((warp - 1) * TD_MAXB + i) * 2 + 1] = s2[i]; }
+                        for (int i = 0; i < TD_MAXB; ++i) {
+                            s1[i] = warp_sum(s1[i]);
+                            s2[i] = warp_sum(s2[i]);
+                            if (lane == 0) { red[((warp - 1) * TD_MAXB + i) * 2] = s1[i]; red[((warp - 1) * TD_MAXB + i) * 2 + 1] = s2[i]; }
+                        }
+                        td_bar();
+                        if (ct < TD_MAXB) {
+                            float a = 0.f, b = 0.f;
+                            for (int w = 0; w < TD_CWARPS; ++w) { a += red[(w * TD_MAXB + ct) * 2]; b += red[(w * TD_MAXB + ct) * 2 + 1]; }
+                            const float mean = P.norm == NORM_LAYER ? a / (float)d : 0.f;
+                            stats[2 * ct] = mean;
+                            stats[2 * ct + 1] = rsqrtf(fmaxf(b / (float)d - mean * mean, 0.f) + P.eps);
+                        }
+                        td_bar();
                     }
-                    td_bar();
-                    if (ct < TD_MAXB) {
-                        float a = 0.f, b = 0.f;
-                        for (int w = 0; w < TD_CWARPS; ++w) { a += red[(w * TD_MAXB + ct) * 2]; b += red[(w * TD_MAXB + ct) * 2 + 1]; }
-                        const float mean = P.norm == NORM_LAYER ? a / (float)d : 0.f;
-                        stats[2 * ct] = mean;
-                        stats[2 * ct + 1] = rsqrtf(fmaxf(b / (float)d - mean * mean, 0.f) + P.eps);
-                    }
-                    td_bar();
                 }
                 for (int ub = u0; ub < u1;) {
                     const TdUnit first = td_unit(ph, ub);
                     int ue = ub + 1; // units [ub, ue) share the k range
                     while (ue < u1 && td_unit(ph, ue).ks == first.ks) ++ue;
                     const int c_lo = first.kb_lo * TG_BK, c_hi = min(ph.K, first.kb_hi * TG_BK);
-                    // ---- prologue: this block's range of the B operand
-                    if (ph.pro == TDP_NORM) {
-                        const int n4r = (c_hi - c_lo) >> 2;
-                        for (int e = ct; e < n4r * nb; e += TD_CTHREADS) {
-                            const int i = e / n4r, c4 = (c_lo >> 2) + (e - i * n4r);
-                            float4 x = x_in4(ph, i, c4);
-                            const float mean = stats[2 * i], rstd = stats[2 * i + 1];
-                            const float4 g = *reinterpret_cast<const float4 *>(ph.gamma + 4 * c4);
-                            x.x = (x.x - mean) * rstd * g.x; x.y = (x.y - mean) * rstd * g.y; x.z = (x.z - mean) * rstd * g.z; x.w = (x.w - mean) * rstd * g.w;
-                            if (ph.beta) x = td_add4(x, *reinterpret_cast<const float4 *>(ph.beta + 4 * c4));
-                            td_b_store4(Bsm, i, 4 * c4 - c_lo, x);
-                        }
-                    } else if (ph.pro == TDP_MERGE) {
-                        // attention output of the heads in [c_lo, c_hi): merge of the sequence splits, a warp per (sample, head)
-                        const int hd = P.head_dim, h_lo = c_lo / hd, h_hi = (c_hi + hd - 1) / hd, nsp = T.n_att_split;
-                        for (int e = warp - 1; e < nb * (h_hi - h_lo); e += TD_CWARPS) {
-                            const int i = e / (h_hi - h_lo), h = h_lo + e % (h_hi - h_lo);
-                            const float *pb = T.att_part + ((size_t)i * P.n_head + h) * nsp * (hd + 2);
-                            float M = -INFINITY;
-                            for (int s2 = 0; s2 < nsp; ++s2) M = fmaxf(M, __ldcg(pb + (size_t)s2 * (hd + 2)));
-                            float Lsum = 0.f;
-                            float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-                            const int e4 = lane; // four elements per lane: head_dim <= 128
-                            for (int s2 = 0; s2 < nsp; ++s2) {
-                                const float ms = __ldcg(pb + (size_t)s2 * (hd + 2));
-                                if (ms == -INFINITY) continue;
-                                const float w = expf(ms - M);
-                                Lsum += __ldcg(pb + (size_t)s2 * (hd + 2) + 1) * w;
-                                if (4 * e4 < hd) {
-                                    const float *po = pb + (size_t)s2 * (hd + 2) + 2 + 4 * e4; // 8-byte aligned only
-                                    const float2 a = __ldcg(reinterpret_cast<const float2 *>(po)), b2 = __ldcg(reinterpret_cast<const float2 *>(po + 2));
-                                    o.x += a.x * w; o.y += a.y * w; o.z += b2.x * w; o.w += b2.y * w;
+                    // ---- prologue: this block's range of the B operand, eight independent loads in flight per thread
+                    {
+                        const int n4r = (c_hi - c_lo) >> 2, tot = n4r * nb;
+                        constexpr int PB = 8;
+                        const bool swiglu = ph.pro == TDP_ACT && ph.n_mat == 1 && P.act == 2;
+                        const float *src2 = ph.src + (size_t)TD_MAXB * ph.K; // ACT with SwiGLU: the "up" rows follow the "gate" rows
+                        for (int e0 = ct; e0 < tot; e0 += PB * TD_CTHREADS) {
+                            float4 xv[PB], yv[PB];
+                            int ii[PB], cc[PB];
+#pragma unroll
+                            for (int u = 0; u < PB; ++u) {
+                                const int e = e0 + u * TD_CTHREADS;
+                                ii[u] = e / n4r;
+                                cc[u] = (c_lo >> 2) + (e - ii[u] * n4r);
+                                if (e < tot) {
+                                    if (ph.pro == TDP_NORM) {
+                                        xv[u] = x_in4(ph, ii[u], cc[u]);
+                                        yv[u] = *reinterpret_cast<const float4 *>(ph.gamma + 4 * cc[u]);
+                                    } else {
+                                        xv[u] = td_ldcg4(ph.src + (size_t)ii[u] * ph.K + 4 * cc[u]);
+                                        if (swiglu) yv[u] = td_ldcg4(src2 + (size_t)ii[u] * ph.K + 4 * cc[u]);
+                                    }
                                 }
                             }
-                            const int c = h * hd + 4 * e4;
-                            if (4 * e4 < hd && c >= c_lo && c < c_hi) {
-                                const float inv = 1.f / Lsum;
-                                td_b_store4(Bsm, i, c - c_lo, make_float4(o.x * inv, o.y * inv, o.z * inv, o.w * inv));
+#pragma unroll
+                            for (int u = 0; u < PB; ++u) {
+                                const int e = e0 + u * TD_CTHREADS;
+                                if (e >= tot) break;
+                                float4 x = xv[u];
+                                if (ph.pro == TDP_NORM) {
+                                    const float mean = stats[2 * ii[u]], rstd = stats[2 * ii[u] + 1];
+                                    x.x = (x.x - mean) * rstd * yv[u].x; x.y = (x.y - mean) * rstd * yv[u].y;
+                                    x.z = (x.z - mean) * rstd * yv[u].z; x.w = (x.w - mean) * rstd * yv[u].w;
+                                    if (ph.beta) x = td_add4(x, *reinterpret_cast<const float4 *>(ph.beta + 4 * cc[u]));
+                                } else if (ph.pro == TDP_ACT) {
+                                    if (swiglu) x = make_float4(pk_silu(x.x) * yv[u].x, pk_silu(x.y) * yv[u].y, pk_silu(x.z) * yv[u].z, pk_silu(x.w) * yv[u].w);
+                                    else x = make_float4(pk_act(x.x, P.act), pk_act(x.y, P.act), pk_act(x.z, P.act), pk_act(x.w, P.act));
+                                }
+                                td_b_store4(Bsm, ii[u], 4 * cc[u] - c_lo, x);
                             }
-                        }
-                    } else { // TDP_ACT: activation of the hidden units in [c_lo, c_hi)
-                        const int n4r = (c_hi - c_lo) >> 2;
-                        const bool swiglu = P.act == 2;
-                        for (int e = ct; e < n4r * nb; e += TD_CTHREADS) {
-                            const int i = e / n4r, c4 = (c_lo >> 2) + (e - i * n4r);
-                            float4 a = ph.bias_in ? *reinterpret_cast<const float4 *>(ph.bias_in + 4 * c4) : make_float4(0.f, 0.f, 0.f, 0.f);
-                            for (int ks = 0; ks < ph.s_in; ++ks) a = td_add4(a, td_ldcg4(ph.part_in + ((size_t)ks * TD_MAXB + i) * ph.ld_in + 4 * c4));
-                            float4 y;
-                            if (swiglu) {
-                                float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-                                const float *up = ph.part_in + (size_t)ph.s_in * TD_MAXB * ph.ld_in;
-                                for (int ks = 0; ks < ph.s_in; ++ks) b = td_add4(b, td_ldcg4(up + ((size_t)ks * TD_MAXB + i) * ph.ld_in + 4 * c4));
-                                y = make_float4(pk_silu(a.x) * b.x, pk_silu(a.y) * b.y, pk_silu(a.z) * b.z, pk_silu(a.w) * b.w);
-                            } else y = make_float4(pk_act(a.x, P.act), pk_act(a.y, P.act), pk_act(a.z, P.act), pk_act(a.w, P.act));
-                            td_b_store4(Bsm, i, 4 * c4 - c_lo, y);
                         }
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -619,11 +661,72 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
                             __syncwarp();
                             if (lane == 0) mbar_arrive(acce0 + 8 * a, 1u);
                             const int row = un.tile * TG_BM + lane_base + lane;
-                            if (row < ph.n_rows && !dead) {
-                                float *dst = ph.out + ((size_t)(un.mat * ph.n_split + un.ks) * TD_MAXB) * ph.n_rows + row;
+                            const bool rv = row < ph.n_rows;
+                            float val[TD_MAXB];
 #pragma unroll
-                                for (int i = 0; i < TD_MAXB; ++i)
-                                    if (i < nb) dst[(size_t)i * ph.n_rows] = __uint_as_float(rr[i]) + __uint_as_float(rr[i + 8]);
+                            for (int i = 0; i < TD_MAXB; ++i) val[i] = __uint_as_float(rr[i]) + __uint_as_float(rr[i + 8]);
+                            bool finish = true;
+                            if (ph.n_split > 1) {
+                                // leave the partial sum, take a ticket of the row tile; whoever takes the last one adds them all up
+                                float *pp = ph.part + ((size_t)(un.mat * ph.n_split + un.ks) * TD_MAXB) * ph.n_rows + row;
+                                if (rv) {
+#pragma unroll
+                                    for (int i = 0; i < TD_MAXB; ++i)
+                                        if (i < nb) pp[(size_t)i * ph.n_rows] = val[i];
+                                }
+                                __threadfence();
+                                td_epi_bar();
+                                if (warp == 4 && lane == 0) {
+                                    int *tk = ph.ticket + un.mat * ph.n_tiles + un.tile;
+                                    const int lastone = atomicAdd(tk, 1) == ph.n_split - 1;
+                                    if (lastone) *tk = 0;
+                                    *s_flag = lastone;
+                                }
+                                td_epi_bar();
+                                finish = *s_flag != 0;
+                                if (finish && rv) {
+                                    __threadfence();
+                                    const float *p0 = ph.part + ((size_t)(un.mat * ph.n_split) * TD_MAXB) * ph.n_rows + row;
+#pragma unroll
+                                    for (int i = 0; i < TD_MAXB; ++i) val[i] = 0.f;
+                                    for (int ks = 0; ks < ph.n_split; ++ks) {
+#pragma unroll
+                                        for (int i = 0; i < TD_MAXB; ++i)
+                                            if (i < nb) val[i] += __ldcg(p0 + ((size_t)ks * TD_MAXB + i) * ph.n_rows);
+                                    }
+                                }
+                            }
+                            if (finish && ph.kind != TD_HEAD) {
+                                if (rv && !dead) {
+                                    const float b = ph.fin_bias ? ph.fin_bias[row] : 0.f;
+                                    const float *resid = ph.fin_resid_ring ? ring_in : ph.fin_resid;
+                                    float *dst = ph.fin_ring ? ring_out : ph.fin + (size_t)un.mat * TD_MAXB * ph.n_rows;
+                                    float rs[TD_MAXB];
+#pragma unroll
+                                    for (int i = 0; i < TD_MAXB; ++i) rs[i] = (resid && i < nb) ? __ldcg(resid + (size_t)i * ph.n_rows + row) : 0.f;
+#pragma unroll
+                                    for (int i = 0; i < TD_MAXB; ++i)
+                                        if (i < nb) dst[(size_t)i * ph.n_rows + row] = val[i] + b + rs[i];
+                                }
+                            } else if (finish) {
+                                // output layer: logits by slot, and this warp's best (value, row) per sample
+#pragma unroll
+                                for (int i = 0; i < TD_MAXB; ++i) {
+                                    if (i >= nb) break;
+                                    float bv = rv ? val[i] : -INFINITY;
+                                    int bi = rv ? row : 0x7fffffff;
+                                    if (rv && !dead) P.logits[(size_t)slots[i] * ph.n_rows + row] = val[i];
+#pragma unroll
+                                    for (int o = 16; o > 0; o >>= 1) {
+                                        const float v2 = __shfl_xor_sync(0xffffffffu, bv, o);
+                                        const int i2 = __shfl_xor_sync(0xffffffffu, bi, o);
+                                        if (v2 > bv || (v2 == bv && i2 < bi)) { bv = v2; bi = i2; }
+                                    }
+                                    if (lane == 0) {
+                                        T.head_pv[(size_t)i * 4 * ph.n_tiles + un.tile * 4 + (warp & 3)] = bv;
+                                        T.head_pi[(size_t)i * 4 * ph.n_tiles + un.tile * 4 + (warp & 3)] = bi;
+                                    }
+                                }
                             }
                         }
                         if (dead) *s_dead = 1;
@@ -634,79 +737,36 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
                     ub = ue;
                 }
                 lap(2);
-                if (ph.kind == TD_HEAD) {
-                    team_barrier();
-                    lap(3);
-                    // ---- logits = sum of the partial sums, per-block argmax over a slice of the vocabulary
-                    const int V = P.vocab, v_lo = (int)((long)cta * V / T.n_cta), v_hi = (int)((long)(cta + 1) * V / T.n_cta);
-                    float bv[TD_MAXB];
-                    int bi[TD_MAXB];
-#pragma unroll
-                    for (int i = 0; i < TD_MAXB; ++i) { bv[i] = -INFINITY; bi[i] = 0x7fffffff; }
-                    for (int vv = v_lo + ct; vv < v_hi; vv += TD_CTHREADS) {
-#pragma unroll
-                        for (int i = 0; i < TD_MAXB; ++i) {
-                            if (i >= nb) break;
-                            float y = 0.f;
-                            for (int ks = 0; ks < ph.n_split; ++ks) y += __ldcg(ph.out + ((size_t)ks * TD_MAXB + i) * V + vv);
-                            P.logits[(size_t)slots[i] * V + vv] = y;
-                            if (y > bv[i] || (y == bv[i] && vv < bi[i])) { bv[i] = y; bi[i] = vv; }
-                        }
-                    }
-#pragma unroll
-                    for (int i = 0; i < TD_MAXB; ++i) {
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) {
-                            const float v2 = __shfl_xor_sync(0xffffffffu, bv[i], o);
-                            const int i2 = __shfl_xor_sync(0xffffffffu, bi[i], o);
-                            if (v2 > bv[i] || (v2 == bv[i] && i2 < bi[i])) { bv[i] = v2; bi[i] = i2; }
-                        }
-                        if (lane == 0) { best_v[(warp - 1) * TD_MAXB + i] = bv[i]; best_i[(warp - 1) * TD_MAXB + i] = bi[i]; }
-                    }
-                    td_bar();
-                    if (ct < nb) {
-                        float b = best_v[ct];
-                        int bi2 = best_i[ct];
-                        for (int w = 1; w < TD_CWARPS; ++w) {
-                            const float v2 = best_v[w * TD_MAXB + ct];
-                            const int i2 = best_i[w * TD_MAXB + ct];
+                team_barrier();
+                lap(3);
+                if (ph.kind == TD_HEAD && cta == 0) {
+                    // ---- token choice: best candidate per sample, lowest id on ties
+                    const int n_cand = 4 * ph.n_tiles;
+                    for (int i = warp - 1; i < nb; i += TD_CWARPS) {
+                        float b = -INFINITY;
+                        int bi2 = 0x7fffffff;
+                        for (int c2 = lane; c2 < n_cand; c2 += 32) {
+                            const float v2 = __ldcg(T.head_pv + (size_t)i * n_cand + c2);
+                            const int i2 = __ldcg(T.head_pi + (size_t)i * n_cand + c2);
                             if (v2 > b || (v2 == b && i2 < bi2)) { b = v2; bi2 = i2; }
                         }
-                        P.head_pv[(size_t)ct * T.n_cta + cta] = b;
-                        P.head_pi[(size_t)ct * T.n_cta + cta] = bi2;
-                    }
-                    team_barrier();
-                    lap(3);
-                    if (cta == 0) {
-                        for (int i = warp - 1; i < nb; i += TD_CWARPS) {
-                            float b = -INFINITY;
-                            int bi2 = 0x7fffffff;
-                            for (int c2 = lane; c2 < T.n_cta; c2 += 32) {
-                                const float v2 = __ldcg(P.head_pv + (size_t)i * T.n_cta + c2);
-                                const int i2 = __ldcg(P.head_pi + (size_t)i * T.n_cta + c2);
-                                if (v2 > b || (v2 == b && i2 < bi2)) { b = v2; bi2 = i2; }
-                            }
 #pragma unroll
-                            for (int o = 16; o > 0; o >>= 1) {
-                                const float v2 = __shfl_xor_sync(0xffffffffu, b, o);
-                                const int i2 = __shfl_xor_sync(0xffffffffu, bi2, o);
-                                if (v2 > b || (v2 == b && i2 < bi2)) { b = v2; bi2 = i2; }
-                            }
-                            if (lane == 0) {
-                                const int slot = j + i * G;
-                                const int g = P.gen_count[slot];
-                                if (g < P.log_stride) P.tok_log[(size_t)slot * P.log_stride + g] = bi2;
-                                int feed = bi2;
-                                if (g < P.n_teacher[slot]) feed = P.teacher[(size_t)slot * P.log_stride + g];
-                                P.cur_tok[slot] = feed;
-                                P.gen_count[slot] = g + 1;
-                            }
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const float v2 = __shfl_xor_sync(0xffffffffu, b, o);
+                            const int i2 = __shfl_xor_sync(0xffffffffu, bi2, o);
+                            if (v2 > b || (v2 == b && i2 < bi2)) { b = v2; bi2 = i2; }
+                        }
+                        if (lane == 0) {
+                            const int slot = j + i * G;
+                            const int g = P.gen_count[slot];
+                            if (g < P.log_stride) P.tok_log[(size_t)slot * P.log_stride + g] = bi2;
+                            int feed = bi2;
+                            if (g < P.n_teacher[slot]) feed = P.teacher[(size_t)slot * P.log_stride + g];
+                            P.cur_tok[slot] = feed;
+                            P.gen_count[slot] = g + 1;
                         }
                     }
                     lap(5);
-                } else {
-                    team_barrier();
-                    lap(3);
                 }
             }
             // ---- output edge
