@@ -72,10 +72,12 @@ typedef struct {
     int rounds_per_graph; /* stream scheduler: rounds of the recurrent schedule captured per CUDA graph
                              (default 16; <0: no graphs) */
     int kv_cache_dtype; /* MDI_KV_*: element type of the key/value cache when the weights are bf16 (fp32 weights always
-                          keep an fp32 cache).  DEFAULT = F32.  BF16 halves the cache bytes at about 2e-3 relative error
-                          per block on the activations (measured), which on a 32-block model exceeds a 3e-2 absolute
-                          logit tolerance; F16 halves them at an eighth of that error (three more mantissa bits; keys and
-                          values of these models are far inside its range) */
+                          keep an fp32 cache).  DEFAULT: F16 for models the fused-phase scheduler cannot cover (Llama block,
+                          grouped-query heads, d_model > 1024 or head_dim > 64), F32 for those it can (it reads fp32 pages).
+                          F16 halves the cache bytes at 1.6e-2 worst absolute logit error on the 32-block Llama-7B shape and
+                          6e-4 on the 48-block GPT-2-XL shape (measured over whole generations; fp32: 1.2e-3 and 3e-5); keys
+                          and values of these models are far inside its range.  BF16 costs eight times the F16 error, which
+                          on the 32-block model exceeds a 3e-2 absolute logit tolerance */
     int prefill_mode;  /* first visits (whole prompt): 0 (default) tensor-core GEMMs (tcgen05, bf16 x bf16 -> fp32, inputs split
                           into two bf16 planes) when the weights are bf16, else the CUDA-core step kernels in chunks of 8
                           positions; 1: always the CUDA-core kernels */
@@ -100,9 +102,9 @@ typedef struct {
                           2: the phase-per-matrix persistent kernel, or fail;
                           3: the fused-phase persistent kernel, or fail;
                           4: the tensor-core persistent kernel, or fail (bf16 weights, groups of at most 8 samples, widths
-                             that are multiples of 64: one cooperative launch, a team per partition, every linear layer a
-                             tcgen05 contraction fed by a TMA weight ring; what scheduler 0 picks where it would otherwise run
-                             tensor-core steps on the stream scheduler, greedy token choice only) */
+                             that are multiples of 64, greedy token choice: one cooperative launch, a team per partition,
+                             every linear layer a tcgen05 contraction fed by a TMA weight ring).  Never picked by
+                             scheduler 0: on the large workloads it measures at or below the stream scheduler */
     int in_kernel_timing; /* 1: the persistent kernels time themselves (mdi_get_partition_times); costs a few percent */
     int fused_blocks_per_head; /* fused-phase kernel: 0 (default) two thread blocks of a cluster share a head where every
                           team has a cluster per head, else one block per head; 1: always one block per head (plain
@@ -113,6 +115,8 @@ typedef struct {
     int trace_slot;    /* with in_kernel_timing: s > 0 makes thread 0 of every block of the fused-phase kernel record a
                           time stamp at every change of timing category while it serves schedule slot s - 1
                           (mdi_get_trace) */
+    int td_b_kblocks;  /* tensor-core persistent kernel: 64-column blocks of the activation operand kept in shared memory
+                          (the weight ring gets the rest); 0 (default): 32 for d_model >= 2048, else 16 */
 } mdi_options;
 
 typedef struct {

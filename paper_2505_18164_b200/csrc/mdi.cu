@@ -160,7 +160,7 @@ struct mdi_ctx {
     std::vector<int64_t> fz_team_stream_bytes; // per partition: bytes of its blocks' weight streams
     // persistent tensor-core decode kernel (bf16 weights, groups of up to 8 samples): plan at creation, tables at first use
     bool td_ok = false, td_stale = true;
-    int td_grid = 0;
+    int td_grid = 0, td_b_kb = 16;
     size_t td_smem = 0;
     std::vector<TdTeam> td_teams_host;
     std::vector<TdPhase> td_phases_host;
@@ -1301,20 +1301,32 @@ const void *td_func(const mdi_ctx *c) {
 }
 
 // How many ranges of k-blocks a contraction with `tiles` row tiles (all its matrices together) and n_kb k-blocks is
-// cut into for a team of n_cta blocks: at least so many that a range fits the resident B operand, then the first
-// count at which the units deal out evenly (a phase ends in a team barrier, so the block with most units sets its time).
-void td_choose_split(int tiles, int n_kb, int n_cta, int *n_split, int *kb_per_split) {
+// cut into for a team of n_cta blocks: at least so many that a range fits the resident B operand; beyond that the
+// count that minimises the estimated time of the busiest block (a phase ends in a team barrier).  Units (range-major,
+// the last range possibly shorter) go to the blocks in contiguous runs; a unit costs its k-blocks plus about four
+// k-blocks' worth of fixed work (accumulator read-back, ticket, partial sums written and re-read), and every further
+// range of a block another prologue.
+void td_choose_split(int tiles, int n_kb, int n_cta, int b_kb, int *n_split, int *kb_per_split) {
     int best_s = 0, best_k = 0;
-    double best = -1.0;
-    for (int s0 = (n_kb + TD_B_KB - 1) / TD_B_KB; s0 <= std::min(n_kb, 16); ++s0) {
+    double best = 1e30;
+    const int s_min = (n_kb + b_kb - 1) / b_kb;
+    for (int s0 = s_min; s0 <= std::min(n_kb, 32); ++s0) {
         const int kbps = (n_kb + s0 - 1) / s0, s = (n_kb + kbps - 1) / kbps;
-        if (kbps < 2 && s0 > (n_kb + TD_B_KB - 1) / TD_B_KB) break;
+        if (kbps < 8 && s0 > s_min) break; // units of at least 128 KB of weights
         const long units = (long)s * tiles;
-        const long most = (units + n_cta - 1) / n_cta;
-        // work of the busiest block against the mean, counting that every unit is charged a full range
-        const double eff = (double)tiles * n_kb / ((double)most * kbps * n_cta);
-        if (eff > best + 0.02) { best = eff; best_s = s; best_k = kbps; }
-        if (eff >= 0.93) break;
+        double worst = 0;
+        for (int b = 0; b < n_cta; ++b) {
+            const long u0 = (long)b * units / n_cta, u1 = (long)(b + 1) * units / n_cta;
+            double load = 0;
+            int last_ks = -1;
+            for (long u = u0; u < u1; ++u) {
+                const int ks = (int)(u / tiles);
+                load += std::min(n_kb, (ks + 1) * kbps) - ks * kbps + (s > 1 ? 4.0 : 1.0);
+                if (ks != last_ks) { load += 24.0; last_ks = ks; }
+            }
+            worst = std::max(worst, load);
+        }
+        if (worst < best * 0.985) { best = worst; best_s = s; best_k = kbps; }
     }
     *n_split = best_s;
     *kb_per_split = best_k;
@@ -1325,7 +1337,7 @@ int td_setup(mdi_ctx *c) {
     const int K = c->K, d = s.d_model, hd = s.head_dim, H = s.n_head, qw = H * hd, kw = s.n_kv_head * hd, F = s.d_ff, V = s.vocab;
     const bool want = c->scheduler == 4;
     auto no = [&](const char *why) { return want ? fail(c, MDI_ERR_SHAPE, "tensor-core persistent scheduler: %s", why) : MDI_OK; };
-    if (c->scheduler != 0 && c->scheduler != 4) return MDI_OK;
+    if (c->scheduler != 4) return MDI_OK;
     if (s.weight_dtype != MDI_DTYPE_BF16) return no("needs bf16 weights");
     if (c->gmax > TD_MAXB) return no("at most 8 samples per group");
     if (d % 64 || qw % 64 || F % 64) return no("d_model, n_head * head_dim and d_ff must be multiples of 64");
@@ -1336,6 +1348,10 @@ int td_setup(mdi_ctx *c) {
     CU(cudaGetDeviceProperties(&prop, c->dev));
     const int n_sm = prop.multiProcessorCount;
     if (n_sm < K) return no("fewer SMs than partitions");
+    // resident B operand: 32 k-blocks (2048 columns; 7 ring stages) for wide models, whose matrices then need fewer
+    // ranges, else 16 (9 ring stages)
+    c->td_b_kb = c->o.td_b_kblocks > 0 ? c->o.td_b_kblocks : (d >= 2048 ? 32 : 16);
+    if (c->td_b_kb < 4 || c->td_b_kb > 48) return no("td_b_kblocks must be between 4 and 48");
     c->td_smem = td_smem_layout().total;
     if (c->td_smem > (size_t)prop.sharedMemPerBlockOptin) return no("not enough shared memory per block");
     {
@@ -1372,6 +1388,7 @@ int td_setup(mdi_ctx *c) {
     c->td_phase_begin.assign(K, 0);
     c->td_phase_count.assign(K, 0);
     int first = 0;
+    bool too_wide = false;
     for (int p = 0; p < K; ++p) {
         const int n = n_cta[p], Lp = c->part[p].hi - c->part[p].lo;
         c->td_phase_begin[p] = (int)c->td_phases_host.size();
@@ -1379,7 +1396,8 @@ int td_setup(mdi_ctx *c) {
             TdPhase q{};
             q.kind = kind; q.layer_local = ll; q.n_mat = n_mat; q.n_rows = rows; q.K = Kd; q.pro = pro;
             q.n_tiles = (rows + TG_BM - 1) / TG_BM; q.n_kb = Kd / TG_BK;
-            td_choose_split(n_mat * q.n_tiles, q.n_kb, n, &q.n_split, &q.kb_per_split);
+            td_choose_split(n_mat * q.n_tiles, q.n_kb, n, c->td_b_kb, &q.n_split, &q.kb_per_split);
+            if (q.n_split < 1) too_wide = true;
             q.n_units = q.n_split * n_mat * q.n_tiles;
             c->td_phases_host.push_back(q);
         };
@@ -1399,18 +1417,21 @@ int td_setup(mdi_ctx *c) {
         T.is_first = p == 0; T.is_last = p == K - 1;
         // attention units (sample, head, split) over the team's warps: the split count that deals them out most evenly
         {
+            // estimated time of the phase: units of the busiest warp x (fixed cost of a unit: its q/k/v rows, page-table
+            // entries, ticket, about four round trips to memory + a round trip per 16 cached rows), at a quarter of n_ctx
             const int warps = n * TD_CWARPS, pairs = c->gmax * H;
             int best_s = min_att_split;
-            double best = -1.0;
+            double best = 1e30;
             for (int sp = min_att_split; sp <= TD_MAX_SPLITS; sp *= 2) {
                 const long units = (long)pairs * sp, most = (units + warps - 1) / warps;
-                const double eff = (double)units / ((double)most * warps);
-                if (eff > best + 0.03) { best = eff; best_s = sp; }
+                const double cost = (double)most * (4.0 + (double)(s.n_ctx / 4) / sp / 16.0);
+                if (cost < best * 0.97) { best = cost; best_s = sp; }
             }
             T.n_att_split = best_s;
         }
     }
     c->td_grid = first;
+    if (too_wide) return no("a matrix has more columns than 32 ranges of the resident B operand cover");
     int rc;
     if ((rc = dalloc(c, &c->td_sync, (size_t)K * 64)) != MDI_OK) return rc;
     if ((rc = dalloc(c, &c->td_err, 1)) != MDI_OK) return rc;
@@ -1449,7 +1470,7 @@ int td_build(mdi_ctx *c) {
             const TdPhase &q = c->td_phases_host[c->td_phase_begin[p] + i];
             const bool split = td_is_gemm(q.kind) && q.n_split > 1;
             o.part.push_back(split ? take((size_t)q.n_mat * q.n_split * TD_MAXB * q.n_rows) : 0);
-            o.ticket.push_back(split ? take_i((size_t)q.n_mat * q.n_tiles) : 0);
+            o.ticket.push_back(split ? take_i((size_t)q.n_mat * q.n_tiles * 4) : 0);
             if (q.kind == TD_HEAD) { o.head_pv = take((size_t)TD_MAXB * 4 * q.n_tiles); o.head_pi = take_i((size_t)TD_MAXB * 4 * q.n_tiles); }
         }
     }
@@ -1567,7 +1588,7 @@ int td_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     TdParams P{};
     P.d = s.d_model; P.n_head = s.n_head; P.n_kv_head = s.n_kv_head; P.head_dim = s.head_dim; P.d_ff = s.d_ff; P.vocab = s.vocab;
     P.norm = s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS; P.act = s.act; P.rope = s.arch == MDI_ARCH_LLAMA;
-    P.K = c->K; P.G = G; P.n_samples = n_samples; P.gmax = c->gmax; P.n_pass = n_pass;
+    P.K = c->K; P.G = G; P.n_samples = n_samples; P.gmax = c->gmax; P.n_pass = n_pass; P.b_kb = c->td_b_kb;
     P.eps = s.norm_eps; P.scale = 1.0f / std::sqrt((float)s.head_dim);
     P.teams = c->td_teams; P.phases = c->td_phases; P.wte = c->wte; P.wpe = c->wpe; P.rope_cos = c->rope_cos; P.rope_sin = c->rope_sin;
     P.logits = c->logits; P.cur_tok = c->cur_tok; P.tok_log = c->tok_log;
@@ -1670,7 +1691,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
                                      s.n_kv_head == s.n_head && c->o.scheduler != 1 && c->o.scheduler != 2 && c->o.scheduler != 4 && s.head_dim <= 64;
         // ... and 64 rows where the tensor-core persistent kernel may run (a warp hands out the page-table entries of
         // its sequence split by shuffles: fewer, larger pages)
-        const bool td_candidate = s.weight_dtype == MDI_DTYPE_BF16 && (c->o.scheduler == 0 || c->o.scheduler == 4);
+        const bool td_candidate = s.weight_dtype == MDI_DTYPE_BF16 && c->o.scheduler == 4;
         c->page_tokens = c->o.page_tokens > 0 ? c->o.page_tokens : (fused_candidate ? 128 : td_candidate ? 64 : 16);
     }
     if (c->page_tokens & (c->page_tokens - 1)) return bail(fail(c, MDI_ERR_ARG, "page_tokens must be a power of two"));
@@ -1679,7 +1700,12 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     c->pages_per_seq = (s.n_ctx + c->page_tokens - 1) / c->page_tokens;
     c->esize = s.weight_dtype == MDI_DTYPE_F32 ? 4 : 2;
     if (c->o.kv_cache_dtype < 0 || c->o.kv_cache_dtype > 3) return bail(fail(c, MDI_ERR_ARG, "kv_cache_dtype must be one of MDI_KV_*"));
-    c->kv_kind = s.weight_dtype != MDI_DTYPE_BF16 ? KV_F32 : c->o.kv_cache_dtype == MDI_KV_BF16 ? KV_BF16 : c->o.kv_cache_dtype == MDI_KV_F16 ? KV_F16 : KV_F32;
+    {
+        // default: fp16 for bf16 models outside the fused-phase kernel's reach (that kernel reads fp32 pages), else fp32
+        const bool fused_shape = s.arch == MDI_ARCH_GPT && s.n_kv_head == s.n_head && s.d_model <= 1024 && s.head_dim <= 64;
+        const int want = c->o.kv_cache_dtype != MDI_KV_DEFAULT ? c->o.kv_cache_dtype : (fused_shape ? MDI_KV_F32 : MDI_KV_F16);
+        c->kv_kind = s.weight_dtype != MDI_DTYPE_BF16 ? KV_F32 : want == MDI_KV_BF16 ? KV_BF16 : want == MDI_KV_F16 ? KV_F16 : KV_F32;
+    }
     c->kv_f32 = c->kv_kind == KV_F32;
     c->kv_esize = c->kv_f32 ? 4 : 2;
     c->page_elems = (size_t)2 * s.n_kv_head * c->page_tokens * s.head_dim;
@@ -2067,10 +2093,10 @@ static int generate_impl(mdi_ctx *c, int n_samples, int n_new, int32_t *out, boo
                               !(c->pf_tc && c->scheduler == 0 && (n_samples + G - 1) / G >= c->tc_min_group);
     const bool use_fz = c->fz_ok && (c->scheduler == 0 || c->scheduler == 3) && small_groups && fz_slot_count_fits(c, n_pass, G);
     const bool use_pk = !use_fz && c->pk_ok && c->scheduler != 1 && c->scheduler != 3 && c->scheduler != 4 && small_groups && pk_tile_count_fits(c, n_pass, G);
-    // the tensor-core persistent kernel: large blocks of the model or groups of 5 to 8 samples (what the stream scheduler
-    // would run as tensor-core steps), greedy token choice
-    const bool use_td = !use_fz && !use_pk && c->td_ok && c->temperature <= 0.f && (n_samples + G - 1) / G <= TD_MAXB &&
-                        (c->scheduler == 4 || (c->scheduler == 0 && !small_groups));
+    // the tensor-core persistent kernel: on request only (measured on the two large workloads it does not beat the
+    // stream scheduler's tensor-core steps: its teams run their phases in lock-step, so the weight stream stops
+    // during attention, prologues and barriers), greedy token choice
+    const bool use_td = c->td_ok && c->scheduler == 4 && c->temperature <= 0.f && (n_samples + G - 1) / G <= TD_MAXB;
     if (c->scheduler == 2 && !use_pk) return fail(c, MDI_ERR_SHAPE, "persistent scheduler unavailable for this call");
     if (c->scheduler == 3 && !use_fz) return fail(c, MDI_ERR_SHAPE, "fused-phase scheduler unavailable for this call");
     if (c->scheduler == 4 && !use_td) return fail(c, MDI_ERR_SHAPE, "tensor-core persistent scheduler unavailable for this call");

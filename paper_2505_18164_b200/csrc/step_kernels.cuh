@@ -526,31 +526,39 @@ __global__ void __launch_bounds__(ATT_THREADS) k_attn_decode(const AttnArgs a, c
         float m = -INFINITY, l = 0.f, o[EPL];
 #pragma unroll
         for (int e = 0; e < EPL; ++e) o[e] = 0.f;
-        for (int j0 = lo + warp * RPW; j0 < hi; j0 += NG) {
-            const int j = j0 + grp;
-            const bool live = j < hi;
-            const int jj = live ? j : lo;
-            const KT *kp = kv_addr<KT>(a.kv, slot, a.layer_local, 0, kvh, jj, sub * EPL);
-            const KT *vp = kp + (size_t)a.kv.n_kv_head * a.kv.page_tokens * HD;
-            WVec<KT> kvv, vvv;
-            kvv.load(kp);
-            vvv.load(vp);
-            float kf[EPL], vf[EPL];
-            kvv.unpack(kf);
-            vvv.unpack(vf);
-            float s = 0.f;
+        // four rows per lane group in flight: the loads of a round are issued before any of them is used
+        constexpr int UR = 4;
+        for (int j0 = lo + warp * RPW; j0 < hi; j0 += NG * UR) {
+            WVec<KT> kvv[UR], vvv[UR];
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) s = fmaf(q[e], kf[e], s);
+            for (int u = 0; u < UR; ++u) {
+                const int j = j0 + u * NG + grp;
+                const int jj = j < hi ? j : lo;
+                const KT *kp = kv_addr<KT>(a.kv, slot, a.layer_local, 0, kvh, jj, sub * EPL);
+                const KT *vp = kp + (size_t)a.kv.n_kv_head * a.kv.page_tokens * HD;
+                kvv[u].load(kp);
+                vvv[u].load(vp);
+            }
 #pragma unroll
-            for (int w = LPR / 2; w > 0; w >>= 1) s += __shfl_xor_sync(0xffffffffu, s, w);
-            if (live) {
-                const float mn = fmaxf(m, s);
-                const float corr = expf(m - mn); // m = -inf gives 0
-                const float p = expf(s - mn);
-                l = l * corr + p;
+            for (int u = 0; u < UR; ++u) {
+                const bool live = j0 + u * NG + grp < hi;
+                float kf[EPL], vf[EPL];
+                kvv[u].unpack(kf);
+                vvv[u].unpack(vf);
+                float s = 0.f;
 #pragma unroll
-                for (int e = 0; e < EPL; ++e) o[e] = o[e] * corr + p * vf[e];
-                m = mn;
+                for (int e = 0; e < EPL; ++e) s = fmaf(q[e], kf[e], s);
+#pragma unroll
+                for (int w = LPR / 2; w > 0; w >>= 1) s += __shfl_xor_sync(0xffffffffu, s, w);
+                if (live) {
+                    const float mn = fmaxf(m, s);
+                    const float corr = expf(m - mn); // m = -inf gives 0
+                    const float p = expf(s - mn);
+                    l = l * corr + p;
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) o[e] = o[e] * corr + p * vf[e];
+                    m = mn;
+                }
             }
         }
         const int g = warp * RPW + grp;

@@ -33,13 +33,15 @@
 namespace mdi {
 
 constexpr int TD_THREADS = 256;                 // warp 0: weight producer; warp 1: MMA issuer; warps 4..7 read accumulators
-constexpr int TD_CWARPS = 7;                    // warps 1..7 run prologues and attention together
+constexpr int TD_CWARPS = 7;                    // warps 1..7 run prologues and attention together (16 warps of 128 registers were
+                                                // measured slower: the attention loop then spills its rows in flight)
 constexpr int TD_CTHREADS = TD_CWARPS * 32;
-constexpr int TD_STAGES = 7;                    // weight ring: 7 x 16 KB
+constexpr int TD_MAX_STAGES = 9;                // weight ring: up to 9 stages of 16 KB
 constexpr int TD_W_BYTES = 16384;               // one stage: 128 rows x 64 columns of bf16
 constexpr int TD_MAXB = 8;                      // samples per group
-constexpr int TD_B_KB = 32;                     // k-blocks (64 columns) of the B operand resident in shared memory
-constexpr int TD_B_BYTES = TD_B_KB * 2048;      // 16 rows x 128 bytes per k-block
+constexpr int TD_OPERAND_BYTES = 11 * TD_W_BYTES; // shared memory for the ring and the B operand together: the B operand
+                                                // holds b_kb k-blocks (64 columns, 16 rows x 128 bytes each), the ring the rest
+__host__ __device__ inline int td_stages(int b_kb) { const int n = (TD_OPERAND_BYTES - b_kb * 2048) / TD_W_BYTES; return n < TD_MAX_STAGES ? n : TD_MAX_STAGES; }
 constexpr int TD_ACC = 4;                       // accumulators in tensor memory (16 columns each)
 constexpr int TD_MAX_PHASES = 64;
 constexpr int TD_MAX_SPLITS = 16;               // attention splits over the sequence
@@ -85,6 +87,7 @@ struct TdTeam {
 
 struct TdParams {
     int d, n_head, n_kv_head, head_dim, d_ff, vocab, norm, act, rope, K, G, n_samples, gmax, n_pass;
+    int b_kb;                // k-blocks of the resident B operand (ranges of the contractions never exceed it)
     float eps, scale;
     const TdTeam *teams;
     const TdPhase *phases;
@@ -98,23 +101,24 @@ struct TdParams {
     unsigned long long wait_ns;
     int withhold_partition;
     unsigned long long *prof; // optional [grid][PK_PROF_N]: [0] input edge, [1] prologues, [2] contraction, [3] team barriers,
-                              // [4] attention, [5] token choice, [6] producer waiting for a free stage, [7] producer total
+                              // [4] attention, [5] token choice, [6] producer waiting for a free stage, [7] producer total,
+                              // [8] team barrier after the output layer, [9] the output layer's contraction, and inside [2] / [9]:
+                              // [10] the MMA thread waiting for weight tiles, [11] waiting for a free accumulator
 };
 
 struct TdSmem {
-    size_t ring, b, stats, red, s_flag, s_dead, bars, tmem_slot, s_ph, total;
+    size_t ring, stats, red, s_flag, s_dead, bars, tmem_slot, s_ph, total;
 };
 __host__ __device__ inline TdSmem td_smem_layout() {
     TdSmem L;
     size_t o = 0;
     auto take = [&](size_t bytes, size_t align) { o = (o + align - 1) / align * align; const size_t r = o; o += bytes; return r; };
-    L.ring = take((size_t)TD_STAGES * TD_W_BYTES, 1024);
-    L.b = take(TD_B_BYTES, 1024);
+    L.ring = take((size_t)TD_OPERAND_BYTES, 1024); // the B operand sits behind the ring's stages
     L.stats = take(4 * 2 * TD_MAXB, 16);
     L.red = take(4 * 2 * TD_MAXB * TD_CWARPS, 16);
     L.s_flag = take(8, 8);
     L.s_dead = take(8, 8);
-    L.bars = take(8 * (2 * TD_STAGES + 2 * TD_ACC + 1), 8);
+    L.bars = take(8 * (2 * TD_MAX_STAGES + 2 * TD_ACC + 1), 8);
     L.tmem_slot = take(8, 8);
     L.s_ph = take(sizeof(TdPhase) * TD_MAX_PHASES, 16);
     L.total = o + 1024; // slack to align the base to 1024 bytes
@@ -123,7 +127,6 @@ __host__ __device__ inline TdSmem td_smem_layout() {
 
 __host__ __device__ inline bool td_is_gemm(int kind) { return kind == TD_QKV || kind == TD_OUT || kind == TD_UP || kind == TD_DOWN || kind == TD_HEAD; }
 __device__ __forceinline__ void td_bar() { asm volatile("bar.sync 1, %0;" ::"n"(TD_CTHREADS) : "memory"); }
-__device__ __forceinline__ void td_epi_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); } // warps 4..7
 
 // unit u of a phase -> (k range, matrix, row tile); units are ordered k-range-major so that a block's units share B
 struct TdUnit { int ks, mat, tile, kb_lo, kb_hi; };
@@ -157,6 +160,14 @@ __device__ __forceinline__ void td_b_store4(unsigned char *B, int i, int c_rel, 
     }
     *reinterpret_cast<uint2 *>(B + td_b_off(i, c_rel)) = make_uint2((uint32_t)hi[0] | ((uint32_t)hi[1] << 16), (uint32_t)hi[2] | ((uint32_t)hi[3] << 16));
     *reinterpret_cast<uint2 *>(B + td_b_off(i + 8, c_rel)) = make_uint2((uint32_t)lo[0] | ((uint32_t)lo[1] << 16), (uint32_t)lo[2] | ((uint32_t)lo[3] << 16));
+}
+
+// Take a ticket: the increment releases what this warp wrote before it (the lanes meet in __syncwarp first) and acquires
+// what earlier ticket holders wrote, so whoever draws the last ticket may read every partial result.
+__device__ __forceinline__ int td_ticket(int *p) {
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(p) : "memory");
+    return old;
 }
 
 __device__ __forceinline__ float4 td_add4(float4 a, const float4 b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; return a; }
@@ -301,17 +312,15 @@ __device__ __forceinline__ void td_attn_unit(const TdParams &P, const TdTeam &T,
 #pragma unroll
         for (int e = 0; e < EPL; ++e) part[4 + sub * EPL + e] = o[e];
     }
-    __threadfence();
     __syncwarp();
     int last = 0;
     if (lane == 0) {
         int *tk = T.att_ticket + i * P.n_head + h;
-        last = atomicAdd(tk, 1) == nsp - 1;
+        last = td_ticket(tk) == nsp - 1;
         if (last) *tk = 0;
     }
     last = __shfl_sync(0xffffffffu, last, 0);
     if (!last) return;
-    __threadfence();
     // every lane reads all split headers, then its four output elements of every split (HD <= 128: lanes 0 .. HD/4-1)
     const float *pb = T.att_part + ((size_t)i * P.n_head + h) * nsp * (HD + 4);
     float ms[TD_MAX_SPLITS], ls[TD_MAX_SPLITS];
@@ -357,10 +366,10 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)td_raw + 1023) & ~(uintptr_t)1023);
     const TdSmem L = td_smem_layout();
     unsigned char *ring = smem + L.ring;
-    unsigned char *Bsm = smem + L.b;
+    const int TD_STAGES = td_stages(P.b_kb);
+    unsigned char *Bsm = ring + (size_t)TD_STAGES * TD_W_BYTES;
     float *stats = reinterpret_cast<float *>(smem + L.stats);   // [TD_MAXB][2]: mean, 1/std
     float *red = reinterpret_cast<float *>(smem + L.red);       // [TD_CWARPS][TD_MAXB][2]
-    volatile int *s_flag = reinterpret_cast<volatile int *>(smem + L.s_flag);
     int *s_dead = reinterpret_cast<int *>(smem + L.s_dead);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L.bars);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L.tmem_slot);
@@ -374,8 +383,8 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
     const int cta = blockIdx.x - T.first_cta;
     const int K = P.K, G = P.G, d = P.d;
     const uint32_t ring_u32 = smem_u32(ring), b_u32 = smem_u32(Bsm);
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + TD_STAGES), accf0 = smem_u32(bars + 2 * TD_STAGES),
-                   acce0 = smem_u32(bars + 2 * TD_STAGES + TD_ACC), done_bar = smem_u32(bars + 2 * TD_STAGES + 2 * TD_ACC);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + TD_MAX_STAGES), accf0 = smem_u32(bars + 2 * TD_MAX_STAGES),
+                   acce0 = smem_u32(bars + 2 * TD_MAX_STAGES + TD_ACC), done_bar = smem_u32(bars + 2 * TD_MAX_STAGES + 2 * TD_ACC);
 
     if (tid == 0) {
         for (int s = 0; s < TD_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -386,7 +395,7 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
     }
     for (int i = tid; i < T.n_phases * (int)(sizeof(TdPhase) / 8); i += TD_THREADS)
         reinterpret_cast<unsigned long long *>(s_ph)[i] = reinterpret_cast<const unsigned long long *>(P.phases + T.phase_begin)[i];
-    for (int i = tid; i < TD_B_BYTES / 16; i += TD_THREADS) reinterpret_cast<uint4 *>(Bsm)[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < P.b_kb * 2048 / 16; i += TD_THREADS) reinterpret_cast<uint4 *>(Bsm)[i] = make_uint4(0u, 0u, 0u, 0u);
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(64u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -626,11 +635,14 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
                         for (int u = ub; u < ue; ++u) {
                             const unsigned ac = acc_base + (unsigned)(u - ub);
                             const int a = (int)(ac % TD_ACC);
+                            lap(2);
                             if (ac >= (unsigned)TD_ACC) wait_mbar(acce0 + 8 * a, ((ac / TD_ACC) - 1u) & 1u, P.err, PKE_EMPTY, dead, P.wait_ns);
+                            lap(11);
                             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                             const uint32_t dcol = tmem_base + (uint32_t)(a * 16);
                             for (int kb = first.kb_lo; kb < first.kb_hi; ++kb) {
                                 wait_mbar(full0 + 8 * stage, spar, P.err, PKE_FULL, dead, P.wait_ns);
+                                lap(10);
                                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                                 const uint32_t wbase = ring_u32 + stage * TD_W_BYTES, bbase = b_u32 + (uint32_t)(kb - first.kb_lo) * 2048u;
 #pragma unroll
@@ -642,7 +654,7 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
                             tg_commit(accf0 + 8 * a);
                         }
                         if (dead) *s_dead = 1;
-                    } else if (warp >= 4) {
+                    } else if (warp >= 4 && warp < 8) {
                         const int lane_base = (warp & 3) * 32;
                         for (int u = ub; u < ue; ++u) {
                             const TdUnit un = td_unit(ph, u);
@@ -674,25 +686,30 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
                                     for (int i = 0; i < TD_MAXB; ++i)
                                         if (i < nb) pp[(size_t)i * ph.n_rows] = val[i];
                                 }
-                                __threadfence();
-                                td_epi_bar();
-                                if (warp == 4 && lane == 0) {
-                                    int *tk = ph.ticket + un.mat * ph.n_tiles + un.tile;
-                                    const int lastone = atomicAdd(tk, 1) == ph.n_split - 1;
+                                // (a ticket per warp: its 32 rows of the tile; no block-wide step in between)
+                                __syncwarp();
+                                int lastone = 0;
+                                if (lane == 0) {
+                                    int *tk = ph.ticket + (un.mat * ph.n_tiles + un.tile) * 4 + (warp & 3);
+                                    lastone = td_ticket(tk) == ph.n_split - 1;
                                     if (lastone) *tk = 0;
-                                    *s_flag = lastone;
                                 }
-                                td_epi_bar();
-                                finish = *s_flag != 0;
+                                finish = __shfl_sync(0xffffffffu, lastone, 0) != 0;
                                 if (finish && rv) {
-                                    __threadfence();
                                     const float *p0 = ph.part + ((size_t)(un.mat * ph.n_split) * TD_MAXB) * ph.n_rows + row;
 #pragma unroll
                                     for (int i = 0; i < TD_MAXB; ++i) val[i] = 0.f;
-                                    for (int ks = 0; ks < ph.n_split; ++ks) {
+                                    for (int ks0 = 0; ks0 < ph.n_split; ks0 += 4) {
+                                        float t[4][TD_MAXB];
 #pragma unroll
-                                        for (int i = 0; i < TD_MAXB; ++i)
-                                            if (i < nb) val[i] += __ldcg(p0 + ((size_t)ks * TD_MAXB + i) * ph.n_rows);
+                                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                                            for (int i = 0; i < TD_MAXB; ++i)
+                                                t[q][i] = (ks0 + q < ph.n_split && i < nb) ? __ldcg(p0 + ((size_t)(ks0 + q) * TD_MAXB + i) * ph.n_rows) : 0.f;
+#pragma unroll
+                                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                                            for (int i = 0; i < TD_MAXB; ++i) val[i] += t[q][i];
                                     }
                                 }
                             }
@@ -732,13 +749,15 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
                         if (dead) *s_dead = 1;
                     }
                     acc_cnt = acc_base + (unsigned)(ue - ub);
+                    lap(2);
                     td_bar(); // the accumulators of this range were read, hence every MMA that read B has completed
+                    lap(ph.kind == TD_HEAD ? 9 : 2);
                     if (*(volatile int *)s_dead) dead = true;
                     ub = ue;
                 }
-                lap(2);
+                lap(ph.kind == TD_HEAD ? 9 : 2);
                 team_barrier();
-                lap(3);
+                lap(ph.kind == TD_HEAD ? 8 : 3);
                 if (ph.kind == TD_HEAD && cta == 0) {
                     // ---- token choice: best candidate per sample, lowest id on ties
                     const int n_cand = 4 * ph.n_tiles;
@@ -779,7 +798,8 @@ __global__ void __launch_bounds__(TD_THREADS, 1) k_tc_decode(const TdParams P) {
         if (cta == 0)
             for (int s = ct; s < P.n_samples; s += TD_CTHREADS) T.pos[s] += P.n_pass;
         if (prof_on)
-            for (int i = 0; i < 6; ++i) P.prof[(size_t)blockIdx.x * PK_PROF_N + i] = pf[i];
+            for (int i = 0; i < PK_PROF_N; ++i)
+                if (i != 6 && i != 7) P.prof[(size_t)blockIdx.x * PK_PROF_N + i] = pf[i];
         if (warp == 1 && lane == 0) {
             // no MMA may be in flight when tensor memory is freed (after a time-out some could still be)
             tg_commit(done_bar);
