@@ -358,14 +358,18 @@ def main():
     ap.add_argument("--kv-cache-dtype", type=int, default=0, help="0 library default, 1 bf16, 2 fp16, 3 fp32")
     ap.add_argument("--n-new", type=int, default=0, help="shorter generation (profiler captures only; not the headline)")
     ap.add_argument("--n-prompt", type=int, default=0, help="shorter prompts (profiler captures only)")
-    ap.add_argument("--n-layer", type=int, default=0, help="fewer blocks, one partition (profiler captures only)")
+    ap.add_argument("--n-layer", type=int, default=0, help="fewer blocks (profiler captures only)")
+    ap.add_argument("--partitions", type=int, default=1, help="with --n-layer: partitions of equal size")
+    ap.add_argument("--n-samples", type=int, default=0, help="fewer samples in flight (profiler captures only)")
     args = ap.parse_args()
     headline_only = args.workload is not None or args.no_per_workload
     w = I.ALL_WORKLOADS[args.workload or HEADLINE]
     if args.n_new or args.n_prompt:
         w = I.scaled(w, n_new=args.n_new or w.n_new, n_prompt=args.n_prompt or w.n_prompt)
     if args.n_layer:
-        w = I.scaled(w, n_layer=args.n_layer, part_bounds=(0, args.n_layer))
+        w = I.scaled(w, n_layer=args.n_layer, part_bounds=tuple(range(0, args.n_layer + 1, args.n_layer // args.partitions)))
+    if args.n_samples:
+        w = I.scaled(w, n_samples=args.n_samples)
     from paper_2505_18164_b200 import build
     build.build_inputs()
 

@@ -96,7 +96,7 @@ struct mdi_ctx {
     float *rope_cos = nullptr, *rope_sin = nullptr;
     // output layers
     float *logits = nullptr; // [S][V]
-    float *head_pv = nullptr;
+    float *head_pv = nullptr, *head_y = nullptr; // head_y: [MAXB][vocab] logits of a tensor-core output layer, by item
     int *head_pi = nullptr;
     unsigned *head_ticket = nullptr;
     int head_grid = 0;
@@ -366,6 +366,7 @@ int enqueue_head(mdi_ctx *c, const Batch &hb, const float *x_rows, const HeadReq
 }
 
 int tc_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in, float *x_out, cudaStream_t st);
+int tc_head(mdi_ctx *c, const Batch &hb, const float *x_rows, const HeadReq &head, cudaStream_t st);
 
 // All kernels of one visit of a batch of items to partition p.
 //   x_in:  [n][d] input activations (ignored for p == 0, which embeds tokens from tok_src)
@@ -439,7 +440,8 @@ int enqueue_partition_step(mdi_ctx *c, int p, const Batch &bt, const float *x_in
     }
     if (head && p == c->K - 1) {
         const Batch hb = head->item < 0 ? bt : slice(bt, head->item, 1);
-        const int rc = enqueue_head(c, hb, head->item < 0 ? x_out : x_out + (size_t)head->item * d, *head, st);
+        const float *xh = head->item < 0 ? x_out : x_out + (size_t)head->item * d;
+        const int rc = (tc && c->head_y) ? tc_head(c, hb, xh, *head, st) : enqueue_head(c, hb, xh, *head, st);
         if (rc != MDI_OK) return rc;
     }
     if (c->capturing) ++c->cap_steps; else ++c->st.stage_steps;
@@ -518,7 +520,7 @@ int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, c
     if ((rc = pf_map(c, P.pf_lo, PF_CHUNK, (uint64_t)K, (uint32_t)n_tile, &mlo)) != MDI_OK) return rc;
     const int grid_x = (n_rows + TG_BM - 1) / TG_BM, n_kb = (K + TG_BK - 1) / TG_BK;
     int splits = 1;
-    if (pending && grid_x < 32) splits = std::max(1, std::min(std::min(PF_SPLIT_MAX, c->n_sm / grid_x), n_kb / 8));
+    if (pending && 2 * grid_x <= c->n_sm) splits = std::max(1, std::min(std::min(PF_SPLIT_MAX, c->n_sm / grid_x), n_kb / 8));
     TgArgs a{};
     a.n_rows = n_rows; a.K = K; a.T = T; a.n_tile = n_tile; a.bias = bias; a.resid = resid; a.act = act; a.y = y; a.ldy = n_rows;
     a.err = c->tg_err; a.partial = P.pf_part; a.out_hi = out_hi; a.out_lo = out_lo;
@@ -558,6 +560,8 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
     __nv_bfloat16 *hi = (__nv_bfloat16 *)P.pf_hi, *lo = (__nv_bfloat16 *)P.pf_lo;
     int rc;
     const bool pdl = c->pdl;
+    // element-wise helpers: few rows (a decode step) are cut into column slices so that their grids are not a handful of blocks
+    const int ysl = std::max(1, std::min(16, 2 * c->n_sm / std::max(T, 1) / 4));
     if (!bt && p == 0) {
         launch_k(pdl, k_pf_embed<__nv_bfloat16>, dim3(T), dim3(256), 0, st, (const __nv_bfloat16 *)c->wte, (const __nv_bfloat16 *)c->wpe, d, s.vocab, tok_dev,
                                                     P.pos_dev, slot, P.pf_xa);
@@ -576,7 +580,7 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
         pend = PfPending();
         if ((rc = pf_gemm(c, P, L.wqkv, qw + 2 * kw, d, T, L.bqkv, nullptr, TG_NONE, P.pf_qkv, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
         if (bt) {
-            KV_DISPATCH(c->kv_kind, launch_k(pdl, k_bt_rope_append<KT>, dim3(T), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf));
+            KV_DISPATCH(c->kv_kind, launch_k(pdl, k_bt_rope_append<KT>, dim3(T, ysl), dim3(256), 0, st, P.pf_qkv, qw, kw, s.head_dim, rope, c->rope_cos, c->rope_sin, kv, ll, P.pos_dev, *bt, P.qbuf));
             count_launch(c);
             AttnArgs a{};
             a.q = P.qbuf; a.o = P.obuf; a.part = P.part; a.ticket = P.attn_ticket; a.kv = kv; a.layer_local = ll; a.n_head = s.n_head;
@@ -599,7 +603,7 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
         if (s.act == MDI_ACT_SWIGLU) {
             if ((rc = pf_gemm(c, P, L.wgate, F, d, T, nullptr, nullptr, TG_NONE, P.pf_h, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
             if ((rc = pf_gemm(c, P, L.wup, F, d, T, nullptr, nullptr, TG_NONE, P.pf_u, nullptr, nullptr, nullptr, st)) != MDI_OK) return rc;
-            launch_k(pdl, k_pf_swiglu_split, dim3(T), dim3(256), 0, st, P.pf_h, P.pf_u, F, hi, lo);
+            launch_k(pdl, k_pf_swiglu_split, dim3(T, ysl), dim3(256), 0, st, P.pf_h, P.pf_u, F, hi, lo);
             count_launch(c);
             if ((rc = pf_gemm(c, P, L.wdown, d, F, T, nullptr, x_out, TG_NONE, x_out, nullptr, nullptr, &pend, st)) != MDI_OK) return rc;
         } else {
@@ -619,6 +623,33 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
     }
     if (bt) launch_k(pdl, k_bt_advance, dim3(1), dim3(32), 0, st, P.pos_dev, *bt);
     else launch_k(pdl, k_pf_advance, dim3(1), dim3(32), 0, st, P.pos_dev, slot, T);
+    count_launch(c);
+    return MDI_OK;
+}
+
+// Output layers of a tensor-core decode step: final norm + hi/lo split, the vocabulary projection as one more GEMM
+// (logits of the hb.n items into head_y), then token choice from those logits.
+int tc_head(mdi_ctx *c, const Batch &hb, const float *x_rows, const HeadReq &head, cudaStream_t st) {
+    const mdi_model_shape &s = c->s;
+    Partition &P = c->part[c->K - 1];
+    const int d = s.d_model, V = s.vocab, T = hb.n;
+    const bool pdl = c->pdl;
+    __nv_bfloat16 *hi = (__nv_bfloat16 *)P.pf_hi, *lo = (__nv_bfloat16 *)P.pf_lo;
+    launch_k(pdl, k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, x_rows, d, s.arch == MDI_ARCH_GPT ? NORM_LAYER : NORM_RMS, c->lnfg, c->lnfb,
+             s.norm_eps, hi, lo, (const float *)nullptr, 0, T, (const float *)nullptr, (float *)nullptr);
+    count_launch(c);
+    int rc = pf_gemm(c, P, s.tied_lm_head ? c->wte : c->lm_head, V, d, T, nullptr, nullptr, TG_NONE, c->head_y, nullptr, nullptr, nullptr, st);
+    if (rc != MDI_OK) return rc;
+    LinArgs a{};
+    a.n_rows = V; a.in_dim = d;
+    a.logits = c->logits; a.part_val = c->head_pv; a.part_idx = c->head_pi; a.ticket = c->head_ticket;
+    a.tok_out = head.tok_out; a.log_stride = s.n_ctx;
+    if (head.update_state) {
+        a.cur_tok = c->cur_tok; a.tok_log = c->tok_log; a.gen_count = c->gen_count;
+        a.teacher = c->teacher; a.n_teacher = c->n_teacher;
+        a.temperature = c->temperature; a.top_k = c->top_k; a.sample_seed = c->sample_seed;
+    }
+    launch_k(pdl, k_head_pick, dim3(std::min(1024, std::max(1, (V + 2047) / 2048 * 4))), dim3(LIN_THREADS), 0, st, a, hb, (const float *)c->head_y);
     count_launch(c);
     return MDI_OK;
 }
@@ -1275,6 +1306,8 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
             // The cooperative launch in clusters was refused by the runtime: plan again with one block per head, rebuild
             // the weight streams and launch that.
             cudaGetLastError();
+            // the clearing of the first plan's buffers is still queued: it must have run before they are released
+            CU(cudaStreamSynchronize(c->main));
             c->fz_no_pair = true;
             c->fz_ok = false;
             const int rs = fz_setup(c);
@@ -1634,7 +1667,7 @@ void mdi_destroy(mdi_ctx *c) {
         if (P.ev_join_cap) cudaEventDestroy(P.ev_join_cap);
         if (P.stream) cudaStreamDestroy(P.stream);
     }
-    void *ptrs[] = {c->rope_cos, c->rope_sin, c->logits, c->head_pv, c->head_pi, c->head_ticket, c->cur_tok, c->tok_log,
+    void *ptrs[] = {c->rope_cos, c->rope_sin, c->logits, c->head_pv, c->head_y, c->head_pi, c->head_ticket, c->cur_tok, c->tok_log,
                     c->gen_count, c->teacher, c->n_teacher, c->prompt_buf, c->pk_teams, c->pk_phases, c->pk_sync, c->pk_err, c->pk_prof, c->tg_err,
                     c->fz_teams, c->fz_phases, c->fz_works, c->fz_blocks, c->fz_segs, c->fz_units, c->fz_err, c->fz_stream, c->fz_acc, c->fz_sync, c->fz_prof, c->fz_trace,
                     c->td_teams, c->td_phases, c->td_maps, c->td_buf, c->td_ints, c->td_sync, c->td_err, c->td_prof};
@@ -1834,6 +1867,7 @@ int mdi_create(const mdi_model_shape *shape, const int *part_bounds, int K, int 
     TRY(dalloc(c, &c->head_pv, (size_t)MAXB * std::max(c->head_grid, 1024), acc));
     TRY(dalloc(c, &c->head_pi, (size_t)MAXB * std::max(c->head_grid, 1024), acc));
     TRY(dalloc(c, &c->head_ticket, 1, acc));
+    if (s.weight_dtype == MDI_DTYPE_BF16 && c->o.prefill_mode != 1) TRY(dalloc(c, &c->head_y, (size_t)MAXB * V, acc));
     TRY(dalloc(c, &c->cur_tok, (size_t)n_samples));
     TRY(dalloc(c, &c->gen_count, (size_t)n_samples));
     TRY(dalloc(c, &c->n_teacher, (size_t)n_samples));

@@ -74,12 +74,12 @@ __global__ void __launch_bounds__(PF_THREADS) k_pf_norm_split(const float *x, in
     }
 }
 
-// h = SiLU(g) * u, split.  grid (T)
+// h = SiLU(g) * u, split.  grid (T, column slices)
 __global__ void k_pf_swiglu_split(const float *g, const float *u, int n, __nv_bfloat16 *hi, __nv_bfloat16 *lo) {
     pdl_launch_dependents();
     pdl_wait();
     const int t = blockIdx.x;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < n; i += gridDim.y * blockDim.x) {
         const size_t k = (size_t)t * n + i;
         pf_split_store(hi, lo, k, silu_f(g[k]) * u[k]);
     }
@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(ATT_THREADS) k_pf_attn(const float *q, __nv_bf
 }
 
 // The same for a batch of items of different slots (a group's decode step): item i sits at pos[slot_i] + off_i.
-// grid (n items)
+// grid (n items, row slices)
 template <typename KT>
 __global__ void k_bt_rope_append(const float *qkv, int q_rows, int kv_rows, int hd, int rope, const float *rope_cos,
                                  const float *rope_sin, KvView kv, int layer_local, const int *pos, Batch bt, float *q_out) {
@@ -179,7 +179,7 @@ __global__ void k_bt_rope_append(const float *qkv, int q_rows, int kv_rows, int 
     pdl_wait();
     const int t = blockIdx.x, slot = bt.slot[t], p = pos[slot] + bt.off[t], half = hd >> 1, rows = q_rows + 2 * kv_rows;
     const float *src = qkv + (size_t)t * rows;
-    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+    for (int r = blockIdx.y * blockDim.x + threadIdx.x; r < rows; r += gridDim.y * blockDim.x) {
         float y = src[r];
         if (rope && r < q_rows + kv_rows) {
             const int e = r % hd, i = e % half;

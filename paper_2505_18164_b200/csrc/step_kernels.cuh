@@ -243,6 +243,118 @@ __device__ int block_sample_top_k(const float *lg, int n, int top_k, float tempe
     return *result;
 }
 
+// Last stage of the output layers, shared by the kernels that produce logits: every block has left its best
+// (value, row) per item in part_val / part_idx; the block that takes the last ticket picks the tokens (greedy: best
+// candidate, lowest row on ties; or a draw from the pmf of the top_k logits) and advances the slots' token state.
+__device__ __forceinline__ void head_finish(const LinArgs &a, const Batch &bt, bool *is_last, float *smp_v, int *smp_i, float *smp_wv,
+                                            int *smp_w, int *smp_res) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) *is_last = atomicAdd(a.ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (*is_last && a.temperature > 0.f && a.gen_count) {
+        // draw from the pmf instead of taking the argmax: one item at a time, the whole block on each
+        __threadfence();
+        for (int i = 0; i < bt.n; ++i) {
+            const int slot = bt.slot[i];
+            const int g = a.gen_count[slot];
+            const float *lg = a.logits + (size_t)(a.logits_by_item ? i : slot) * a.n_rows;
+            const int tok = block_sample_top_k(lg, a.n_rows, a.top_k, a.temperature, sample_uniform(a.sample_seed, slot, g), smp_v, smp_i,
+                                               smp_wv, smp_w, smp_res);
+            __syncthreads();
+            if (tid == 0) {
+                if (a.tok_out) a.tok_out[i] = tok;
+                if (g < a.log_stride) a.tok_log[(size_t)slot * a.log_stride + g] = tok;
+                int feed = tok;
+                if (a.teacher && g < a.n_teacher[slot]) feed = a.teacher[(size_t)slot * a.log_stride + g];
+                a.cur_tok[slot] = feed;
+                a.gen_count[slot] = g + 1;
+            }
+            __syncthreads();
+        }
+        if (tid == 0) *a.ticket = 0u;
+    } else if (*is_last) {
+        __threadfence();
+        for (int i = warp; i < bt.n; i += LIN_WARPS) {
+            float bv = -INFINITY;
+            int bi = 0x7fffffff;
+            for (int c = lane; c < (int)gridDim.x; c += 32) {
+                const float v = __ldcg(a.part_val + (size_t)i * gridDim.x + c);
+                const int ix = __ldcg(a.part_idx + (size_t)i * gridDim.x + c);
+                if (v > bv || (v == bv && ix < bi)) { bv = v; bi = ix; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float v = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int ix = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (v > bv || (v == bv && ix < bi)) { bv = v; bi = ix; }
+            }
+            if (lane == 0) {
+                const int slot = bt.slot[i];
+                if (a.tok_out) a.tok_out[i] = bi;
+                if (a.gen_count) {
+                    const int g = a.gen_count[slot];
+                    if (g < a.log_stride) a.tok_log[(size_t)slot * a.log_stride + g] = bi;
+                    int feed = bi;
+                    if (a.teacher && g < a.n_teacher[slot]) feed = a.teacher[(size_t)slot * a.log_stride + g];
+                    a.cur_tok[slot] = feed;
+                    a.gen_count[slot] = g + 1;
+                }
+            }
+        }
+        if (tid == 0) *a.ticket = 0u;
+    }
+}
+
+// Token choice from finished logits y[item][n_rows] (what a tensor-core contraction left): copies them to the
+// context's logits (by slot), finds every block's best row per item over its slice of the rows, then head_finish.
+// grid (row slices), LIN_THREADS threads.
+__global__ void __launch_bounds__(LIN_THREADS) k_head_pick(const LinArgs a, const Batch bt, const float *y) {
+    __shared__ float hv[LIN_WARPS][MAXB];
+    __shared__ int hi_[LIN_WARPS][MAXB];
+    __shared__ bool is_last;
+    __shared__ float smp_v[64];
+    __shared__ int smp_i[64], smp_w[LIN_WARPS], smp_res;
+    __shared__ float smp_wv[LIN_WARPS];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = (a.n_rows + gridDim.x - 1) / gridDim.x, r_lo = blockIdx.x * per, r_hi = min(a.n_rows, r_lo + per);
+    for (int i = 0; i < bt.n; ++i) {
+        float *lg = a.logits + (size_t)(a.logits_by_item ? i : bt.slot[i]) * a.n_rows;
+        const float *src = y + (size_t)i * a.n_rows;
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int r = r_lo + tid; r < r_hi; r += LIN_THREADS) {
+            const float v = __ldcg(src + r);
+            lg[r] = v;
+            if (v > bv) { bv = v; bi = r; } // rows ascend within a thread: the first maximum is the lowest row
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float v = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int ix = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (v > bv || (v == bv && ix < bi)) { bv = v; bi = ix; }
+        }
+        if (lane == 0) { hv[warp][i] = bv; hi_[warp][i] = bi; }
+    }
+    __syncthreads();
+    if (tid < bt.n) {
+        float bv = hv[0][tid];
+        int bi = hi_[0][tid];
+#pragma unroll
+        for (int w = 1; w < LIN_WARPS; ++w) {
+            const float v = hv[w][tid];
+            const int i = hi_[w][tid];
+            if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+        }
+        a.part_val[(size_t)tid * gridDim.x + blockIdx.x] = bv;
+        a.part_idx[(size_t)tid * gridDim.x + blockIdx.x] = bi;
+    }
+    head_finish(a, bt, &is_last, smp_v, smp_i, smp_wv, smp_w, &smp_res);
+}
+
 // ---- weight-streaming linear layer ------------------------------------------------------------
 // Each warp owns one unit of two weight rows and streams them once with 16-byte loads; the NB
 // input vectors sit in shared memory as fp32 (normalised in the prologue where asked).
@@ -421,62 +533,7 @@ __global__ void __launch_bounds__(LIN_THREADS) k_linear(const LinArgs a, const B
             a.part_val[(size_t)tid * gridDim.x + blockIdx.x] = bv;
             a.part_idx[(size_t)tid * gridDim.x + blockIdx.x] = bi;
         }
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) is_last = atomicAdd(a.ticket, 1u) == gridDim.x - 1;
-        __syncthreads();
-        if (is_last && a.temperature > 0.f && a.gen_count) {
-            // draw from the pmf instead of taking the argmax: one item at a time, the whole block on each
-            __threadfence();
-            for (int i = 0; i < bt.n; ++i) {
-                const int slot = bt.slot[i];
-                const int g = a.gen_count[slot];
-                const float *lg = a.logits + (size_t)(a.logits_by_item ? i : slot) * a.n_rows;
-                const int tok = block_sample_top_k(lg, a.n_rows, a.top_k, a.temperature, sample_uniform(a.sample_seed, slot, g), smp_v, smp_i,
-                                                   smp_wv, smp_w, &smp_res);
-                __syncthreads();
-                if (tid == 0) {
-                    if (a.tok_out) a.tok_out[i] = tok;
-                    if (g < a.log_stride) a.tok_log[(size_t)slot * a.log_stride + g] = tok;
-                    int feed = tok;
-                    if (a.teacher && g < a.n_teacher[slot]) feed = a.teacher[(size_t)slot * a.log_stride + g];
-                    a.cur_tok[slot] = feed;
-                    a.gen_count[slot] = g + 1;
-                }
-                __syncthreads();
-            }
-            if (tid == 0) *a.ticket = 0u;
-        } else if (is_last) {
-            __threadfence();
-            for (int i = warp; i < bt.n; i += LIN_WARPS) {
-                float bv = -INFINITY;
-                int bi = 0x7fffffff;
-                for (int c = lane; c < (int)gridDim.x; c += 32) {
-                    const float v = __ldcg(a.part_val + (size_t)i * gridDim.x + c);
-                    const int ix = __ldcg(a.part_idx + (size_t)i * gridDim.x + c);
-                    if (v > bv || (v == bv && ix < bi)) { bv = v; bi = ix; }
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    const float v = __shfl_xor_sync(0xffffffffu, bv, o);
-                    const int ix = __shfl_xor_sync(0xffffffffu, bi, o);
-                    if (v > bv || (v == bv && ix < bi)) { bv = v; bi = ix; }
-                }
-                if (lane == 0) {
-                    const int slot = bt.slot[i];
-                    if (a.tok_out) a.tok_out[i] = bi;
-                    if (a.gen_count) {
-                        const int g = a.gen_count[slot];
-                        if (g < a.log_stride) a.tok_log[(size_t)slot * a.log_stride + g] = bi;
-                        int feed = bi;
-                        if (a.teacher && g < a.n_teacher[slot]) feed = a.teacher[(size_t)slot * a.log_stride + g];
-                        a.cur_tok[slot] = feed;
-                        a.gen_count[slot] = g + 1;
-                    }
-                }
-            }
-            if (tid == 0) *a.ticket = 0u;
-        }
+        head_finish(a, bt, &is_last, smp_v, smp_i, smp_wv, smp_w, &smp_res);
     }
 }
 
