@@ -108,10 +108,9 @@ typedef struct {
     int in_kernel_timing; /* 1: the persistent kernels time themselves (mdi_get_partition_times); costs a few percent */
     int fused_blocks_per_head; /* fused-phase kernel: 0 (default) two thread blocks of a cluster share a head where every
                           team has a cluster per head, else one block per head; 1: always one block per head (plain
-                          cooperative launch, no clusters) */
-    int debug_refuse_cluster_launch; /* checking aid: 1 makes the first fused-phase launch in clusters behave as if the
-                          runtime had refused it (nothing is launched), so that the library plans again with one block
-                          per head, as it does after a real refusal */
+                          cooperative launch, no clusters: the choice for a runtime or tool that refuses cooperative launches
+                          in clusters, which otherwise fail with MDI_ERR_CUDA) */
+    int reserved0;     /* must be 0 */
     int trace_slot;    /* with in_kernel_timing: s > 0 makes thread 0 of every block of the fused-phase kernel record a
                           time stamp at every change of timing category while it serves schedule slot s - 1
                           (mdi_get_trace) */

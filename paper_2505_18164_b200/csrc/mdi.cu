@@ -149,13 +149,11 @@ struct mdi_ctx {
     FzSeg *fz_segs = nullptr;
     int *fz_units = nullptr, *fz_err = nullptr;
     int fz_kv_pps = 1, fz_pair = 0, fz_kv_rows = 16;
-    bool fz_no_pair = false; // a cluster launch was refused once: one block per head from then on
     uint4 *fz_stream = nullptr;
     long long *fz_acc = nullptr;
     unsigned *fz_sync = nullptr;
     unsigned long long *fz_prof = nullptr, *fz_trace = nullptr;
     int fz_trace_blocks = 0;
-    bool fz_refusal_faked = false;
     int64_t fz_stream_bytes = 0;
     std::vector<int64_t> fz_team_stream_bytes; // per partition: bytes of its blocks' weight streams
     // persistent tensor-core decode kernel (bf16 weights, groups of up to 8 samples): plan at creation, tables at first use
@@ -915,6 +913,7 @@ int pk_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     const int nb = (n_samples + G - 1) / G;
     const int tnb = nb <= 1 ? 1 : nb <= 2 ? 2 : 4;
     const void *fn = pk_func_for(c, tnb);
+    CU(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pk_smem)); // per function, not per context
     void *args[] = {&P};
     CU(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(PK_THREADS), args, c->pk_smem, c->main));
     ++c->st.kernel_launches;
@@ -953,7 +952,7 @@ int fz_setup(mdi_ctx *c) {
     // Pair mode: a head is served by the two blocks of a cluster (halves of its q,k,v rows, of the rows of every cache
     // page and of its output rows).  Needs even tile counts, pages of at least two rows, even team sizes with a cluster
     // per head, and all clusters resident at once.
-    bool pair = !c->fz_no_pair && c->o.fused_blocks_per_head != 1 && c->page_tokens >= 2 && (3 * hd / 16) % 2 == 0 && (d / 16) % 2 == 0 && n_sm >= 2;
+    bool pair = c->o.fused_blocks_per_head != 1 && c->page_tokens >= 2 && (3 * hd / 16) % 2 == 0 && (d / 16) % 2 == 0 && n_sm >= 2;
     if (pair) {
         for (int nb : {1, 2, 4}) CU(cudaFuncSetAttribute(fz_func(nb), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prop.sharedMemPerBlockOptin));
         cudaLaunchConfig_t cfg = {};
@@ -1088,11 +1087,6 @@ int fz_setup(mdi_ctx *c) {
     c->fz_smem = fz_smem_layout(NB, c->fz_slots, d, hd, c->fz_part_floats, c->pages_per_seq, c->fz_xb_stride, c->fz_hb_stride, c->fz_ob_stride).total;
     for (int nb : {1, 2, 4}) CU(cudaFuncSetAttribute(fz_func(nb), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->fz_smem));
     int rc;
-    {   // (a second plan after a refused cluster launch replaces the first one's buffers)
-        void *prev[] = {c->fz_sync, c->fz_err, c->fz_acc, c->fz_prof};
-        for (void *q : prev) if (q) cudaFree(q);
-        c->fz_sync = nullptr; c->fz_err = nullptr; c->fz_acc = nullptr; c->fz_prof = nullptr;
-    }
     if ((rc = dalloc(c, &c->fz_sync, (size_t)K * 64)) != MDI_OK) return rc;
     if ((rc = dalloc(c, &c->fz_err, 1)) != MDI_OK) return rc;
     if ((rc = dalloc(c, &c->fz_acc, (size_t)K * 3 * FZ_MAXNB * d)) != MDI_OK) return rc;
@@ -1288,6 +1282,7 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     }
     // the template parameter fixes the accumulator stride, so it is the context's group size, not this call's
     const void *fn = fz_func(c->fz_nb);
+    CU(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->fz_smem)); // per function, not per context
     void *args[] = {&P};
     if (c->fz_pair) {
         // cooperative (all blocks resident: teams wait on one another) and in clusters of two (the halves of a head)
@@ -1298,23 +1293,11 @@ int fz_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
         at[1].id = cudaLaunchAttributeClusterDimension;
         at[1].val.clusterDim.x = 2; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 2;
-        // (debug_refuse_cluster_launch: behave once as if the runtime had refused, without launching anything)
-        const bool pretend = c->o.debug_refuse_cluster_launch == 1 && !c->fz_refusal_faked;
-        c->fz_refusal_faked = c->fz_refusal_faked || pretend;
-        const cudaError_t le = pretend ? cudaErrorCooperativeLaunchTooLarge : cudaLaunchKernelExC(&cfg, fn, args);
+        const cudaError_t le = cudaLaunchKernelExC(&cfg, fn, args);
         if (le != cudaSuccess) {
-            // The cooperative launch in clusters was refused by the runtime: plan again with one block per head, rebuild
-            // the weight streams and launch that.
             cudaGetLastError();
-            // the clearing of the first plan's buffers is still queued: it must have run before they are released
-            CU(cudaStreamSynchronize(c->main));
-            c->fz_no_pair = true;
-            c->fz_ok = false;
-            const int rs = fz_setup(c);
-            if (rs != MDI_OK) return rs;
-            if (!c->fz_ok || c->fz_pair) return fail(c, MDI_ERR_CUDA, "cluster launch refused (%s) and no plan without clusters", cudaGetErrorString(le));
-            c->fz_stale = true;
-            return fz_launch(c, n_samples, G, n_pass);
+            return fail(c, MDI_ERR_CUDA, "the runtime refused the cooperative launch in clusters of two (%s): create the context with "
+                        "fused_blocks_per_head = 1 (one block per head, no clusters)", cudaGetErrorString(le));
         }
     } else {
         CU(cudaLaunchCooperativeKernel(fn, dim3(c->fz_grid), dim3(FZ_THREADS), args, c->fz_smem, c->main));
@@ -1631,6 +1614,7 @@ int td_launch(mdi_ctx *c, int n_samples, int G, int n_pass) {
     c->withhold_once = -1;
     P.prof = c->td_prof;
     void *args[] = {&P};
+    CU(cudaFuncSetAttribute(td_func(c), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->td_smem)); // per function, not per context
     CU(cudaLaunchCooperativeKernel(td_func(c), dim3(c->td_grid), dim3(TD_THREADS), args, c->td_smem, c->main));
     ++c->st.kernel_launches;
     c->st.stage_steps += (int64_t)c->K * n_pass * G;

@@ -44,7 +44,7 @@ class Options(ctypes.Structure):
     _fields_ = [("page_tokens", ctypes.c_int), ("kv_pool_tokens", ctypes.c_int), ("attn_splits", ctypes.c_int),
                 ("rounds_per_graph", ctypes.c_int), ("kv_cache_dtype", ctypes.c_int), ("prefill_mode", ctypes.c_int), ("tc_min_group", ctypes.c_int), ("wait_limit_ms", ctypes.c_int), ("debug_withhold_handoff", ctypes.c_int),
                 ("scheduler", ctypes.c_int), ("in_kernel_timing", ctypes.c_int), ("fused_blocks_per_head", ctypes.c_int),
-                ("debug_refuse_cluster_launch", ctypes.c_int), ("trace_slot", ctypes.c_int), ("td_b_kblocks", ctypes.c_int)]
+                ("reserved0", ctypes.c_int), ("trace_slot", ctypes.c_int), ("td_b_kblocks", ctypes.c_int)]
 
 
 class Stats(ctypes.Structure):
@@ -120,7 +120,7 @@ class Context:
                  kv_pool_tokens: int = 0, attn_splits: int = 0, rounds_per_graph: int = 0, scheduler: int = 0,
                  kv_cache_dtype: int = 0, prefill_mode: int = 0, tc_min_group: int = 0,
                  wait_limit_ms: int = 0, debug_withhold_handoff: int = 0, in_kernel_timing: int = 0,
-                 fused_blocks_per_head: int = 0, debug_refuse_cluster_launch: int = 0, trace_slot: int = 0, td_b_kblocks: int = 0):
+                 fused_blocks_per_head: int = 0, trace_slot: int = 0, td_b_kblocks: int = 0):
         self._h = None
         self.shape = shape
         self.K = len(part_bounds) - 1
@@ -129,7 +129,7 @@ class Context:
         bounds = (ctypes.c_int * len(part_bounds))(*part_bounds)
         opts = Options(page_tokens, kv_pool_tokens, attn_splits, rounds_per_graph, kv_cache_dtype, prefill_mode, tc_min_group,
                        wait_limit_ms, debug_withhold_handoff, scheduler, in_kernel_timing, fused_blocks_per_head,
-                       debug_refuse_cluster_launch, trace_slot, td_b_kblocks)
+                       0, trace_slot, td_b_kblocks)
         h = ctypes.c_void_p()
         rc = lib().mdi_create(ctypes.byref(cs), bounds, self.K, n_samples, ctypes.byref(opts), ctypes.byref(h))
         if rc != MDI_OK:

@@ -145,30 +145,3 @@ def test_fused_kernel_one_or_two_blocks_per_head_agree():
         ctx.close()
     assert np.abs(res[0] - res[1]).max() < 1e-3
 
-
-def test_refused_cluster_launch_plans_again_with_one_block_per_head():
-    """When the runtime refuses the cooperative launch in clusters the library plans again without clusters, rebuilds
-    its per-block weight streams and carries on.  The refusal is played on the host (debug_refuse_cluster_launch:
-    nothing is launched in its place); the re-planned run must give the tokens and logits of a context that was
-    created with one block per head, and later calls on the same context must keep working."""
-    shape = tiny_shape("gpt", I.DT_BF16, L=4, d=256, H=4, V=523, C=192)
-    orc, w = make_oracle(shape, seed=21, std=0.04)
-    prompts = I.make_prompts(523, 3, 40, seed=8)
-    runs = []
-    for kw in (dict(fused_blocks_per_head=1), dict(debug_refuse_cluster_launch=1)):
-        ctx = _ctx(shape, [0, 2, 4], 3, w, scheduler=3, page_tokens=32, **kw)
-        for s in range(3):
-            ctx.prefill(s, prompts[s])
-        a = ctx.generate(3, 20).copy()
-        b = ctx.generate(3, 20).copy()
-        lg = np.stack([ctx.get_logits(s) for s in range(3)])
-        runs.append((a, b, lg))
-        ctx.close()
-    assert np.array_equal(runs[0][0], runs[1][0]) and np.array_equal(runs[0][1], runs[1][1])
-    assert np.array_equal(runs[0][2], runs[1][2])          # same plan, integer accumulators: bit-identical logits
-    toks, lgs, margins = oracle_reference(orc, prompts, 40)
-    tol = parity_tolerance(shape)
-    got = np.concatenate([runs[1][0], runs[1][1]], axis=1)
-    for s in range(3):
-        first_low = int(np.argmax(margins[s] <= 2 * tol)) if (margins[s] <= 2 * tol).any() else 40
-        assert np.array_equal(got[s][:first_low], np.asarray(toks[s])[:first_low])
