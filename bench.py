@@ -248,7 +248,8 @@ def run_workload(w: I.Workload, args, steps: int, warmup: int, e2e_steps: int, w
     s = w.shape
     S, P, N = w.n_samples, w.n_prompt, w.n_new
     ctx = mdi.Context(s, list(w.part_bounds), S, kv_pool_tokens=S * ((P + N + 15) // 16 * 16), rounds_per_graph=args.rounds_per_graph,
-                      scheduler=args.scheduler, tc_min_group=args.tc_min_group, kv_cache_dtype=args.kv_cache_dtype)
+                      scheduler=args.scheduler, tc_min_group=args.tc_min_group, kv_cache_dtype=args.kv_cache_dtype,
+                      in_kernel_timing=1 if args.in_kernel_timing else 0, td_b_kblocks=args.td_b_kblocks)
     weights = {}
     for name, a in I.iter_weights(s, w.weight_seed):
         ctx.load_weights(name, a)
@@ -311,7 +312,13 @@ def run_workload(w: I.Workload, args, steps: int, warmup: int, e2e_steps: int, w
         barrier()
         assert np.array_equal(out_np, tokens_dev), "host and device entry points disagree"
     kv_stored_bpe = int(st1.kv_element_bytes)
-    res = {"run_ms": run_ms, "gen_ms": gen_ms, "pf_ms": pf_ms, "e2e_s": e2e_s, "clocks": clocks,
+    ptimes = None
+    if args.in_kernel_timing:
+        try:
+            ptimes = [dict(zip(("blocks", "ms"), ctx.partition_times(p))) for p in range(w.n_partitions)]
+        except Exception as e:  # the stream scheduler has no in-kernel timing
+            ptimes = str(e)
+    res = {"run_ms": run_ms, "gen_ms": gen_ms, "pf_ms": pf_ms, "e2e_s": e2e_s, "clocks": clocks, "partition_times_ms": ptimes,
            "launches": int(st1.kernel_launches - st0.kernel_launches), "kv_stored_bpe": kv_stored_bpe}
     ctx.close()
     del ctx
@@ -356,6 +363,9 @@ def main():
     ap.add_argument("--scheduler", type=int, default=0, help="0 auto (a persistent kernel when the shape fits), 1 streams, 2 phase-per-matrix persistent kernel, 3 fused-phase persistent kernel")
     ap.add_argument("--tc-min-group", type=int, default=0, help="smallest group whose decode steps run on the tensor cores (0 = library default)")
     ap.add_argument("--kv-cache-dtype", type=int, default=0, help="0 library default, 1 bf16, 2 fp16, 3 fp32")
+    ap.add_argument("--in-kernel-timing", action="store_true", help="persistent kernels time themselves; adds partition_times_ms "
+                    "(per partition: blocks, milliseconds per category of the last generate call) to the line")
+    ap.add_argument("--td-b-kblocks", type=int, default=0, help="scheduler 4: k-blocks of the resident activation operand")
     ap.add_argument("--n-new", type=int, default=0, help="shorter generation (profiler captures only; not the headline)")
     ap.add_argument("--n-prompt", type=int, default=0, help="shorter prompts (profiler captures only)")
     ap.add_argument("--n-layer", type=int, default=0, help="fewer blocks (profiler captures only)")
@@ -428,6 +438,8 @@ def main():
             "clocks": r["clocks"],
             "cpu_baseline": r.get("cpu_baseline"),
         }
+        if r.get("partition_times_ms") is not None:
+            line["partition_times_ms"] = r["partition_times_ms"]
         if per:
             out = []
             for item in per:
