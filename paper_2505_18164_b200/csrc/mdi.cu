@@ -609,7 +609,7 @@ int tc_layers(mdi_ctx *c, int p, const Batch *bt, int slot, const int *tok_dev, 
             if ((rc = pf_gemm(c, P, L.w1, F, d, T, L.b1, nullptr, s.act == MDI_ACT_GELU_ERF ? TG_GELU_ERF : TG_GELU_TANH, P.pf_h, nullptr, nullptr,
                               nullptr, st)) != MDI_OK)
                 return rc;
-            launch_k(pdl, k_pf_norm_split, dim3(T), dim3(PF_THREADS), 0, st, P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo, nullptr, 0, T, nullptr, nullptr);
+            launch_k(pdl, k_pf_norm_split, dim3(T, ysl), dim3(PF_THREADS), 0, st, P.pf_h, F, NORM_NONE, nullptr, nullptr, 0.f, hi, lo, nullptr, 0, T, nullptr, nullptr);
             count_launch(c);
             if ((rc = pf_gemm(c, P, L.w2, d, F, T, L.b2, x_out, TG_NONE, x_out, nullptr, nullptr, &pend, st)) != MDI_OK) return rc;
         }

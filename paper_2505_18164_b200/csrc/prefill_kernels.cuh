@@ -7,7 +7,7 @@
 
 namespace mdi {
 
-constexpr int PF_THREADS = 256;
+constexpr int PF_THREADS = 512;
 
 __device__ __forceinline__ void pf_split_store(__nv_bfloat16 *hi, __nv_bfloat16 *lo, size_t i, float v) {
     const __nv_bfloat16 h = __float2bfloat16_rn(v);
@@ -32,15 +32,104 @@ __global__ void k_pf_embed(const WT *wte, const WT *wpe, int d, int vocab, const
 
 // Row t of the input is x[t][:] (+ bias + the split-K partial sums of the GEMM that produced it, added in a
 // fixed order; the completed row is then stored to x_store, which becomes the residual stream).  Followed by
-// LayerNorm / RMSNorm (skipped when gamma is null) and the hi/lo split (skipped when hi is null).  grid (T)
+// LayerNorm / RMSNorm (skipped when gamma is null) and the hi/lo split (skipped when hi is null).
+// grid (T, column slices): more than one slice only for the purely element-wise uses (no norm).  A thread keeps up
+// to PF_VPT float4 of its row in registers from the first load to the last store (rows of up to 16384 elements);
+// longer rows go through the plain loops at the end.
+constexpr int PF_VPT = 4;
+__device__ __forceinline__ void pf_split_store4(__nv_bfloat16 *hi, __nv_bfloat16 *lo, size_t i, const float4 v) {
+    const float f[4] = {v.x, v.y, v.z, v.w};
+    uint16_t h[4], l[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat16 hb = __float2bfloat16_rn(f[e]);
+        h[e] = __bfloat16_as_ushort(hb);
+        l[e] = __bfloat16_as_ushort(__float2bfloat16_rn(f[e] - __bfloat162float(hb)));
+    }
+    *reinterpret_cast<uint2 *>(hi + i) = make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
+    *reinterpret_cast<uint2 *>(lo + i) = make_uint2((uint32_t)l[0] | ((uint32_t)l[1] << 16), (uint32_t)l[2] | ((uint32_t)l[3] << 16));
+}
 __global__ void __launch_bounds__(PF_THREADS) k_pf_norm_split(const float *x, int n, int norm, const float *gamma, const float *beta,
                                                                float eps, __nv_bfloat16 *hi, __nv_bfloat16 *lo, const float *partial,
                                                                int n_split, int T, const float *bias, float *x_store) {
     pdl_launch_dependents();
     pdl_wait();
     __shared__ float red[2 * PF_THREADS / 32];
+    __shared__ float s_pilot;
     const int t = blockIdx.x, tid = threadIdx.x;
     const float *row = x + (size_t)t * n;
+    const int n4 = n >> 2;
+    if ((n & 3) == 0 && n4 <= PF_VPT * PF_THREADS) {
+        // this block's float4 columns: all of the row, or a slice of it (element-wise uses only)
+        const int per = (n4 + gridDim.y - 1) / gridDim.y, c_lo = blockIdx.y * per, c_hi = min(n4, c_lo + per);
+        float4 v[PF_VPT];
+#pragma unroll
+        for (int u = 0; u < PF_VPT; ++u) {
+            const int i4 = c_lo + tid + u * PF_THREADS;
+            v[u] = i4 < c_hi ? __ldcg(reinterpret_cast<const float4 *>(row) + i4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (n_split > 0) {
+#pragma unroll
+            for (int u = 0; u < PF_VPT; ++u) {
+                const int i4 = c_lo + tid + u * PF_THREADS;
+                if (i4 < c_hi && bias) { const float4 b = reinterpret_cast<const float4 *>(bias)[i4]; v[u].x += b.x; v[u].y += b.y; v[u].z += b.z; v[u].w += b.w; }
+            }
+            for (int z = 0; z < n_split; ++z) {
+                float4 p[PF_VPT];
+#pragma unroll
+                for (int u = 0; u < PF_VPT; ++u) {
+                    const int i4 = c_lo + tid + u * PF_THREADS;
+                    p[u] = i4 < c_hi ? __ldcg(reinterpret_cast<const float4 *>(partial + ((size_t)z * T + t) * n) + i4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int u = 0; u < PF_VPT; ++u) { v[u].x += p[u].x; v[u].y += p[u].y; v[u].z += p[u].z; v[u].w += p[u].w; }
+            }
+#pragma unroll
+            for (int u = 0; u < PF_VPT; ++u) {
+                const int i4 = c_lo + tid + u * PF_THREADS;
+                if (i4 < c_hi) reinterpret_cast<float4 *>(x_store + (size_t)t * n)[i4] = v[u];
+            }
+        }
+        if (!hi) return;
+        float mean = 0.f, rstd = 1.f;
+        if (gamma) { // (one slice: the block holds the whole row)
+            if (tid == 0) s_pilot = norm == NORM_LAYER ? v[0].x : 0.f;
+            __syncthreads();
+            const float pilot = s_pilot;
+            float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+            for (int u = 0; u < PF_VPT; ++u)
+                if (c_lo + tid + u * PF_THREADS < c_hi) {
+                    const float a = v[u].x - pilot, b = v[u].y - pilot, c2 = v[u].z - pilot, d2 = v[u].w - pilot;
+                    s1 += (a + b) + (c2 + d2);
+                    s2 += (a * a + b * b) + (c2 * c2 + d2 * d2);
+                }
+            s1 = warp_sum(s1);
+            s2 = warp_sum(s2);
+            if ((tid & 31) == 0) { red[tid >> 5] = s1; red[PF_THREADS / 32 + (tid >> 5)] = s2; }
+            __syncthreads();
+            s1 = s2 = 0.f;
+            for (int w = 0; w < PF_THREADS / 32; ++w) { s1 += red[w]; s2 += red[PF_THREADS / 32 + w]; }
+            const float dm = norm == NORM_LAYER ? s1 / (float)n : 0.f;
+            mean = pilot + dm;
+            rstd = rsqrtf(fmaxf(s2 / (float)n - dm * dm, 0.f) + eps);
+        }
+#pragma unroll
+        for (int u = 0; u < PF_VPT; ++u) {
+            const int i4 = c_lo + tid + u * PF_THREADS;
+            if (i4 >= c_hi) continue;
+            float4 y = v[u];
+            if (gamma) {
+                const float4 g = reinterpret_cast<const float4 *>(gamma)[i4];
+                y.x = (y.x - mean) * rstd * g.x; y.y = (y.y - mean) * rstd * g.y; y.z = (y.z - mean) * rstd * g.z; y.w = (y.w - mean) * rstd * g.w;
+                if (beta) { const float4 b = reinterpret_cast<const float4 *>(beta)[i4]; y.x += b.x; y.y += b.y; y.z += b.z; y.w += b.w; }
+            }
+            pf_split_store4(hi, lo, (size_t)t * n + 4 * (size_t)i4, y);
+        }
+        return;
+    }
+    // ---- long or odd rows: plain loops (one slice)
+    if (blockIdx.y != 0) return;
     if (n_split > 0) {
         float *dst = x_store + (size_t)t * n;
         for (int i = tid; i < n; i += PF_THREADS) {
