@@ -476,6 +476,9 @@ __global__ void __launch_bounds__(PK_THREADS, 1) k_persistent_decode(const PkPar
             for (int b = 0; b < NB; ++b) {
                 const bool live = b < nb;
                 const int slot = slots[b];
+                // columns past the row's end (up to the next multiple of 256) meet zero weights in the last chunk:
+                // they must be finite, whatever the shared memory held before
+                for (int i = Kd + tid; i < Kpad; i += PK_CTHREADS) xs[b * Kpad + xs_perm<ES>(i)] = 0.f;
                 // Common case (the source is a plain fp32 vector of at most 4096 elements: every phase but the
                 // embedding and the split merge): float4 loads, the values stay in registers through the norm
                 // statistics, and shared memory is written once.
