@@ -510,7 +510,7 @@ struct PfPending {
 // to add (pending must be non-null for matrices with d_model rows).
 int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, const float *bias, const float *resid, int act,
             float *y, __nv_bfloat16 *out_hi, __nv_bfloat16 *out_lo, PfPending *pending, cudaStream_t st) {
-    const int n_tile = T <= 16 ? 16 : T <= 32 ? 32 : T <= 64 ? 64 : 128;
+    const int n_tile = T <= TG_NT_PACKED ? TG_NT_PACKED : T <= 16 ? 16 : T <= 32 ? 32 : T <= 64 ? 64 : 128;
     const CUtensorMap *mw, *mhi, *mlo;
     int rc;
     if ((rc = pf_map(c, W, (uint64_t)n_rows, (uint64_t)K, TG_BM, &mw)) != MDI_OK) return rc;

@@ -25,10 +25,15 @@ constexpr int TG_MAX_NT = 128;  // positions per block (MMA N), a multiple of 16
 constexpr int TG_THREADS = 192;
 constexpr int TG_W_BYTES = TG_BM * TG_BK * 2;          // 16 KB per stage
 constexpr int TG_RING_BYTES = 196608;                  // operand ring for tiles of 64 or 128 positions (4 stages at 128)
-constexpr int TG_RING_BYTES_SMALL = 98304;             // for tiles of 16 or 32 positions (4 stages): two blocks fit on one SM,
+constexpr int TG_RING_BYTES_SMALL = 102400;            // for tiles of 16 (5 stages) or 32 positions (4 stages): two blocks fit on one SM,
                                                        // so GEMMs launched on different streams share SMs and overlap
+constexpr int TG_RING_BYTES_PACKED = 110592;           // for 8 positions (6 stages), two blocks per SM as well
+constexpr int TG_NT_PACKED = 8; // n_tile of the packed form: the hi rows and the lo rows of up to 8 positions make ONE 16-row B
+                                // operand (one MMA per k-step; columns j and j + 8 of the accumulator are added in the epilogue)
 constexpr size_t TG_SMEM = (size_t)TG_RING_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
-__host__ __device__ inline int tg_ring_bytes(int n_tile) { return n_tile <= 32 ? TG_RING_BYTES_SMALL : TG_RING_BYTES; }
+__host__ __device__ inline int tg_ring_bytes(int n_tile) {
+    return n_tile <= TG_NT_PACKED ? TG_RING_BYTES_PACKED : n_tile <= 32 ? TG_RING_BYTES_SMALL : TG_RING_BYTES;
+}
 __host__ __device__ inline size_t tg_smem_bytes(int n_tile) { return (size_t)tg_ring_bytes(n_tile) + 1024 + 256; }
 // bytes of one stage: a 128 x 64 weight tile and two n_tile x 64 input tiles (hi, lo); every part 1024-byte aligned
 __host__ __device__ inline int tg_stage_bytes(int n_tile) { return TG_W_BYTES + 2 * n_tile * TG_BK * 2; }
@@ -183,7 +188,8 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
     } else if (warp == 1) {
         if (lane == 0) {
             // ---- MMA issuer
-            const uint32_t idesc = tg_idesc(TG_BM, a.n_tile);
+            const bool packed = a.n_tile == TG_NT_PACKED;
+            const uint32_t idesc = tg_idesc(TG_BM, packed ? 16 : a.n_tile);
             bool ok = true;
             for (int kb = 0; kb < n_kb && ok; ++kb) {
                 const int s = kb % TG_STAGES;
@@ -195,7 +201,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 for (int k = 0; k < TG_BK / 16; ++k) {
                     const uint64_t ad = tg_desc(base + k * 32);
                     tg_mma(tmem_base, ad, tg_desc(base + TG_W_BYTES + k * 32), idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    tg_mma(tmem_base, ad, tg_desc(base + TG_W_BYTES + TG_X_BYTES + k * 32), idesc, 1u);
+                    if (!packed) tg_mma(tmem_base, ad, tg_desc(base + TG_W_BYTES + TG_X_BYTES + k * 32), idesc, 1u);
                 }
                 tg_commit(empty0 + 8 * s);      // the stage may be refilled once these MMAs have read it
             }
@@ -210,6 +216,7 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         const int row = m0 + lane_base + lane;
         const float bias = (a.bias && row < a.n_rows) ? a.bias[row] : 0.f;
         if (ok) {
+            const bool packed = a.n_tile == TG_NT_PACKED;
             for (int c = 0; c < a.n_tile; c += 16) {
                 uint32_t r[16];
                 const uint32_t taddr = tmem_base + ((uint32_t)lane_base << 16) + (uint32_t)c;
@@ -218,10 +225,14 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                                "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
                              : "r"(taddr) : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (packed) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r[j + 8]));
+                }
                 if (row < a.n_rows) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
-                        const int t = t0 + c + j;
+                        const int t = (packed && j >= 8) ? a.T : t0 + c + j;
                         if (t < a.T && gridDim.z > 1) {
                             a.partial[((size_t)blockIdx.z * a.T + t) * a.ldy + row] = __uint_as_float(r[j]);
                         } else if (t < a.T) {
