@@ -93,6 +93,9 @@ struct mdi_ctx {
     float *lnfg = nullptr, *lnfb = nullptr;
     std::map<std::string, TensorSlot> tensors;
     int n_loaded = 0;
+    // tensor-core linear layers: every matrix they multiply by also as contiguous 128 x 64 tiles (row-major pointer -> copy)
+    std::map<const void *, void *> w_tiled;
+    bool tiles_stale = true;
     float *rope_cos = nullptr, *rope_sin = nullptr;
     // output layers
     float *logits = nullptr; // [S][V]
@@ -513,15 +516,18 @@ int pf_gemm(mdi_ctx *c, Partition &P, const void *W, int n_rows, int K, int T, c
     const int n_tile = T <= TG_NT_PACKED ? TG_NT_PACKED : T <= 16 ? 16 : T <= 32 ? 32 : T <= 64 ? 64 : 128;
     const CUtensorMap *mw, *mhi, *mlo;
     int rc;
-    if ((rc = pf_map(c, W, (uint64_t)n_rows, (uint64_t)K, TG_BM, &mw)) != MDI_OK) return rc;
+    const int grid_x = (n_rows + TG_BM - 1) / TG_BM, n_kb = (K + TG_BK - 1) / TG_BK;
+    const auto tiled = c->w_tiled.find(W);
+    if (tiled != c->w_tiled.end()) rc = pf_map(c, tiled->second, (uint64_t)grid_x * n_kb * TG_BM, (uint64_t)TG_BK, TG_BM, &mw);
+    else rc = pf_map(c, W, (uint64_t)n_rows, (uint64_t)K, TG_BM, &mw);
+    if (rc != MDI_OK) return rc;
     if ((rc = pf_map(c, P.pf_hi, PF_CHUNK, (uint64_t)K, (uint32_t)n_tile, &mhi)) != MDI_OK) return rc;
     if ((rc = pf_map(c, P.pf_lo, PF_CHUNK, (uint64_t)K, (uint32_t)n_tile, &mlo)) != MDI_OK) return rc;
-    const int grid_x = (n_rows + TG_BM - 1) / TG_BM, n_kb = (K + TG_BK - 1) / TG_BK;
     int splits = 1;
     if (pending && 2 * grid_x <= c->n_sm) splits = std::max(1, std::min(std::min(PF_SPLIT_MAX, c->n_sm / grid_x), n_kb / 8));
     TgArgs a{};
     a.n_rows = n_rows; a.K = K; a.T = T; a.n_tile = n_tile; a.bias = bias; a.resid = resid; a.act = act; a.y = y; a.ldy = n_rows;
-    a.err = c->tg_err; a.partial = P.pf_part; a.out_hi = out_hi; a.out_lo = out_lo;
+    a.err = c->tg_err; a.w_tiled = tiled != c->w_tiled.end(); a.partial = P.pf_part; a.out_hi = out_hi; a.out_lo = out_lo;
     launch_k(c->pdl, k_tc_gemm, dim3(grid_x, (T + n_tile - 1) / n_tile, splits), dim3(TG_THREADS), tg_smem_bytes(n_tile), st, *mw, *mhi, *mlo, a);
     count_launch(c);
     if (pending) {
@@ -675,10 +681,45 @@ int pf_check(mdi_ctx *c) {
     return MDI_OK;
 }
 
+// (Re)build the tiled copies of the matrices of the tensor-core linear layers after weights were loaded.
+int pf_tile_weights(mdi_ctx *c) {
+    const mdi_model_shape &s = c->s;
+    const int d = s.d_model, F = s.d_ff, qw = s.n_head * s.head_dim, kw = s.n_kv_head * s.head_dim;
+    struct M { const void *w; int rows, K, part; };
+    std::vector<M> ms;
+    for (int p = 0; p < c->K; ++p)
+        for (int l = c->part[p].lo; l < c->part[p].hi; ++l) {
+            const LayerW &L = c->layer[l];
+            ms.push_back({L.wqkv, qw + 2 * kw, d, p});
+            ms.push_back({L.wo, d, qw, p});
+            ms.push_back({L.wgate, F, d, p});
+            ms.push_back({L.wup, F, d, p});
+            ms.push_back({L.wdown, d, F, p});
+            ms.push_back({L.w1, F, d, p});
+            ms.push_back({L.w2, d, F, p});
+        }
+    ms.push_back({s.tied_lm_head ? c->wte : c->lm_head, s.vocab, d, c->K - 1});
+    for (const M &m : ms) {
+        if (!m.w) continue;
+        const size_t n_chunks = (size_t)((m.rows + TG_BM - 1) / TG_BM) * ((m.K + TG_BK - 1) / TG_BK) * (TG_BM * TG_BK / 8);
+        void *&t = c->w_tiled[m.w];
+        if (!t) {
+            CU(cudaMalloc(&t, n_chunks * 16));
+            c->part[m.part].buffer_bytes += (int64_t)n_chunks * 16;
+        }
+        k_tile_weights<<<(unsigned)((n_chunks + 255) / 256), 256, 0, c->main>>>((const __nv_bfloat16 *)m.w, m.rows, m.K, (__nv_bfloat16 *)t, n_chunks);
+    }
+    CU(cudaStreamSynchronize(c->main));
+    CU(cudaGetLastError());
+    c->tiles_stale = false;
+    return MDI_OK;
+}
+
 int check_weights(mdi_ctx *c) {
-    if (c->n_loaded == (int)c->tensors.size()) return MDI_OK;
-    for (auto &kv : c->tensors)
-        if (!kv.second.loaded) return fail(c, MDI_ERR_STATE, "tensor '%s' was never loaded", kv.first.c_str());
+    if (c->n_loaded != (int)c->tensors.size())
+        for (auto &kv : c->tensors)
+            if (!kv.second.loaded) return fail(c, MDI_ERR_STATE, "tensor '%s' was never loaded", kv.first.c_str());
+    if (c->pf_tc && c->tiles_stale) return pf_tile_weights(c);
     return MDI_OK;
 }
 
@@ -1636,6 +1677,7 @@ void mdi_destroy(mdi_ctx *c) {
     cudaSetDevice(c->dev);
     cudaDeviceSynchronize();
     for (auto &g : c->graphs) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
+    for (auto &t : c->w_tiled) if (t.second) cudaFree(t.second);
     for (auto &t : c->tensors) {
         if (t.second.mat && *t.second.mat) cudaFree(*t.second.mat);
         if (t.second.vec && *t.second.vec) cudaFree(*t.second.vec);
@@ -1896,6 +1938,7 @@ int mdi_load_weights(mdi_ctx *c, const char *name, const void *host, size_t nbyt
     c->pk_tables_stale = true;
     c->fz_stale = true;
     c->td_stale = true;
+    c->tiles_stale = true;
     return MDI_OK;
 }
 

@@ -53,6 +53,7 @@ struct TgArgs {
     float *y;                 // [T][ldy]
     int ldy;
     int *err;                 // set to 1 when a wait gave up
+    int w_tiled;              // the weights come as contiguous 128 x 64 tiles [row tile][k-block][128][64] (k_tile_weights)
     float *partial;           // split-K (gridDim.z > 1): raw partial sums [z][T][ldy]; bias/resid/act/y are then unused
     __nv_bfloat16 *out_hi, *out_lo; // optional: the result also (or, with y null, only) as two bf16 planes [T][ldy]
 };
@@ -165,7 +166,8 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
             for (int kb = 0; kb < pre; ++kb) {
                 const uint32_t full = full0 + 8 * kb, base = tg_smem_u32(smem + (size_t)kb * TG_STAGE_BYTES);
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full), "r"(stage_bytes) : "memory");
-                tg_tma_2d(base, &tm_w, (kb_lo + kb) * TG_BK, m0, full);
+                if (a.w_tiled) tg_tma_2d(base, &tm_w, 0, (blockIdx.x * n_kb_all + kb_lo + kb) * TG_BM, full);
+                else tg_tma_2d(base, &tm_w, (kb_lo + kb) * TG_BK, m0, full);
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int kb = 0; kb < pre; ++kb) {
@@ -180,7 +182,8 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
                 const uint32_t full = full0 + 8 * s;
                 const uint32_t base = tg_smem_u32(smem + (size_t)s * TG_STAGE_BYTES);
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(full), "r"(stage_bytes) : "memory");
-                tg_tma_2d(base, &tm_w, (kb_lo + kb) * TG_BK, m0, full);
+                if (a.w_tiled) tg_tma_2d(base, &tm_w, 0, (blockIdx.x * n_kb_all + kb_lo + kb) * TG_BM, full);
+                else tg_tma_2d(base, &tm_w, (kb_lo + kb) * TG_BK, m0, full);
                 tg_tma_2d(base + TG_W_BYTES, &tm_xhi, (kb_lo + kb) * TG_BK, t0, full);
                 tg_tma_2d(base + TG_W_BYTES + TG_X_BYTES, &tm_xlo, (kb_lo + kb) * TG_BK, t0, full);
             }
@@ -257,6 +260,23 @@ k_tc_gemm(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUte
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
+}
+
+// Copy of a row-major bf16 matrix [n_rows][K] as contiguous tiles [ceil(n_rows / 128)][ceil(K / 64)][128][64], zero
+// outside the matrix: a block's weight tile is then one run of 16 KB in memory instead of 128 runs of 128 bytes a
+// row pitch apart.  One thread per 8 elements.
+__global__ void k_tile_weights(const __nv_bfloat16 *w, int n_rows, int K, __nv_bfloat16 *out, size_t n_chunks) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_chunks) return;
+    const int n_kb = (K + TG_BK - 1) / TG_BK;
+    const int c8 = (int)(i & 7), r = (int)((i >> 3) & (TG_BM - 1));
+    const size_t tile = i >> 10;
+    const int kb = (int)(tile % (size_t)n_kb), rt = (int)(tile / (size_t)n_kb);
+    const int row = rt * TG_BM + r, col = kb * TG_BK + c8 * 8;
+    __nv_bfloat16 v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = (row < n_rows && col + e < K) ? w[(size_t)row * K + col + e] : __float2bfloat16_rn(0.f);
+    *reinterpret_cast<uint4 *>(out + i * 8) = *reinterpret_cast<const uint4 *>(v);
 }
 
 // Host: 2-D tensor map over a row-major bf16 matrix [rows][cols] with a box of box_rows x 64 columns,
