@@ -45,7 +45,9 @@ NOMINAL_HBM_GBS = 8000.0
 # (algorithmic bytes) of the dominant kernel on a short capture.  Weights are ~90-99% of both and are read once per
 # group and pass, so traffic grows with the number of passes like the algorithmic bytes do.  None where no capture of
 # the current kernel exists.
-TRAFFIC_RATIO: dict = {}
+# llama_7b, stream scheduler: three consecutive k_tc_gemm launches on the workload's widths (8 positions, tiled weights)
+# read 226.1 MB and wrote 7.6 MB for 224.4 MB of matrices (profiles/stream_scheduler_llama_7b_launch_list.md).
+TRAFFIC_RATIO: dict = {("llama_7b", 0): 1.04, ("llama_7b", 1): 1.04}
 
 
 def measured_peaks():
