@@ -130,3 +130,26 @@ def test_a_withheld_handoff_times_out_and_the_context_survives():
         n = _safe_prefix(toks[s], margins[s], 1e-4)
         assert list(out[s, :n]) == toks[s][:n]
     ctx.close()
+
+
+def test_weights_loaded_again_replace_the_tiled_copies():
+    """The tensor-core linear layers read tiled copies of the matrices: loading other weights into the same context
+    must rebuild them (first visits and decode steps both on the tensor-core path)."""
+    from paper_2505_18164_b200 import mdi
+    shape = tiny_shape("llama", I.DT_BF16, L=2, d=256, H=2, V=300, C=40, n_kv=1)
+    prompts = I.make_prompts(300, 3, 9, seed=4)
+    ctx = mdi.Context(shape, [0, 1, 2], 3, scheduler=1, tc_min_group=1)
+    for seed in (3, 11):
+        orc, w = make_oracle(shape, seed=seed, std=0.04)
+        toks, lgs, margins = oracle_reference(orc, prompts, 6)
+        ctx.load_all(w)
+        for s in range(3):
+            ctx.reset_sample(s)
+            ctx.prefill(s, prompts[s])
+        out = ctx.generate(3, 6)
+        for s in range(3):
+            n = _safe_prefix(toks[s], margins[s], 3e-2)
+            assert list(out[s, :n]) == toks[s][:n], (seed, s)
+            if n == 6:
+                assert np.abs(ctx.get_logits(s) - lgs[s][5]).max() < 3e-2
+    ctx.close()
