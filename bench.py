@@ -251,7 +251,8 @@ def run_workload(w: I.Workload, args, steps: int, warmup: int, e2e_steps: int, w
     S, P, N = w.n_samples, w.n_prompt, w.n_new
     ctx = mdi.Context(s, list(w.part_bounds), S, kv_pool_tokens=S * ((P + N + 15) // 16 * 16), rounds_per_graph=args.rounds_per_graph,
                       scheduler=args.scheduler, tc_min_group=args.tc_min_group, kv_cache_dtype=args.kv_cache_dtype,
-                      in_kernel_timing=1 if args.in_kernel_timing else 0, td_b_kblocks=args.td_b_kblocks)
+                      in_kernel_timing=1 if args.in_kernel_timing else 0, td_b_kblocks=args.td_b_kblocks,
+                      fused_blocks_per_head=args.fused_blocks_per_head)
     weights = {}
     for name, a in I.iter_weights(s, w.weight_seed):
         ctx.load_weights(name, a)
@@ -367,6 +368,7 @@ def main():
     ap.add_argument("--kv-cache-dtype", type=int, default=0, help="0 library default, 1 bf16, 2 fp16, 3 fp32")
     ap.add_argument("--in-kernel-timing", action="store_true", help="persistent kernels time themselves; adds partition_times_ms "
                     "(per partition: blocks, milliseconds per category of the last generate call) to the line")
+    ap.add_argument("--fused-blocks-per-head", type=int, default=0, help="scheduler 3: 1 = one block per head (no clusters), 0 = library default")
     ap.add_argument("--td-b-kblocks", type=int, default=0, help="scheduler 4: k-blocks of the resident activation operand")
     ap.add_argument("--n-new", type=int, default=0, help="shorter generation (profiler captures only; not the headline)")
     ap.add_argument("--n-prompt", type=int, default=0, help="shorter prompts (profiler captures only)")
