@@ -152,7 +152,11 @@ void mdi_destroy(mdi_ctx *ctx);
  * "h.<i>.attn.bqkv", "h.<i>.attn.wo" [d][n_head head_dim], "h.<i>.attn.bo", "h.<i>.ln2.g",
  * "h.<i>.ln2.b", GPT: "h.<i>.mlp.w1" [d_ff][d], ".b1", ".w2" [d][d_ff], ".b2";
  * Llama: "h.<i>.mlp.wgate" [d_ff][d], ".wup" [d_ff][d], ".wdown" [d][d_ff].
- * The data is copied to the device before the call returns.
+ * The data is copied to the device before the call returns.  With bf16 weights (and prefill_mode != 1)
+ * the first mdi_prefill / mdi_step / mdi_generate after a load also builds, on the device, a second copy
+ * of every matrix of the blocks and of the output layer as contiguous 128 x 64 tiles for the tensor-core
+ * linear layers (device memory of those matrices doubles; counted by mdi_memory_bytes among the buffers of the
+ * partition that owns the matrix).
  * Errors: ARG (unknown name), SHAPE (nbytes mismatch), CUDA. */
 int mdi_load_weights(mdi_ctx *ctx, const char *tensor_name, const void *host_data, size_t nbytes);
 
